@@ -1,0 +1,186 @@
+/*
+ * apar.h - C ABI of the APAR decode hot path on one NVIDIA B200 (sm_100a).
+ *
+ * APAR (Auto-Parallel Auto-Regressive decoding) lets a model fork generation threads.
+ * A forked thread shares its parent's prefix; with a paged KV cache the fork shares all
+ * full blocks of the parent and copies at most one block (paper, Section 2.3 "Decoding").
+ * A new token attends only to the tokens on its path to the root of the paragraph tree,
+ * itself included (Section 2.2 "Training attention"; Section 2.4 feature 3).  When a
+ * thread finishes, the cache belonging only to it is released (Section 2.3; feature 2).
+ *
+ * This library owns the host-side bookkeeping (block tables, reference counts, free list)
+ * and launches the CUDA kernels for: the copy of the partial last block at fork, the
+ * scatter of new K/V rows into the pool, and the batched decode attention in which every
+ * shared block is read once for all threads and query heads that see it.
+ *
+ * Conventions
+ *   - Every pointer is tagged [host] or [device].  The caller owns all device memory (pool,
+ *     q, out, k_new, v_new, workspace) and the stream; the library owns host tables and
+ *     its pinned staging buffers.
+ *   - Calls return after enqueueing their kernels on `cuda_stream` (a cudaStream_t passed
+ *     as void*; NULL = the default stream).  Host bookkeeping is complete on return.  All
+ *     calls on one context must use streams that are ordered with respect to each other
+ *     (normally one stream); a context is not thread-safe.
+ *   - Batched calls process their entries in index order and are all-or-nothing: on any
+ *     error no host state changes and nothing is launched.
+ *   - No exceptions, aborts or device traps cross this boundary; errors are status codes.
+ *     There is no CPU fallback: without a usable CUDA device calls fail with APAR_ERR_CUDA.
+ *
+ * Layout of the KV pool (fixed): K pool and V pool are each
+ *       bf16 [num_blocks][num_kv_heads][block_size = 16][head_dim = 128],
+ *   so the rows of one (block, kv head) form a contiguous 4 KiB tile.  Q, out:
+ *   bf16 [n][num_q_heads][128].  k_new, v_new: bf16 [rows][num_kv_heads][128].
+ *   Query head h reads KV head h / (num_q_heads / num_kv_heads).
+ *
+ * Deterministic policy (the paper is silent; stated so that block ids are reproducible)
+ *   - Thread ids are handed out 0, 1, 2, ... and never reused.
+ *   - The free list is a stack.  A fresh pool hands out blocks 0, 1, 2, ...; released
+ *     blocks are pushed in table order and reused last-in first-out.
+ *   - Fork is eager: the CHILD receives a newly allocated block holding a copy of the
+ *     r = len mod 16 valid rows of the parent's partial last block; the parent keeps its
+ *     block and continues to append in place.  r = 0 copies nothing.  Rows r..15 of the
+ *     new block are unspecified and never read.
+ */
+#ifndef APAR_H_
+#define APAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct apar_ctx apar_ctx;   /* opaque; host state owned by the library */
+typedef int32_t apar_status;
+
+enum {
+  APAR_OK = 0,
+  APAR_ERR_INVALID_ARG = -1,          /* null pointer, negative count, duplicate id, bad shape   */
+  APAR_ERR_BAD_THREAD = -2,           /* unknown, released or (in release) repeated thread id     */
+  APAR_ERR_NO_BLOCKS = -3,            /* the pool cannot supply the blocks the whole call needs   */
+  APAR_ERR_NO_THREADS = -4,           /* more than max_threads live threads                       */
+  APAR_ERR_TABLE_FULL = -5,           /* a thread would exceed max_blocks_per_thread              */
+  APAR_ERR_EMPTY_CONTEXT = -6,        /* attention requested for a thread with no tokens          */
+  APAR_ERR_WORKSPACE_TOO_SMALL = -7,  /* workspace_bytes < apar_workspace_bytes(), or a plan that
+                                         does not fit the partial-result area                     */
+  APAR_ERR_CUDA = -8,                 /* a CUDA runtime call failed; see apar_last_cuda_error     */
+  APAR_ERR_UNSUPPORTED = -9           /* block_size != 16, head_dim != 128, heads not divisible   */
+};
+
+typedef struct {
+  int32_t num_blocks;             /* blocks in each of k_pool and v_pool                         */
+  int32_t block_size;             /* must be 16                                                  */
+  int32_t num_q_heads;
+  int32_t num_kv_heads;           /* must divide num_q_heads                                     */
+  int32_t head_dim;               /* must be 128                                                 */
+  int32_t max_threads;            /* live generation threads at any time                         */
+  int32_t max_blocks_per_thread;  /* longest chain, in blocks                                    */
+  void*   k_pool;                 /* [device] caller-owned, 1024-byte aligned                    */
+  void*   v_pool;                 /* [device] caller-owned, 1024-byte aligned                    */
+  void*   workspace;              /* [device] caller-owned scratch, 256-byte aligned             */
+  size_t  workspace_bytes;        /* >= apar_workspace_bytes(cfg)                                */
+} apar_config;
+
+typedef struct {
+  int64_t live_threads;
+  int64_t free_blocks;
+  int64_t used_blocks;
+  int64_t forks;                  /* threads created by apar_fork so far                         */
+  int64_t cow_blocks;             /* blocks copied by forks so far (<= forks)                    */
+  int64_t cow_rows;               /* token rows copied by forks so far                           */
+  /* the most recent attention call: */
+  int64_t attn_threads;           /* queries                                                     */
+  int64_t attn_attended_tokens;   /* sum of chain lengths ("attended tokens", Section 3.4)       */
+  int64_t attn_unique_tokens;     /* distinct KV token rows read (each shared row counted once)  */
+  int64_t attn_work_items;        /* (segment chunk) items, before the kv-head dimension         */
+  int64_t attn_partials;          /* partial (m, l, o) rows per query head written and merged    */
+  int64_t attn_kernels;           /* kernels launched by the call                                */
+  int64_t attn_plan_reused;       /* 1 if the cached plan of the previous call was reused        */
+  int64_t attn_vec_items;         /* items on the CUDA-core vector path                          */
+  int64_t attn_mma_items;         /* items on the tensor-core path                               */
+  int64_t kernels_total;          /* kernels launched by this context since creation             */
+} apar_stats;
+
+/* Bytes of device scratch a context with this configuration needs (pool pointers and the
+ * workspace fields are ignored).  Returns 0 for an unsupported configuration. */
+size_t apar_workspace_bytes(const apar_config* cfg /*[host]*/);
+
+/* Creates a context over an empty pool.  Allocates host memory and pinned staging only.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL, CUDA. */
+apar_status apar_create(const apar_config* cfg /*[host]*/, apar_ctx** out /*[host]*/);
+apar_status apar_destroy(apar_ctx* ctx);
+
+/* n new prompt sequences (roots of paragraph trees, Algorithm 1 "G <- {p}"): empty block
+ * tables, length 0.  tid_out [host] receives n ids.  Errors: NO_THREADS. */
+apar_status apar_new_threads(apar_ctx* ctx, int32_t n, int32_t* tid_out /*[host]*/);
+
+/* Fork (Algorithm 1 "s' <- s"; Section 2.3: "copies at most 1 KV cache block and shares all
+ * other blocks").  For each parent, in order: the child's table is the parent's first
+ * floor(len/16) block ids (their reference counts go up by one); if r = len mod 16 != 0 a
+ * block is taken from the free list and the r valid rows of the parent's last block (K and V,
+ * all KV heads) are copied into it by a kernel enqueued on the stream.  Child length = len.
+ * The same parent may appear several times.  child_tid_out [host] receives n ids.
+ * Errors: BAD_THREAD, NO_THREADS, NO_BLOCKS (needs one block per parent with r != 0). */
+apar_status apar_fork(apar_ctx* ctx, int32_t n, const int32_t* parent_tid /*[host]*/,
+                      int32_t* child_tid_out /*[host]*/, void* cuda_stream);
+
+/* KV append (Algorithm 1 "s.append_token(x)" and the K, V rows the model writes for it).
+ * Thread tid[i] receives n_tok[i] rows (n_tok NULL = one row each), taken consecutively from
+ * k_new / v_new [device] bf16 [sum n_tok][num_kv_heads][128].  A row at position p goes to
+ * slot p mod 16 of the thread's block p / 16; a block is allocated whenever p mod 16 == 0.
+ * Blocks are allocated in (entry, position) order.  Thread ids must be distinct.
+ * Errors: BAD_THREAD, INVALID_ARG, TABLE_FULL, NO_BLOCKS. */
+apar_status apar_append_kv(apar_ctx* ctx, int32_t n, const int32_t* tid /*[host]*/,
+                           const int32_t* n_tok /*[host] or NULL*/,
+                           const void* k_new /*[device]*/, const void* v_new /*[device]*/,
+                           void* cuda_stream);
+
+/* Tree decode attention (Section 2.2 "Training attention", Section 2.4 feature 3): for
+ * query i, owned by thread tid[i], and every query head h,
+ *     out[i][h] = softmax_j(sm_scale * <q[i][h], K_j>) . V_j
+ * over the len(tid[i]) tokens of that thread's chain (everything it inherited at its forks
+ * plus its own rows, the newest row included), KV head h / group.  bf16 in, fp32
+ * accumulation, bf16 out (round to nearest even).  Each physical block is read once per
+ * call for all queries and heads that share it.  A thread may be listed more than once;
+ * n <= max_threads.
+ * q [device] bf16 [n][num_q_heads][128]; out [device] same shape.
+ * Errors: INVALID_ARG, BAD_THREAD, EMPTY_CONTEXT, WORKSPACE_TOO_SMALL, CUDA. */
+apar_status apar_tree_decode_attention(apar_ctx* ctx, int32_t n, const int32_t* tid /*[host]*/,
+                                       const void* q /*[device]*/, void* out /*[device]*/,
+                                       float sm_scale, void* cuda_stream);
+
+/* ReleaseCache (Algorithm 1; Section 2.3: "the KV cache belonging only to s is released"):
+ * one reference is dropped per table entry, in table order; blocks reaching zero go back to
+ * the free list; the ids become invalid.  Errors: BAD_THREAD (also for a repeated id). */
+apar_status apar_release(apar_ctx* ctx, int32_t n, const int32_t* tid /*[host]*/);
+
+/* The same attention for a caller that keeps its own block tables (an external scheduler):
+ * block_tables [host] int32 [n_threads][max_blocks_per_thread] (row stride from cfg),
+ * ctx_lens [host] int32 [n_threads] tokens per query; n_threads <= cfg->max_threads.  Uses
+ * cfg->workspace for the whole call; no state survives it, and it returns only after its own
+ * host-to-device copies have completed (it synchronises the stream).  Blocks that appear in
+ * several rows are read once, provided they are full for every row that lists them.
+ * Errors: INVALID_ARG, UNSUPPORTED, EMPTY_CONTEXT, WORKSPACE_TOO_SMALL, CUDA. */
+apar_status apar_tree_decode_attention_tables(const apar_config* cfg /*[host]*/, int32_t n_threads,
+                                              const int32_t* block_tables /*[host]*/,
+                                              const int32_t* ctx_lens /*[host]*/,
+                                              const void* q /*[device]*/, void* out /*[device]*/,
+                                              float sm_scale, void* cuda_stream);
+
+/* Introspection (host state only; used to compare bookkeeping entry by entry). */
+apar_status apar_get_thread(apar_ctx* ctx, int32_t tid, int32_t* len, int32_t* n_blocks,
+                            int32_t* blocks /*[host] cap entries, may be NULL*/, int32_t cap);
+apar_status apar_get_refcounts(apar_ctx* ctx, int32_t* refcnt /*[host] [num_blocks]*/);
+/* ids in the order they will be handed out; n receives the count (<= cap are written). */
+apar_status apar_get_free_list(apar_ctx* ctx, int32_t* ids /*[host]*/, int32_t cap, int32_t* n);
+apar_status apar_get_stats(apar_ctx* ctx, apar_stats* out /*[host]*/);
+
+/* cudaError_t value of the most recent failing CUDA call of this context (0 if none). */
+int32_t     apar_last_cuda_error(apar_ctx* ctx);
+const char* apar_status_string(apar_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* APAR_H_ */

@@ -1,0 +1,184 @@
+"""ctypes binding of libapar.so: the same names and arguments as include/apar.h.
+
+Argument marshalling only.  Device buffers are passed as integer addresses (for example
+`tensor.data_ptr()`), host arrays as sequences of ints.  There is no fallback: if the
+library has not been built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libapar.so")
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_2401_06761_b200.build`")
+lib = C.CDLL(_LIB_PATH)
+
+APAR_OK = 0
+STATUS = {0: "OK", -1: "INVALID_ARG", -2: "BAD_THREAD", -3: "NO_BLOCKS", -4: "NO_THREADS",
+          -5: "TABLE_FULL", -6: "EMPTY_CONTEXT", -7: "WORKSPACE_TOO_SMALL", -8: "CUDA",
+          -9: "UNSUPPORTED"}
+
+
+class AparError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        self.code = STATUS.get(status, "UNKNOWN")
+        super().__init__(lib.apar_status_string(status).decode())
+
+
+class apar_config(C.Structure):
+    _fields_ = [("num_blocks", C.c_int32), ("block_size", C.c_int32),
+                ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("max_threads", C.c_int32),
+                ("max_blocks_per_thread", C.c_int32),
+                ("k_pool", C.c_void_p), ("v_pool", C.c_void_p),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
+
+
+class apar_stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in (
+        "live_threads", "free_blocks", "used_blocks", "forks", "cow_blocks", "cow_rows",
+        "attn_threads", "attn_attended_tokens", "attn_unique_tokens", "attn_work_items",
+        "attn_partials", "attn_kernels", "attn_plan_reused", "attn_vec_items",
+        "attn_mma_items", "kernels_total")]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+_i32p = C.POINTER(C.c_int32)
+_ctx = C.c_void_p
+_cfgp = C.POINTER(apar_config)
+
+_SIGS = {
+    "apar_workspace_bytes": (C.c_size_t, [_cfgp]),
+    "apar_create": (C.c_int32, [_cfgp, C.POINTER(_ctx)]),
+    "apar_destroy": (C.c_int32, [_ctx]),
+    "apar_new_threads": (C.c_int32, [_ctx, C.c_int32, _i32p]),
+    "apar_fork": (C.c_int32, [_ctx, C.c_int32, _i32p, _i32p, C.c_void_p]),
+    "apar_append_kv": (C.c_int32, [_ctx, C.c_int32, _i32p, _i32p, C.c_void_p, C.c_void_p,
+                                   C.c_void_p]),
+    "apar_tree_decode_attention": (C.c_int32, [_ctx, C.c_int32, _i32p, C.c_void_p, C.c_void_p,
+                                               C.c_float, C.c_void_p]),
+    "apar_release": (C.c_int32, [_ctx, C.c_int32, _i32p]),
+    "apar_tree_decode_attention_tables": (C.c_int32, [_cfgp, C.c_int32, _i32p, _i32p,
+                                                      C.c_void_p, C.c_void_p, C.c_float,
+                                                      C.c_void_p]),
+    "apar_get_thread": (C.c_int32, [_ctx, C.c_int32, _i32p, _i32p, _i32p, C.c_int32]),
+    "apar_get_refcounts": (C.c_int32, [_ctx, _i32p]),
+    "apar_get_free_list": (C.c_int32, [_ctx, _i32p, C.c_int32, _i32p]),
+    "apar_get_stats": (C.c_int32, [_ctx, C.POINTER(apar_stats)]),
+    "apar_last_cuda_error": (C.c_int32, [_ctx]),
+    "apar_status_string": (C.c_char_p, [C.c_int32]),
+}
+for _name, (_res, _args) in _SIGS.items():
+    _f = getattr(lib, _name)
+    _f.restype, _f.argtypes = _res, _args
+
+EXPORTS = tuple(_SIGS)
+
+
+def _arr(xs):
+    xs = list(xs)
+    return (C.c_int32 * len(xs))(*xs), len(xs)
+
+
+def _check(status: int):
+    if status != APAR_OK:
+        raise AparError(status)
+
+
+def make_config(num_blocks, num_q_heads, num_kv_heads, max_threads, max_blocks_per_thread,
+                k_pool=0, v_pool=0, workspace=0, workspace_bytes=0, block_size=16, head_dim=128):
+    return apar_config(num_blocks, block_size, num_q_heads, num_kv_heads, head_dim, max_threads,
+                       max_blocks_per_thread, k_pool, v_pool, workspace, workspace_bytes)
+
+
+def apar_workspace_bytes(cfg: apar_config) -> int:
+    return lib.apar_workspace_bytes(C.byref(cfg))
+
+
+def apar_create(cfg: apar_config):
+    ctx = _ctx()
+    _check(lib.apar_create(C.byref(cfg), C.byref(ctx)))
+    return ctx
+
+
+def apar_destroy(ctx):
+    _check(lib.apar_destroy(ctx))
+
+
+def apar_new_threads(ctx, n: int):
+    out = (C.c_int32 * max(n, 1))()
+    _check(lib.apar_new_threads(ctx, n, out))
+    return list(out[:n])
+
+
+def apar_fork(ctx, parent_tid, stream=0):
+    parents, n = _arr(parent_tid)
+    out = (C.c_int32 * max(n, 1))()
+    _check(lib.apar_fork(ctx, n, parents, out, stream))
+    return list(out[:n])
+
+
+def apar_append_kv(ctx, tid, n_tok, k_new: int, v_new: int, stream=0):
+    tids, n = _arr(tid)
+    counts = _arr(n_tok)[0] if n_tok is not None else None
+    _check(lib.apar_append_kv(ctx, n, tids, counts, k_new, v_new, stream))
+
+
+def apar_tree_decode_attention(ctx, tid, q: int, out: int, sm_scale: float, stream=0):
+    tids, n = tid if isinstance(tid, tuple) else _arr(tid)
+    _check(lib.apar_tree_decode_attention(ctx, n, tids, q, out, sm_scale, stream))
+
+
+def apar_release(ctx, tid):
+    tids, n = _arr(tid)
+    _check(lib.apar_release(ctx, n, tids))
+
+
+def apar_tree_decode_attention_tables(cfg, block_tables, ctx_lens, q: int, out: int,
+                                      sm_scale: float, stream=0):
+    """block_tables: n rows, each padded by the caller to cfg.max_blocks_per_thread ints."""
+    lens, n = _arr(ctx_lens)
+    flat, _ = _arr(x for row in block_tables for x in row)
+    _check(lib.apar_tree_decode_attention_tables(C.byref(cfg), n, flat, lens, q, out,
+                                                 sm_scale, stream))
+
+
+def apar_get_thread(ctx, tid: int, cap: int = 0):
+    """Returns (len, blocks)."""
+    ln, nb = C.c_int32(), C.c_int32()
+    _check(lib.apar_get_thread(ctx, tid, C.byref(ln), C.byref(nb), None, 0))
+    blocks = (C.c_int32 * max(nb.value, 1))()
+    _check(lib.apar_get_thread(ctx, tid, None, None, blocks, nb.value))
+    return ln.value, list(blocks[:nb.value])
+
+
+def apar_get_refcounts(ctx, num_blocks: int):
+    out = (C.c_int32 * num_blocks)()
+    _check(lib.apar_get_refcounts(ctx, out))
+    return list(out)
+
+
+def apar_get_free_list(ctx, num_blocks: int):
+    out = (C.c_int32 * max(num_blocks, 1))()
+    n = C.c_int32()
+    _check(lib.apar_get_free_list(ctx, out, num_blocks, C.byref(n)))
+    return list(out[:min(n.value, num_blocks)])
+
+
+def apar_get_stats(ctx) -> dict:
+    s = apar_stats()
+    _check(lib.apar_get_stats(ctx, C.byref(s)))
+    return s.as_dict()
+
+
+def apar_last_cuda_error(ctx) -> int:
+    return lib.apar_last_cuda_error(ctx)
+
+
+def int32_array(xs):
+    """Pre-marshalled id list for repeated calls of apar_tree_decode_attention."""
+    return _arr(xs)

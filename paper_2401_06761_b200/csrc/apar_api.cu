@@ -1,0 +1,667 @@
+// C-ABI entry points (include/apar.h): host bookkeeping of the paged pool, staging of
+// per-call metadata, and the launch sequence of each call.
+#include <algorithm>
+#include <climits>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/apar.h"
+#include "apar_internal.h"
+
+using namespace apar;
+
+namespace {
+
+constexpr int kRing = 4;              // pinned staging buffers in flight
+constexpr int kSlotsPerThread = 6;    // partial-result rows provisioned per live thread
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {            // partition of the caller's workspace
+  size_t tables, lens, stage, plan_items, plan_users, plan_merges, part_ml, part_o, total;
+  size_t stage_cap;        // bytes of the transient staging area
+  int64_t slot_capacity;   // partial rows (before the head dimension)
+  int64_t entry_capacity;  // (item, user) pairs a plan may hold
+};
+
+bool supported(const apar_config* c) {
+  return c && c->block_size == kBlock && c->head_dim == kDim && c->num_blocks > 0 &&
+         c->num_kv_heads > 0 && c->num_q_heads > 0 && c->num_q_heads % c->num_kv_heads == 0 &&
+         c->max_threads > 0 && c->max_blocks_per_thread > 0 &&
+         (int64_t)c->num_blocks * kBlock < INT32_MAX;
+}
+
+Layout make_layout(const apar_config* c) {
+  Layout L;
+  const size_t table_bytes = (size_t)c->max_threads * c->max_blocks_per_thread * 4;
+  L.slot_capacity = (int64_t)c->max_threads * kSlotsPerThread;
+  L.entry_capacity = L.slot_capacity + c->max_threads;
+  L.stage_cap = std::min<size_t>(std::max<size_t>(table_bytes / 4 + (64 << 10), 1 << 20), 64 << 20);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  L.tables = take(table_bytes);
+  L.lens = take((size_t)c->max_threads * 4);
+  L.stage = take(L.stage_cap);
+  L.plan_items = take((size_t)L.entry_capacity * sizeof(WorkItem));
+  L.plan_users = take((size_t)L.entry_capacity * sizeof(UserRef));
+  L.plan_merges = take((size_t)c->max_threads * sizeof(MergeRef));
+  L.part_ml = take((size_t)L.slot_capacity * c->num_q_heads * sizeof(float2));
+  L.part_o = take((size_t)L.slot_capacity * c->num_q_heads * kDim * sizeof(float));
+  L.total = off;
+  return L;
+}
+
+struct ThreadRec {
+  int32_t tid = -1;       // -1: slot free
+  int32_t len = 0;
+  int32_t n_blocks = 0;
+  int32_t synced = 0;     // table entries already on the device
+  int32_t dev_len = -1;   // length the device array holds for this slot
+};
+
+struct Staging {
+  char* host = nullptr;
+  cudaEvent_t done = nullptr;
+  bool in_flight = false;
+};
+
+}  // namespace
+
+struct apar_ctx {
+  apar_config cfg;
+  Shape shape;
+  Layout lay;
+  // ---- host bookkeeping
+  std::vector<int32_t> free_stack;     // top of the stack at the back
+  std::vector<int32_t> refcnt;
+  std::vector<int32_t> tables;         // [max_threads][max_blocks_per_thread] by slot
+  std::vector<ThreadRec> slots;
+  std::vector<int32_t> free_slots;
+  std::vector<int32_t> tid_slot;       // tid -> slot or -1
+  int32_t next_tid = 0;
+  int64_t live = 0;
+  int64_t forks = 0, cow_blocks = 0, cow_rows = 0, kernels_total = 0;
+  apar_stats last = {};
+  std::vector<uint32_t> mark;          // per slot, duplicate detection
+  uint32_t mark_epoch = 0;
+  // ---- staging
+  Staging ring[kRing];
+  size_t ring_bytes = 0;
+  int ring_next = 0;
+  // ---- planning
+  Planner planner;
+  Plan plan;
+  std::vector<PlanQuery> pq;
+  std::vector<int32_t> plan_tids;
+  uint64_t struct_epoch = 1, plan_epoch = 0;
+  int64_t plan_attended = 0;
+  int plan_age = 0;
+  int mma_min_rows = INT_MAX;
+  int32_t last_cuda = 0;
+  bool external_tables = false;        // the table-driven entry point owns no pool state
+
+  int32_t* row(int slot) { return tables.data() + (size_t)slot * cfg.max_blocks_per_thread; }
+  char* ws(size_t off) { return (char*)cfg.workspace + off; }
+};
+
+namespace {
+
+#define APAR_CUDA(ctx, expr)                         \
+  do {                                               \
+    cudaError_t e_ = (expr);                         \
+    if (e_ != cudaSuccess) {                         \
+      (ctx)->last_cuda = (int32_t)e_;                \
+      return APAR_ERR_CUDA;                          \
+    }                                                \
+  } while (0)
+
+// Next pinned buffer, once the copy that last used it has completed.
+apar_status acquire(apar_ctx* c, Staging** out) {
+  Staging* s = &c->ring[c->ring_next];
+  c->ring_next = (c->ring_next + 1) % kRing;
+  if (s->in_flight) {
+    APAR_CUDA(c, cudaEventSynchronize(s->done));
+    s->in_flight = false;
+  }
+  *out = s;
+  return APAR_OK;
+}
+
+apar_status send(apar_ctx* c, Staging* s, void* dst, size_t bytes, cudaStream_t st) {
+  if (bytes) APAR_CUDA(c, cudaMemcpyAsync(dst, s->host, bytes, cudaMemcpyHostToDevice, st));
+  APAR_CUDA(c, cudaEventRecord(s->done, st));
+  s->in_flight = true;
+  return APAR_OK;
+}
+
+int slot_of(apar_ctx* c, int32_t tid) {
+  if (tid < 0 || tid >= (int32_t)c->tid_slot.size()) return -1;
+  return c->tid_slot[tid];
+}
+
+uint32_t next_mark(apar_ctx* c) {
+  if (++c->mark_epoch == 0) {
+    std::fill(c->mark.begin(), c->mark.end(), 0u);
+    c->mark_epoch = 1;
+  }
+  return c->mark_epoch;
+}
+
+int32_t new_slot(apar_ctx* c) {
+  const int32_t s = c->free_slots.back();
+  c->free_slots.pop_back();
+  ThreadRec& t = c->slots[s];
+  t = ThreadRec();
+  t.tid = c->next_tid++;
+  c->tid_slot.push_back(s);
+  ++c->live;
+  return s;
+}
+
+int32_t alloc_block(apar_ctx* c) {
+  const int32_t b = c->free_stack.back();
+  c->free_stack.pop_back();
+  c->refcnt[b] = 1;
+  return b;
+}
+
+// Brings the device copies of block tables and lengths up to date for the given slots.
+apar_status sync_device_tables(apar_ctx* c, const int32_t* slots, int n, cudaStream_t st) {
+  int i = 0;
+  while (i < n) {
+    Staging* s;
+    apar_status rc = acquire(c, &s);
+    if (rc) return rc;
+    // layout inside the staging area: [deltas][pairs][data]; sized so that all three fit
+    const size_t cap = c->lay.stage_cap;
+    const int max_entries = (int)std::min<size_t>(cap / 4 / sizeof(TableDelta), 1 << 20);
+    TableDelta* deltas = (TableDelta*)s->host;
+    int32_t* pairs = (int32_t*)(s->host + (size_t)max_entries * sizeof(TableDelta));
+    int32_t* data = pairs + 2 * (size_t)max_entries;
+    const size_t data_cap = (cap - ((char*)data - s->host)) / 4;
+    int nd = 0, np = 0;
+    size_t used = 0;
+    const uint32_t mk = next_mark(c);
+    for (; i < n; ++i) {
+      ThreadRec& t = c->slots[slots[i]];
+      if (c->mark[slots[i]] == mk) continue;           // listed twice in this round
+      const int need = t.n_blocks - t.synced;
+      if (need > 0 && (nd >= max_entries || used + need > data_cap)) break;
+      if (t.dev_len != t.len && np >= max_entries) break;
+      c->mark[slots[i]] = mk;
+      if (need > 0) {
+        deltas[nd++] = TableDelta{slots[i], t.synced, need, (int32_t)used};
+        memcpy(data + used, c->row(slots[i]) + t.synced, (size_t)need * 4);
+        used += need;
+        t.synced = t.n_blocks;
+      }
+      if (t.dev_len != t.len) {
+        pairs[2 * np] = slots[i];
+        pairs[2 * np + 1] = t.len;
+        ++np;
+        t.dev_len = t.len;
+      }
+    }
+    if (nd == 0 && np == 0) {
+      if (i < n) return APAR_ERR_WORKSPACE_TOO_SMALL;   // one row larger than the staging area
+      break;
+    }
+    const size_t bytes = ((char*)(data + used)) - s->host;
+    char* d_stage = c->ws(c->lay.stage);
+    rc = send(c, s, d_stage, bytes, st);
+    if (rc) return rc;
+    APAR_CUDA(c, launch_sync((int32_t*)c->ws(c->lay.tables), c->cfg.max_blocks_per_thread,
+                             (int32_t*)c->ws(c->lay.lens), (const TableDelta*)d_stage,
+                             (const int32_t*)(d_stage + ((char*)data - s->host)), nd,
+                             (const int32_t*)(d_stage + ((char*)pairs - s->host)), np, st));
+    ++c->kernels_total;
+    ++c->last.attn_kernels;
+  }
+  return APAR_OK;
+}
+
+// The attention launch sequence for queries given as slots (already validated, len > 0).
+apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32_t* tids,
+                          bool has_dups, const void* q, void* out, float sm_scale,
+                          cudaStream_t st) {
+  c->last.attn_kernels = 0;
+  int64_t attended = 0;
+  for (int i = 0; i < n; ++i) attended += c->slots[qslots[i]].len;
+
+  const bool cacheable = tids != nullptr && !has_dups;
+  bool reuse = cacheable && c->plan_epoch == c->struct_epoch && c->plan_age < 64 &&
+               (int)c->plan_tids.size() == n &&
+               memcmp(c->plan_tids.data(), tids, (size_t)n * 4) == 0 &&
+               attended - c->plan_attended < c->plan_attended / 4 + 64;
+  if (!reuse) {
+    c->pq.resize(n);
+    for (int i = 0; i < n; ++i)
+      c->pq[i] = PlanQuery{c->row(qslots[i]), qslots[i], c->slots[qslots[i]].len};
+    if (!c->planner.build(c->pq.data(), n, c->lay.slot_capacity, cacheable, c->mma_min_rows,
+                          &c->plan))
+      return APAR_ERR_WORKSPACE_TOO_SMALL;
+    if ((int64_t)c->plan.users.size() > c->lay.entry_capacity ||
+        (int64_t)c->plan.items.size() > c->lay.entry_capacity)
+      return APAR_ERR_WORKSPACE_TOO_SMALL;
+  }
+  apar_status rc = sync_device_tables(c, qslots, n, st);
+  if (rc) return rc;
+
+  const Plan& p = c->plan;
+  if (!reuse) {
+    const size_t b_items = p.items.size() * sizeof(WorkItem);
+    const size_t b_users = p.users.size() * sizeof(UserRef);
+    const size_t b_merges = p.merges.size() * sizeof(MergeRef);
+    struct Part { const void* src; size_t bytes, dst; } parts[3] = {
+        {p.items.data(), b_items, c->lay.plan_items},
+        {p.users.data(), b_users, c->lay.plan_users},
+        {p.merges.data(), b_merges, c->lay.plan_merges}};
+    for (const Part& part : parts) {
+      size_t done = 0;
+      while (done < part.bytes) {
+        Staging* s;
+        rc = acquire(c, &s);
+        if (rc) return rc;
+        const size_t chunk = std::min(part.bytes - done, c->ring_bytes);
+        memcpy(s->host, (const char*)part.src + done, chunk);
+        rc = send(c, s, c->ws(part.dst) + done, chunk, st);
+        if (rc) return rc;
+        done += chunk;
+      }
+    }
+    if (cacheable) {
+      c->plan_tids.assign(tids, tids + n);
+      c->plan_epoch = c->struct_epoch;
+      c->plan_attended = attended;
+      c->plan_age = 0;
+    } else {
+      c->plan_epoch = 0;
+    }
+  } else {
+    ++c->plan_age;
+  }
+
+  AttnArgs a;
+  a.q = q;
+  a.out = out;
+  a.k_pool = c->cfg.k_pool;
+  a.v_pool = c->cfg.v_pool;
+  a.d_tables = (const int32_t*)c->ws(c->lay.tables);
+  a.d_lens = (const int32_t*)c->ws(c->lay.lens);
+  a.d_items = (const WorkItem*)c->ws(c->lay.plan_items);
+  a.d_users = (const UserRef*)c->ws(c->lay.plan_users);
+  a.part_o = (float*)c->ws(c->lay.part_o);
+  a.part_ml = (float2*)c->ws(c->lay.part_ml);
+  a.shape = c->shape;
+  a.scale_log2e = sm_scale * 1.4426950408889634f;
+  int launches = 0;
+  if (p.n_mma) {
+    APAR_CUDA(c, launch_attention_mma(a, p.n_vec, p.n_mma, st));
+    ++launches;
+  }
+  if (p.n_vec) {
+    APAR_CUDA(c, launch_attention_vec(a, 0, p.n_vec, c->shape.group == 1 && c->mma_min_rows <= 2, st));
+    ++launches;
+  }
+  if (!p.merges.empty()) {
+    APAR_CUDA(c, launch_merge(a, (const MergeRef*)c->ws(c->lay.plan_merges),
+                              (int)p.merges.size(), st));
+    ++launches;
+  }
+  c->kernels_total += launches;
+  c->last.attn_kernels += launches;
+  c->last.attn_threads = n;
+  c->last.attn_attended_tokens = attended;
+  c->last.attn_unique_tokens = p.unique_tokens + (reuse ? attended - c->plan_attended : 0);
+  c->last.attn_work_items = (int64_t)p.items.size();
+  c->last.attn_partials = p.total_slots * c->shape.num_q_heads;
+  c->last.attn_plan_reused = reuse ? 1 : 0;
+  c->last.attn_vec_items = p.n_vec;
+  c->last.attn_mma_items = p.n_mma;
+  return APAR_OK;
+}
+
+apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
+  if (!cfg || !out) return APAR_ERR_INVALID_ARG;
+  if (!supported(cfg)) return APAR_ERR_UNSUPPORTED;
+  if (!cfg->k_pool || !cfg->v_pool || !cfg->workspace) return APAR_ERR_INVALID_ARG;
+  if (((uintptr_t)cfg->k_pool | (uintptr_t)cfg->v_pool) & 1023) return APAR_ERR_INVALID_ARG;
+  if ((uintptr_t)cfg->workspace & 255) return APAR_ERR_INVALID_ARG;
+  const Layout lay = make_layout(cfg);
+  if (cfg->workspace_bytes < lay.total) return APAR_ERR_WORKSPACE_TOO_SMALL;
+  apar_ctx* c = new (std::nothrow) apar_ctx();
+  if (!c) return APAR_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->lay = lay;
+  c->shape = Shape{cfg->num_q_heads, cfg->num_kv_heads, cfg->num_q_heads / cfg->num_kv_heads,
+                   cfg->max_blocks_per_thread};
+  c->external_tables = external;
+  c->refcnt.assign(cfg->num_blocks, 0);
+  c->free_stack.resize(cfg->num_blocks);
+  for (int i = 0; i < cfg->num_blocks; ++i) c->free_stack[i] = cfg->num_blocks - 1 - i;
+  c->tables.assign((size_t)cfg->max_threads * cfg->max_blocks_per_thread, 0);
+  c->slots.assign(cfg->max_threads, ThreadRec());
+  c->free_slots.resize(cfg->max_threads);
+  for (int i = 0; i < cfg->max_threads; ++i) c->free_slots[i] = cfg->max_threads - 1 - i;
+  c->mark.assign(cfg->max_threads, 0);
+  c->planner.init(cfg->num_blocks, c->shape.group, cfg->num_kv_heads);
+  const char* path = getenv("APAR_ATTN_PATH");     // "vec": CUDA-core kernel for every item
+  c->mma_min_rows = (path && !strcmp(path, "vec")) ? INT_MAX : 2;
+  c->ring_bytes = lay.stage_cap;
+  for (int i = 0; i < kRing; ++i) {
+    cudaError_t e = cudaMallocHost((void**)&c->ring[i].host, c->ring_bytes);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ring[i].done, cudaEventDisableTiming);
+    if (e != cudaSuccess) {
+      apar_destroy(c);
+      return APAR_ERR_CUDA;
+    }
+  }
+  *out = c;
+  return APAR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t apar_workspace_bytes(const apar_config* cfg) {
+  if (!supported(cfg)) return 0;
+  return make_layout(cfg).total;
+}
+
+apar_status apar_create(const apar_config* cfg, apar_ctx** out) {
+  return create_impl(cfg, false, out);
+}
+
+apar_status apar_destroy(apar_ctx* c) {
+  if (!c) return APAR_ERR_INVALID_ARG;
+  for (int i = 0; i < kRing; ++i) {
+    if (c->ring[i].in_flight) cudaEventSynchronize(c->ring[i].done);
+    if (c->ring[i].done) cudaEventDestroy(c->ring[i].done);
+    if (c->ring[i].host) cudaFreeHost(c->ring[i].host);
+  }
+  delete c;
+  return APAR_OK;
+}
+
+apar_status apar_new_threads(apar_ctx* c, int32_t n, int32_t* tid_out) {
+  if (!c || n < 0 || (n > 0 && !tid_out)) return APAR_ERR_INVALID_ARG;
+  if (c->live + n > c->cfg.max_threads) return APAR_ERR_NO_THREADS;
+  for (int i = 0; i < n; ++i) tid_out[i] = c->slots[new_slot(c)].tid;
+  if (n) ++c->struct_epoch;
+  return APAR_OK;
+}
+
+apar_status apar_fork(apar_ctx* c, int32_t n, const int32_t* parent_tid, int32_t* child_tid_out,
+                      void* cuda_stream) {
+  if (!c || n < 0 || (n > 0 && (!parent_tid || !child_tid_out))) return APAR_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int need = 0;
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, parent_tid[i]);
+    if (s < 0) return APAR_ERR_BAD_THREAD;
+    if (c->slots[s].len % kBlock) ++need;
+  }
+  if (c->live + n > c->cfg.max_threads) return APAR_ERR_NO_THREADS;
+  if (need > (int)c->free_stack.size()) return APAR_ERR_NO_BLOCKS;
+  if ((size_t)need * sizeof(CowCopy) > c->lay.stage_cap) return APAR_ERR_WORKSPACE_TOO_SMALL;
+  Staging* stg = nullptr;
+  if (need) {
+    apar_status rc = acquire(c, &stg);
+    if (rc) return rc;
+  }
+  CowCopy* copies = stg ? (CowCopy*)stg->host : nullptr;
+  int nc = 0;
+  for (int i = 0; i < n; ++i) {
+    const int ps = slot_of(c, parent_tid[i]);
+    const int32_t L = c->slots[ps].len, full = L / kBlock, r = L % kBlock;
+    const int cs = new_slot(c);
+    ThreadRec& ch = c->slots[cs];
+    int32_t* ct = c->row(cs);
+    const int32_t* pt = c->row(ps);
+    for (int b = 0; b < full; ++b) {
+      ct[b] = pt[b];
+      ++c->refcnt[pt[b]];
+    }
+    ch.n_blocks = full;
+    if (r) {
+      const int32_t dst = alloc_block(c);
+      copies[nc++] = CowCopy{pt[full], dst, r, 0};
+      ct[full] = dst;
+      ch.n_blocks = full + 1;
+      ++c->cow_blocks;
+      c->cow_rows += r;
+    }
+    ch.len = L;
+    child_tid_out[i] = ch.tid;
+    ++c->forks;
+  }
+  if (n) ++c->struct_epoch;
+  if (nc) {
+    char* d_stage = c->ws(c->lay.stage);
+    apar_status rc = send(c, stg, d_stage, (size_t)nc * sizeof(CowCopy), st);
+    if (rc) return rc;
+    APAR_CUDA(c, launch_cow_copy(c->cfg.k_pool, c->cfg.v_pool, (const CowCopy*)d_stage, nc,
+                                 c->cfg.num_kv_heads, st));
+    ++c->kernels_total;
+  }
+  return APAR_OK;
+}
+
+apar_status apar_append_kv(apar_ctx* c, int32_t n, const int32_t* tid, const int32_t* n_tok,
+                           const void* k_new, const void* v_new, void* cuda_stream) {
+  if (!c || n < 0 || (n > 0 && (!tid || !k_new || !v_new))) return APAR_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  for (int i = 0; i < n; ++i)
+    if (slot_of(c, tid[i]) < 0) return APAR_ERR_BAD_THREAD;
+  const uint32_t mk = next_mark(c);
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, tid[i]);
+    if (c->mark[s] == mk || (n_tok && n_tok[i] < 0)) return APAR_ERR_INVALID_ARG;
+    c->mark[s] = mk;
+  }
+  int64_t need = 0, rows = 0;
+  for (int i = 0; i < n; ++i) {
+    const ThreadRec& t = c->slots[slot_of(c, tid[i])];
+    const int64_t cnt = n_tok ? n_tok[i] : 1;
+    const int64_t after = (t.len + cnt + kBlock - 1) / kBlock;
+    if (after > c->cfg.max_blocks_per_thread) return APAR_ERR_TABLE_FULL;
+    need += after - t.n_blocks;
+    rows += cnt;
+  }
+  if (need > (int64_t)c->free_stack.size()) return APAR_ERR_NO_BLOCKS;
+  if (rows > INT32_MAX) return APAR_ERR_INVALID_ARG;
+  // bookkeeping and slot list, streamed to the device in staging-sized pieces
+  const size_t cap_rows = c->lay.stage_cap / 4;
+  Staging* stg = nullptr;
+  int32_t* slots = nullptr;
+  size_t filled = 0;
+  int64_t first_row = 0;
+  auto flush = [&]() -> apar_status {
+    if (!filled) return APAR_OK;
+    char* d_stage = c->ws(c->lay.stage);
+    apar_status rc = send(c, stg, d_stage, filled * 4, st);
+    if (rc) return rc;
+    APAR_CUDA(c, launch_append(c->cfg.k_pool, c->cfg.v_pool, k_new, v_new,
+                               (const int32_t*)d_stage, first_row, (int)filled,
+                               c->cfg.num_kv_heads, st));
+    ++c->kernels_total;
+    first_row += (int64_t)filled;
+    filled = 0;
+    stg = nullptr;
+    return APAR_OK;
+  };
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, tid[i]);
+    ThreadRec& t = c->slots[s];
+    int32_t* tab = c->row(s);
+    const int cnt = n_tok ? n_tok[i] : 1;
+    for (int k = 0; k < cnt; ++k) {
+      const int32_t pos = t.len;
+      if (pos % kBlock == 0) {
+        // a thread without a private tail gains one: cached plans no longer describe it
+        if (t.n_blocks == 0 || c->refcnt[tab[t.n_blocks - 1]] > 1) ++c->struct_epoch;
+        tab[t.n_blocks++] = alloc_block(c);
+      }
+      if (!stg) {
+        apar_status rc = acquire(c, &stg);
+        if (rc) return rc;   // bookkeeping of earlier rows stands; the CUDA error is sticky
+        slots = (int32_t*)stg->host;
+      }
+      slots[filled++] = tab[pos / kBlock] * kBlock + pos % kBlock;
+      t.len = pos + 1;
+      if (filled == cap_rows) {
+        apar_status rc = flush();
+        if (rc) return rc;
+      }
+    }
+  }
+  return flush();
+}
+
+apar_status apar_tree_decode_attention(apar_ctx* c, int32_t n, const int32_t* tid, const void* q,
+                                       void* out, float sm_scale, void* cuda_stream) {
+  if (!c || n < 0 || n > c->cfg.max_threads || (n > 0 && (!tid || !q || !out)))
+    return APAR_ERR_INVALID_ARG;
+  if (n == 0) return APAR_OK;
+  std::vector<int32_t> qslots(n);
+  const uint32_t mk = next_mark(c);
+  bool dups = false;
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, tid[i]);
+    if (s < 0) return APAR_ERR_BAD_THREAD;
+    qslots[i] = s;
+  }
+  for (int i = 0; i < n; ++i) {
+    if (c->slots[qslots[i]].len == 0) return APAR_ERR_EMPTY_CONTEXT;
+    if (c->mark[qslots[i]] == mk) dups = true;
+    c->mark[qslots[i]] = mk;
+  }
+  return run_attention(c, n, qslots.data(), tid, dups, q, out, sm_scale,
+                       (cudaStream_t)cuda_stream);
+}
+
+apar_status apar_release(apar_ctx* c, int32_t n, const int32_t* tid) {
+  if (!c || n < 0 || (n > 0 && !tid)) return APAR_ERR_INVALID_ARG;
+  const uint32_t mk = next_mark(c);
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, tid[i]);
+    if (s < 0 || c->mark[s] == mk) return APAR_ERR_BAD_THREAD;
+    c->mark[s] = mk;
+  }
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, tid[i]);
+    ThreadRec& t = c->slots[s];
+    const int32_t* tab = c->row(s);
+    for (int b = 0; b < t.n_blocks; ++b)
+      if (--c->refcnt[tab[b]] == 0) c->free_stack.push_back(tab[b]);
+    c->tid_slot[tid[i]] = -1;
+    t = ThreadRec();
+    c->free_slots.push_back(s);
+    --c->live;
+  }
+  if (n) ++c->struct_epoch;
+  return APAR_OK;
+}
+
+apar_status apar_tree_decode_attention_tables(const apar_config* cfg, int32_t n,
+                                              const int32_t* block_tables, const int32_t* ctx_lens,
+                                              const void* q, void* out, float sm_scale,
+                                              void* cuda_stream) {
+  if (!cfg || n < 0 || (n > 0 && (!block_tables || !ctx_lens || !q || !out)))
+    return APAR_ERR_INVALID_ARG;
+  if (!supported(cfg)) return APAR_ERR_UNSUPPORTED;
+  if (n > cfg->max_threads) return APAR_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    if (ctx_lens[i] < 0) return APAR_ERR_INVALID_ARG;
+    if (ctx_lens[i] == 0) return APAR_ERR_EMPTY_CONTEXT;
+    const int nb = (ctx_lens[i] + kBlock - 1) / kBlock;
+    if (nb > cfg->max_blocks_per_thread) return APAR_ERR_INVALID_ARG;
+    for (int b = 0; b < nb; ++b) {
+      const int32_t id = block_tables[(size_t)i * cfg->max_blocks_per_thread + b];
+      if (id < 0 || id >= cfg->num_blocks) return APAR_ERR_INVALID_ARG;
+    }
+  }
+  if (n == 0) return APAR_OK;
+  apar_ctx* c = nullptr;
+  apar_status rc = create_impl(cfg, true, &c);
+  if (rc) return rc;
+  std::vector<int32_t> qslots(n);
+  for (int i = 0; i < n; ++i) {
+    ThreadRec& t = c->slots[i];
+    t.tid = i;
+    t.len = ctx_lens[i];
+    t.n_blocks = (t.len + kBlock - 1) / kBlock;
+    memcpy(c->row(i), block_tables + (size_t)i * cfg->max_blocks_per_thread,
+           (size_t)t.n_blocks * 4);
+    qslots[i] = i;
+  }
+  rc = run_attention(c, n, qslots.data(), nullptr, false, q, out, sm_scale,
+                     (cudaStream_t)cuda_stream);
+  if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess && rc == APAR_OK)
+    rc = APAR_ERR_CUDA;
+  apar_destroy(c);
+  return rc;
+}
+
+apar_status apar_get_thread(apar_ctx* c, int32_t tid, int32_t* len, int32_t* n_blocks,
+                            int32_t* blocks, int32_t cap) {
+  if (!c) return APAR_ERR_INVALID_ARG;
+  const int s = slot_of(c, tid);
+  if (s < 0) return APAR_ERR_BAD_THREAD;
+  const ThreadRec& t = c->slots[s];
+  if (len) *len = t.len;
+  if (n_blocks) *n_blocks = t.n_blocks;
+  if (blocks) memcpy(blocks, c->row(s), (size_t)std::max(0, std::min(cap, t.n_blocks)) * 4);
+  return APAR_OK;
+}
+
+apar_status apar_get_refcounts(apar_ctx* c, int32_t* refcnt) {
+  if (!c || !refcnt) return APAR_ERR_INVALID_ARG;
+  memcpy(refcnt, c->refcnt.data(), c->refcnt.size() * 4);
+  return APAR_OK;
+}
+
+apar_status apar_get_free_list(apar_ctx* c, int32_t* ids, int32_t cap, int32_t* n) {
+  if (!c || !n || cap < 0 || (cap > 0 && !ids)) return APAR_ERR_INVALID_ARG;
+  const int32_t total = (int32_t)c->free_stack.size();
+  *n = total;
+  for (int i = 0; i < std::min(cap, total); ++i) ids[i] = c->free_stack[total - 1 - i];
+  return APAR_OK;
+}
+
+apar_status apar_get_stats(apar_ctx* c, apar_stats* out) {
+  if (!c || !out) return APAR_ERR_INVALID_ARG;
+  *out = c->last;
+  out->live_threads = c->live;
+  out->free_blocks = (int64_t)c->free_stack.size();
+  out->used_blocks = c->cfg.num_blocks - out->free_blocks;
+  out->forks = c->forks;
+  out->cow_blocks = c->cow_blocks;
+  out->cow_rows = c->cow_rows;
+  out->kernels_total = c->kernels_total;
+  return APAR_OK;
+}
+
+int32_t apar_last_cuda_error(apar_ctx* c) { return c ? c->last_cuda : 0; }
+
+const char* apar_status_string(apar_status s) {
+  switch (s) {
+    case APAR_OK: return "APAR_OK";
+    case APAR_ERR_INVALID_ARG: return "APAR_ERR_INVALID_ARG";
+    case APAR_ERR_BAD_THREAD: return "APAR_ERR_BAD_THREAD";
+    case APAR_ERR_NO_BLOCKS: return "APAR_ERR_NO_BLOCKS";
+    case APAR_ERR_NO_THREADS: return "APAR_ERR_NO_THREADS";
+    case APAR_ERR_TABLE_FULL: return "APAR_ERR_TABLE_FULL";
+    case APAR_ERR_EMPTY_CONTEXT: return "APAR_ERR_EMPTY_CONTEXT";
+    case APAR_ERR_WORKSPACE_TOO_SMALL: return "APAR_ERR_WORKSPACE_TOO_SMALL";
+    case APAR_ERR_CUDA: return "APAR_ERR_CUDA";
+    case APAR_ERR_UNSUPPORTED: return "APAR_ERR_UNSUPPORTED";
+    default: return "APAR_ERR_UNKNOWN";
+  }
+}
+
+}  // extern "C"

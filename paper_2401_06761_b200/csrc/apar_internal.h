@@ -1,0 +1,128 @@
+// Internal declarations shared by the host side (bookkeeping, planner) and the kernel
+// launchers.  Not part of the public boundary (include/apar.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include <vector>
+
+namespace apar {
+
+constexpr int kBlock = 16;      // tokens per KV block
+constexpr int kDim = 128;       // head dimension
+constexpr int kTileBytes = kBlock * kDim * 2;   // one (block, kv head) tile of K or of V
+constexpr int kMaxRowsPerItem = 64;             // query rows one work item may carry
+
+// One unit of attention work: a run of consecutive blocks of one table row, read once for
+// every (query, head-in-group) row that shares it.  The kv head is the second grid dimension.
+struct WorkItem {
+  int32_t table_row;   // row of the device block table to walk
+  int32_t tok_begin;   // first token of the run in chain coordinates (multiple of 16)
+  int32_t tok_end;     // one past the last token; < 0: "the current length of table_row"
+  int32_t user_begin;  // first entry of this item's users in the UserRef array
+  int32_t n_users;     // queries sharing the run (rows = n_users * group)
+  int32_t slot_add;    // added to every user's partial slot (chunk ordinal inside the run)
+  int32_t pad0, pad1;
+};
+
+// A query that reads a work item.  slot < 0: the item covers the query's whole chain and
+// writes the final output; otherwise partial row (slot + item.slot_add) receives (m, l, o).
+struct UserRef {
+  int32_t query;
+  int32_t slot;
+};
+
+// A query whose chain was covered by n >= 2 items: merge partial slots [slot_begin, +n).
+struct MergeRef {
+  int32_t query;
+  int32_t slot_begin;
+  int32_t n;
+  int32_t pad;
+};
+
+// A contiguous update of the device block table: table[row][pos .. pos+count) = data[...].
+struct TableDelta {
+  int32_t row, pos, count, data_off;
+};
+
+// Copy of the valid rows of a partial block at fork.
+struct CowCopy {
+  int32_t src_block, dst_block, rows, pad;
+};
+
+struct Shape {
+  int32_t num_q_heads, num_kv_heads, group;
+  int32_t table_stride;        // ints per device table row
+};
+
+// ---- kernel launchers (kernels.cu); all enqueue on `st` and return cudaGetLastError() ----
+cudaError_t launch_cow_copy(void* k_pool, void* v_pool, const CowCopy* d_copies, int n,
+                            int num_kv_heads, cudaStream_t st);
+// slots[r] = block * 16 + offset for new row r.
+cudaError_t launch_append(void* k_pool, void* v_pool, const void* k_new, const void* v_new,
+                          const int32_t* d_slots, int64_t first_row, int n_rows,
+                          int num_kv_heads, cudaStream_t st);
+// Applies table deltas and (row, length) pairs to the device copies in one launch.
+cudaError_t launch_sync(int32_t* d_tables, int table_stride, int32_t* d_lens,
+                        const TableDelta* d_deltas, const int32_t* d_data, int n_deltas,
+                        const int32_t* d_len_pairs, int n_pairs, cudaStream_t st);
+
+struct AttnArgs {
+  const void* q; void* out;
+  const void* k_pool; const void* v_pool;
+  const int32_t* d_tables; const int32_t* d_lens;
+  const WorkItem* d_items; const UserRef* d_users;
+  float* part_o; float2* part_ml;     // [slots][num_q_heads][128], [slots][num_q_heads]
+  Shape shape;
+  float scale_log2e;                  // sm_scale * log2(e)
+};
+// single_row: every item carries exactly one query row.
+cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items, bool single_row,
+                                 cudaStream_t st);
+cudaError_t launch_attention_mma(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st);
+cudaError_t launch_merge(const AttnArgs& a, const MergeRef* d_merge, int n_merge, cudaStream_t st);
+
+// ---- planner (planner.cpp) ----
+struct PlanQuery {
+  const int32_t* table;   // host block ids of the query's thread
+  int32_t table_row;      // row in the device table
+  int32_t len;            // tokens
+};
+
+struct Plan {
+  std::vector<WorkItem> items;     // vec items first, then mma items; each class longest first
+  int32_t n_vec = 0, n_mma = 0;
+  std::vector<UserRef> users;
+  std::vector<MergeRef> merges;
+  int64_t total_slots = 0;         // partial rows (before the head dimension)
+  int64_t unique_tokens = 0, attended_tokens = 0;
+  int32_t chunk_tokens = 0;
+};
+
+class Planner {
+ public:
+  void init(int num_blocks, int group, int num_kv_heads);
+  // open_tails: the last chunk of a private tail run gets tok_end < 0 (resolved on the device
+  // from the length array), so the plan stays valid while threads only grow.
+  // Items with at least mma_min_rows query rows go to the tensor-core kernel.
+  // Returns false if the partial rows cannot fit `slot_capacity` even without splitting.
+  bool build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_tails,
+             int mma_min_rows, Plan* out);
+
+ private:
+  int num_blocks_ = 0, group_ = 1, hint_kv_heads_ = 1;
+  uint32_t epoch_ = 0;
+  std::vector<uint32_t> stamp_;
+  std::vector<int32_t> cnt_, seg_of_;
+  std::vector<uint8_t> partial_;
+  struct Seg { int32_t table_row, tok_begin, tok_end, n_blocks, n_users, user_off, priv, open; };
+  struct SegUser { int32_t seg, query, ord; };
+  std::vector<Seg> segs_;
+  std::vector<SegUser> seg_users_;
+  std::vector<int32_t> n_parts_, qbeg_, part_off_;
+  std::vector<WorkItem> vec_items_, mma_items_;
+};
+
+}  // namespace apar

@@ -1,0 +1,307 @@
+// CUDA kernels of the APAR decode hot path for sm_100a: copy-on-fork of a partial block,
+// KV append scatter, device-table sync, the vectorised CUDA-core attention path for
+// work items with few query rows (private tails under MHA), and the cross-item merge.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "apar_internal.h"
+
+namespace apar {
+
+// ------------------------------------------------------------------ fork: copy r rows
+// One CTA per (copy, kv head, K|V): the r valid rows of a (block, head) tile are r * 256
+// contiguous bytes.
+__global__ void __launch_bounds__(128) cow_copy_kernel(uint4* __restrict__ k_pool,
+                                                       uint4* __restrict__ v_pool,
+                                                       const CowCopy* __restrict__ copies,
+                                                       int num_kv_heads) {
+  const CowCopy c = copies[blockIdx.x];
+  uint4* pool = blockIdx.z ? v_pool : k_pool;
+  const size_t tile = kTileBytes / 16;
+  const uint4* src = pool + ((size_t)c.src_block * num_kv_heads + blockIdx.y) * tile;
+  uint4* dst = pool + ((size_t)c.dst_block * num_kv_heads + blockIdx.y) * tile;
+  const int n = c.rows * (kDim * 2 / 16);
+  for (int i = threadIdx.x; i < n; i += blockDim.x) dst[i] = src[i];
+}
+
+cudaError_t launch_cow_copy(void* k_pool, void* v_pool, const CowCopy* d_copies, int n,
+                            int num_kv_heads, cudaStream_t st) {
+  if (n <= 0) return cudaSuccess;
+  cow_copy_kernel<<<dim3(n, num_kv_heads, 2), 128, 0, st>>>((uint4*)k_pool, (uint4*)v_pool,
+                                                            d_copies, num_kv_heads);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ append: scatter new rows
+// One thread per 16 bytes of a new row; blockIdx.y selects K or V.
+__global__ void __launch_bounds__(256) append_kernel(uint4* __restrict__ k_pool,
+                                                     uint4* __restrict__ v_pool,
+                                                     const uint4* __restrict__ k_new,
+                                                     const uint4* __restrict__ v_new,
+                                                     const int32_t* __restrict__ slots,
+                                                     long long first_row, int n_rows,
+                                                     int num_kv_heads) {
+  const int per_row = num_kv_heads * 16;                 // 16-byte pieces per token row
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)n_rows * per_row) return;
+  const int r = (int)(idx / per_row), rem = (int)(idx % per_row);
+  const int h = rem >> 4, c = rem & 15;
+  const int slot = slots[r];
+  const int block = slot >> 4, off = slot & 15;
+  const uint4* src = (blockIdx.y ? v_new : k_new) + (first_row + r) * per_row + rem;
+  uint4* dst = (blockIdx.y ? v_pool : k_pool) +
+               (((size_t)block * num_kv_heads + h) * kBlock + off) * 16 + c;
+  *dst = *src;
+}
+
+cudaError_t launch_append(void* k_pool, void* v_pool, const void* k_new, const void* v_new,
+                          const int32_t* d_slots, int64_t first_row, int n_rows,
+                          int num_kv_heads, cudaStream_t st) {
+  if (n_rows <= 0) return cudaSuccess;
+  const long long total = (long long)n_rows * num_kv_heads * 16;
+  const unsigned grid = (unsigned)((total + 255) / 256);
+  append_kernel<<<dim3(grid, 2), 256, 0, st>>>((uint4*)k_pool, (uint4*)v_pool,
+                                               (const uint4*)k_new, (const uint4*)v_new, d_slots,
+                                               (long long)first_row, n_rows, num_kv_heads);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ device table / length sync
+__global__ void __launch_bounds__(128) sync_kernel(int32_t* __restrict__ tables, int stride,
+                                                   int32_t* __restrict__ lens,
+                                                   const TableDelta* __restrict__ deltas,
+                                                   const int32_t* __restrict__ data, int n_deltas,
+                                                   const int32_t* __restrict__ pairs, int n_pairs) {
+  if ((int)blockIdx.x < n_deltas) {
+    const TableDelta d = deltas[blockIdx.x];
+    int32_t* dst = tables + (size_t)d.row * stride + d.pos;
+    const int32_t* src = data + d.data_off;
+    for (int i = threadIdx.x; i < d.count; i += blockDim.x) dst[i] = src[i];
+  } else {
+    const int i = ((int)blockIdx.x - n_deltas) * blockDim.x + threadIdx.x;
+    if (i < n_pairs) lens[pairs[2 * i]] = pairs[2 * i + 1];
+  }
+}
+
+cudaError_t launch_sync(int32_t* d_tables, int table_stride, int32_t* d_lens,
+                        const TableDelta* d_deltas, const int32_t* d_data, int n_deltas,
+                        const int32_t* d_len_pairs, int n_pairs, cudaStream_t st) {
+  const int grid = n_deltas + (n_pairs + 127) / 128;
+  if (grid <= 0) return cudaSuccess;
+  sync_kernel<<<grid, 128, 0, st>>>(d_tables, table_stride, d_lens, d_deltas, d_data, n_deltas,
+                                    d_len_pairs, n_pairs);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ attention, vector path
+__device__ __forceinline__ void bf16x8_to_float(const uint4& u, float* f) {
+  f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);
+  f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xffff0000u);
+  f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xffff0000u);
+  f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xffff0000u);
+}
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// A CTA of four warps owns one (work item, kv head).  Each warp takes every fourth block of
+// the item.  A 16-token tile of K (4 KiB) is fetched with eight coalesced 16-byte loads per
+// lane: load j brings tokens 2j (lanes 0-15) and 2j+1 (lanes 16-31), lane c of a half holding
+// dims [8c, 8c+8).  Scores are reduced over the 16 lanes of a half with shuffles; the online
+// softmax state (m, l) is kept identical in both halves, o is per half and folded at the end.
+// ROWS query rows are carried at once; items with more rows loop over groups of ROWS.
+template <int ROWS>
+__global__ void __launch_bounds__(128) attn_vec_kernel(const AttnArgs a, int item_begin) {
+  const WorkItem it = a.d_items[item_begin + blockIdx.x];
+  const int kvh = blockIdx.y;
+  const int G = a.shape.group, HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;
+  const int tok_end = it.tok_end < 0 ? a.d_lens[it.table_row] : it.tok_end;
+  const int n_tok = tok_end - it.tok_begin;
+  const int n_blk = (n_tok + kBlock - 1) / kBlock;
+  const int32_t* table = a.d_tables + (size_t)it.table_row * a.shape.table_stride +
+                         it.tok_begin / kBlock;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int half = lane >> 4, c = lane & 15;
+  const int R = it.n_users * G;
+
+  __shared__ float sm_m[4][ROWS], sm_l[4][ROWS];
+  __shared__ __align__(16) float sm_o[4][ROWS][kDim];
+
+  for (int r0 = 0; r0 < R; r0 += ROWS) {
+    float qf[ROWS][8], o[ROWS][8], m[ROWS], l[ROWS];
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      m[r] = -INFINITY;
+      l[r] = 0.f;
+#pragma unroll
+      for (int d = 0; d < 8; ++d) { o[r][d] = 0.f; qf[r][d] = 0.f; }
+      if (r0 + r < R) {
+        const int u = (r0 + r) / G, hg = (r0 + r) % G;
+        const int query = a.d_users[it.user_begin + u].query;
+        const uint4 qv = *((const uint4*)a.q + ((size_t)query * HQ + kvh * G + hg) * 16 + c);
+        bf16x8_to_float(qv, qf[r]);
+#pragma unroll
+        for (int d = 0; d < 8; ++d) qf[r][d] *= a.scale_log2e;
+      }
+    }
+    for (int b = warp; b < n_blk; b += 4) {
+      const int bid = table[b];
+      const size_t tile = ((size_t)bid * HKV + kvh) * (kTileBytes / 16);
+      const uint4* kt = (const uint4*)a.k_pool + tile + half * 16 + c;
+      const uint4* vt = (const uint4*)a.v_pool + tile + half * 16 + c;
+      const int nv = min(kBlock, n_tok - b * kBlock);
+      uint4 kk[8], vv[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) kk[j] = ld_stream(kt + j * 32);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) vv[j] = ld_stream(vt + j * 32);
+      float s[ROWS][8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float kf[8];
+        bf16x8_to_float(kk[j], kf);
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) {
+          float acc = 0.f;
+#pragma unroll
+          for (int d = 0; d < 8; ++d) acc = fmaf(qf[r][d], kf[d], acc);
+          s[r][j] = acc;
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < ROWS; ++r)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          float x = s[r][j];
+          x += __shfl_xor_sync(0xffffffffu, x, 8);
+          x += __shfl_xor_sync(0xffffffffu, x, 4);
+          x += __shfl_xor_sync(0xffffffffu, x, 2);
+          x += __shfl_xor_sync(0xffffffffu, x, 1);
+          s[r][j] = (2 * j + half < nv) ? x : -INFINITY;   // rows past the length are never used
+        }
+#pragma unroll
+      for (int r = 0; r < ROWS; ++r) {
+        float bm = s[r][0];
+#pragma unroll
+        for (int j = 1; j < 8; ++j) bm = fmaxf(bm, s[r][j]);
+        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));   // token 0 is always valid
+        const float mn = fmaxf(m[r], bm);
+        const float corr = exp2f(m[r] - mn);
+        m[r] = mn;
+        float ps = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          s[r][j] = exp2f(s[r][j] - mn);
+          ps += s[r][j];
+        }
+        l[r] = l[r] * corr + ps;
+#pragma unroll
+        for (int d = 0; d < 8; ++d) o[r][d] *= corr;
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float vf[8];
+        bf16x8_to_float(vv[j], vf);
+        if (2 * j + half >= nv) {          // unspecified bits (possibly NaN patterns): drop them
+#pragma unroll
+          for (int d = 0; d < 8; ++d) vf[d] = 0.f;
+        }
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r)
+#pragma unroll
+          for (int d = 0; d < 8; ++d) o[r][d] = fmaf(s[r][j], vf[d], o[r][d]);
+      }
+    }
+    // fold the two halves of the warp, then the four warps
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      l[r] += __shfl_xor_sync(0xffffffffu, l[r], 16);
+#pragma unroll
+      for (int d = 0; d < 8; ++d) o[r][d] += __shfl_xor_sync(0xffffffffu, o[r][d], 16);
+      if (half == 0) {
+#pragma unroll
+        for (int d = 0; d < 8; ++d) sm_o[warp][r][8 * c + d] = o[r][d];
+      }
+      if (lane == 0) { sm_m[warp][r] = m[r]; sm_l[warp][r] = l[r]; }
+    }
+    __syncthreads();
+    const int t = threadIdx.x;
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      if (r0 + r < R) {
+        const float M = fmaxf(fmaxf(sm_m[0][r], sm_m[1][r]), fmaxf(sm_m[2][r], sm_m[3][r]));
+        float L = 0.f, O = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const float wgt = sm_m[w][r] == -INFINITY ? 0.f : exp2f(sm_m[w][r] - M);
+          L += sm_l[w][r] * wgt;
+          O += sm_o[w][r][t] * wgt;
+        }
+        const int u = (r0 + r) / G, hg = (r0 + r) % G;
+        const UserRef ur = a.d_users[it.user_begin + u];
+        const int head = kvh * G + hg;
+        if (ur.slot < 0) {
+          ((__nv_bfloat16*)a.out)[((size_t)ur.query * HQ + head) * kDim + t] =
+              __float2bfloat16_rn(O / L);
+        } else {
+          const size_t prow = (size_t)(ur.slot + it.slot_add) * HQ + head;
+          a.part_o[prow * kDim + t] = O;
+          if (t == 0) a.part_ml[prow] = make_float2(M, L);
+        }
+      }
+    }
+    __syncthreads();
+  }
+}
+
+cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items, bool single_row,
+                                 cudaStream_t st) {
+  if (n_items <= 0) return cudaSuccess;
+  const dim3 grid(n_items, a.shape.num_kv_heads);
+  if (single_row) attn_vec_kernel<1><<<grid, 128, 0, st>>>(a, item_begin);
+  else attn_vec_kernel<4><<<grid, 128, 0, st>>>(a, item_begin);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ merge of partial results
+// One warp per (query, head): out = sum_j o_j 2^(m_j - M) / sum_j l_j 2^(m_j - M).
+__global__ void __launch_bounds__(128) merge_kernel(const AttnArgs a,
+                                                    const MergeRef* __restrict__ merges) {
+  const MergeRef mr = merges[blockIdx.x];
+  const int head = blockIdx.y * 4 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  const int HQ = a.shape.num_q_heads;
+  if (head >= HQ) return;
+  float M = -INFINITY;
+  for (int j = 0; j < mr.n; ++j)
+    M = fmaxf(M, a.part_ml[(size_t)(mr.slot_begin + j) * HQ + head].x);
+  float L = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int j = 0; j < mr.n; ++j) {
+    const size_t prow = (size_t)(mr.slot_begin + j) * HQ + head;
+    const float2 ml = a.part_ml[prow];
+    const float w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
+    const float4 o = ((const float4*)(a.part_o + prow * kDim))[lane];
+    L += ml.y * w;
+    acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
+  }
+  const float inv = 1.f / L;
+  __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+  __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+  uint2 packed;
+  packed.x = *(uint32_t*)&lo;
+  packed.y = *(uint32_t*)&hi;
+  ((uint2*)((__nv_bfloat16*)a.out + ((size_t)mr.query * HQ + head) * kDim))[lane] = packed;
+}
+
+cudaError_t launch_merge(const AttnArgs& a, const MergeRef* d_merge, int n_merge, cudaStream_t st) {
+  if (n_merge <= 0) return cudaSuccess;
+  merge_kernel<<<dim3(n_merge, (a.shape.num_q_heads + 3) / 4), 128, 0, st>>>(a, d_merge);
+  return cudaGetLastError();
+}
+
+}  // namespace apar

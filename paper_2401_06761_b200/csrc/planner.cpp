@@ -1,0 +1,193 @@
+// Host planner: turns the block tables of the queried threads into work items in which every
+// physical block is read once for all queries that share it.
+//
+// Sharing only arises through fork (paper, Section 2.3: the child shares the parent's full
+// blocks), so the sets of threads that hold a block are nested along a chain and a block id
+// identifies the whole prefix before it.  The planner therefore needs no tree: it counts, per
+// block id, how many queries list it, and cuts each query's table into runs of equal count.
+// A run listed by several queries becomes one shared work item; runs are found again through
+// the id of their first block.  A block that is ragged (not full) for some query is never
+// shared: each query that lists it reads it on its own.
+#include <algorithm>
+#include <climits>
+#include <cstring>
+
+#include "apar_internal.h"
+
+namespace apar {
+
+void Planner::init(int num_blocks, int group, int num_kv_heads) {
+  num_blocks_ = num_blocks;
+  group_ = group;
+  hint_kv_heads_ = num_kv_heads;
+  epoch_ = 0;
+  stamp_.assign(num_blocks, 0);
+  cnt_.assign(num_blocks, 0);
+  seg_of_.assign(num_blocks, -1);
+  partial_.assign(num_blocks, 0);
+}
+
+static inline int64_t round_up16(int64_t x) { return (x + 15) / 16 * 16; }
+
+bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_tails,
+                    int mma_min_rows, Plan* out) {
+  if (++epoch_ == 0) {
+    std::fill(stamp_.begin(), stamp_.end(), 0u);
+    epoch_ = 1;
+  }
+  // ---- pass 1: how many queries list each block; which blocks are ragged for someone
+  int64_t attended = 0;
+  for (int i = 0; i < n; ++i) {
+    const int32_t len = q[i].len, nb = (len + kBlock - 1) / kBlock;
+    attended += len;
+    for (int p = 0; p < nb; ++p) {
+      const int32_t b = q[i].table[p];
+      if (stamp_[b] != epoch_) {
+        stamp_[b] = epoch_;
+        cnt_[b] = 0;
+        partial_[b] = 0;
+        seg_of_[b] = -1;
+      }
+      ++cnt_[b];
+    }
+    if (len % kBlock) partial_[q[i].table[nb - 1]] = 1;
+  }
+  // ---- pass 2: runs -> segments; a query's SegUser entries are contiguous, in chain order
+  segs_.clear();
+  seg_users_.clear();
+  qbeg_.assign(n + 1, 0);
+  int64_t unique = 0;
+  for (int i = 0; i < n; ++i) {
+    qbeg_[i] = (int32_t)seg_users_.size();
+    const int32_t len = q[i].len, nb = (len + kBlock - 1) / kBlock;
+    const int32_t* tab = q[i].table;
+    int p0 = 0;
+    while (p0 < nb) {
+      const int32_t b0 = tab[p0];
+      const bool priv0 = partial_[b0] || cnt_[b0] == 1;
+      const int32_t key0 = priv0 ? 0 : cnt_[b0];
+      int p1 = p0 + 1;
+      while (p1 < nb) {
+        const int32_t b = tab[p1];
+        const int32_t key = (partial_[b] || cnt_[b] == 1) ? 0 : cnt_[b];
+        if (key != key0) break;
+        ++p1;
+      }
+      const int32_t t0 = p0 * kBlock, t1 = std::min(p1 * kBlock, len);
+      int32_t s = -1;
+      if (!priv0) {
+        s = seg_of_[b0];
+        // tables that do not come from forks could disagree on where the run ends
+        if (s >= 0 && (segs_[s].n_blocks != p1 - p0 || segs_[s].tok_begin != t0)) s = -1;
+      }
+      if (s < 0) {
+        Seg g;
+        g.table_row = q[i].table_row;
+        g.tok_begin = t0;
+        g.tok_end = t1;
+        g.n_blocks = p1 - p0;
+        g.n_users = 0;
+        g.user_off = 0;
+        g.priv = priv0;
+        g.open = (priv0 && p1 == nb && open_tails) ? 1 : 0;
+        s = (int32_t)segs_.size();
+        segs_.push_back(g);
+        if (!priv0 && seg_of_[b0] < 0) seg_of_[b0] = s;
+        unique += t1 - t0;
+      }
+      ++segs_[s].n_users;
+      seg_users_.push_back(SegUser{s, i, 0});
+      p0 = p1;
+    }
+  }
+  qbeg_[n] = (int32_t)seg_users_.size();
+
+  // ---- chunk length: enough items to fill the machine, never below 128 tokens
+  const int64_t kInf = (int64_t)1 << 40;
+  int64_t chunk = std::max<int64_t>(128, round_up16(unique * hint_kv_heads_ / (148 * 8)));
+  n_parts_.assign(n, 0);
+  int64_t total_slots = 0;
+  for (int attempt = 0;; ++attempt) {
+    total_slots = 0;
+    for (int i = 0; i < n; ++i) {
+      int32_t ord = 0;
+      for (int k = qbeg_[i]; k < qbeg_[i + 1]; ++k) {
+        const Seg& g = segs_[seg_users_[k].seg];
+        seg_users_[k].ord = ord;
+        ord += (int32_t)((g.tok_end - g.tok_begin + chunk - 1) / chunk);
+      }
+      n_parts_[i] = ord;
+      if (ord >= 2) total_slots += ord;
+    }
+    if (total_slots <= slot_capacity) break;
+    if (chunk >= kInf) return false;
+    chunk = attempt >= 3 ? kInf : chunk * 4;
+  }
+
+  // ---- partial slots and merges
+  out->merges.clear();
+  part_off_.assign(n, -1);
+  int32_t off = 0;
+  for (int i = 0; i < n; ++i) {
+    if (n_parts_[i] >= 2) {
+      part_off_[i] = off;
+      out->merges.push_back(MergeRef{i, off, n_parts_[i], 0});
+      off += n_parts_[i];
+    }
+  }
+  // ---- users grouped by segment
+  int32_t uo = 0;
+  for (Seg& g : segs_) {
+    g.user_off = uo;
+    uo += g.n_users;
+    g.n_users = 0;
+  }
+  out->users.resize(seg_users_.size());
+  for (const SegUser& su : seg_users_) {
+    Seg& g = segs_[su.seg];
+    out->users[g.user_off + g.n_users++] =
+        UserRef{su.query, part_off_[su.query] >= 0 ? part_off_[su.query] + su.ord : -1};
+  }
+  // ---- items
+  const int max_users = std::max(1, kMaxRowsPerItem / group_);
+  vec_items_.clear();
+  mma_items_.clear();
+  for (const Seg& g : segs_) {
+    const int32_t n_chunks = (int32_t)((g.tok_end - g.tok_begin + chunk - 1) / chunk);
+    for (int u0 = 0; u0 < g.n_users; u0 += max_users) {
+      const int nu = std::min(max_users, g.n_users - u0);
+      for (int c = 0; c < n_chunks; ++c) {
+        WorkItem it;
+        it.table_row = g.table_row;
+        it.tok_begin = g.tok_begin + (int32_t)(c * chunk);
+        it.tok_end = (int32_t)std::min<int64_t>(g.tok_end, it.tok_begin + chunk);
+        // An open tail keeps its planned token count, sign-folded, for sorting; the kernels
+        // only test the sign and then read the device length array.
+        if (g.open && c == n_chunks - 1) it.tok_end = -(it.tok_end - it.tok_begin) - 1;
+        it.user_begin = g.user_off + u0;
+        it.n_users = nu;
+        it.slot_add = c;
+        it.pad0 = it.pad1 = 0;
+        (nu * group_ >= mma_min_rows ? mma_items_ : vec_items_).push_back(it);
+      }
+    }
+  }
+  auto cost = [](const WorkItem& w) {
+    return w.tok_end < 0 ? -w.tok_end - 1 : w.tok_end - w.tok_begin;
+  };
+  auto by_cost = [&](const WorkItem& a, const WorkItem& b) { return cost(a) > cost(b); };
+  std::stable_sort(vec_items_.begin(), vec_items_.end(), by_cost);
+  std::stable_sort(mma_items_.begin(), mma_items_.end(), by_cost);
+  out->n_vec = (int32_t)vec_items_.size();
+  out->n_mma = (int32_t)mma_items_.size();
+  out->items.clear();
+  out->items.insert(out->items.end(), vec_items_.begin(), vec_items_.end());
+  out->items.insert(out->items.end(), mma_items_.begin(), mma_items_.end());
+  out->total_slots = total_slots;
+  out->unique_tokens = unique;
+  out->attended_tokens = attended;
+  out->chunk_tokens = (int32_t)std::min<int64_t>(chunk, INT32_MAX);
+  return true;
+}
+
+}  // namespace apar
