@@ -1,0 +1,363 @@
+#!/usr/bin/env python
+"""Benchmark of the APAR decode hot path on B200: one step = (the step's fork, if the workload
+has one) + KV append of one token per live thread + tree decode attention over all live
+threads, for one attention layer.  Prints one JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl reference]
+
+With N > 1 (under torchrun) every rank runs its own shard of requests (a different seed of the
+same workload) on its own GPU; there is no exchange between shards.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2401_06761_b200 import synth  # noqa: E402
+
+METRIC = "tree decode-attention thread-tokens/s"
+UNIT = "thread-tokens/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc, self.lines, self.index = None, [], index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def parse_workload(name: str) -> int:
+    if not (name.startswith("cfg") and name[3:].isdigit() and int(name[3:]) in synth.LAYER_SHAPES):
+        raise SystemExit(f"unknown workload {name}; use cfg1..cfg5")
+    return int(name[3:])
+
+
+# ------------------------------------------------------------------------------ CPU baseline
+def oracle_sample(spec, budget_s: float, min_threads: int = 2):
+    """Times the fp64 checker, as it stands, on live threads of `spec` until the budget is used.
+    Returns (thread-tokens per second, threads done, cores used)."""
+    import numpy as np
+    from oracle import Forest, tree_decode_attention
+    torch.set_num_threads(1)
+    live = spec.live_nodes()
+    order = list(range(0, len(live), max(1, len(live) // 64))) + list(range(len(live)))
+    scale = spec.shape.head_dim ** -0.5
+    q_all = synth.queries(spec, len(live), "cpu").to(torch.float64).numpy()
+    done, spent = 0, 0.0
+    for i in order:
+        node = live[i]
+        k, v = synth.chain_kv(spec, node, "cpu")          # input generation: not timed
+        k, v = k.to(torch.float64).numpy(), v.to(torch.float64).numpy()
+        t0 = time.perf_counter()
+        f = Forest(spec.shape.num_kv_heads, spec.shape.head_dim)
+        t = f.new_thread()
+        f.append(t, k, v)
+        out = tree_decode_attention(f, [t], q_all[i:i + 1], scale)
+        spent += time.perf_counter() - t0
+        assert np.isfinite(out).all()
+        done += 1
+        if spent >= budget_s and done >= min_threads:
+            break
+    return done / spent, done, 1
+
+
+def run_reference(args, cfg_id):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    spec = synth.forest_spec(cfg_id)
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(spec, per_step / 4)
+    rates, threads = [], 0
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        r, n, cores = oracle_sample(spec, per_step)
+        rates.append(r); threads += n
+    wall = time.perf_counter() - t0
+    value = statistics.mean(rates)
+    sample = (f"{threads} live threads of {args.workload} over {args.steps} steps, one thread "
+              f"at a time: chain materialised in fp64 + dense softmax attention, all "
+              f"{spec.shape.num_q_heads} query heads")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wall / max(1, args.steps),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": args.workload},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------------------ GPU arm
+def run_ours(args, cfg_id):
+    from paper_2401_06761_b200 import build
+    build.build()
+    from paper_2401_06761_b200.session import PagedSession, pool_requirements
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    # shard = the same workload with a rank-specific seed: independent requests, no exchange
+    spec = synth.forest_spec(cfg_id, seed=synth.default_seed(cfg_id, rank))
+    shape = spec.shape
+    steps_total = args.warmup + args.steps
+    nb, nt, mb = pool_requirements(spec)
+    n_live = len(spec.live_nodes())
+    n_step_forks = sum(1 for n in spec.nodes if n.step_fork)
+    grow_blocks = (n_live + n_step_forks) * (2 * steps_total // 16 + 2) + 2 * n_step_forks
+    sess = PagedSession(shape, nb + grow_blocks, nt + n_step_forks, mb + 2 * steps_total // 16 + 2,
+                        device=dev)
+    t_setup = time.perf_counter()
+    step0 = synth.build_forest(spec, sess, device=dev)
+    torch.cuda.synchronize()
+    t_setup = time.perf_counter() - t_setup
+
+    from paper_2401_06761_b200 import binding as B
+    stream = torch.cuda.current_stream().cuda_stream
+    base_live = [h for h, n in zip(step0.live_handles, step0.live_nodes) if not n.step_fork]
+    base_live_arr = B.int32_array(base_live)
+    T = n_live
+    g = torch.Generator(device=dev).manual_seed(spec.seed + 99)
+    row_shape = (T, shape.num_kv_heads, shape.head_dim)
+    q_shape = (T, shape.num_q_heads, shape.head_dim)
+
+    def fresh(shp):
+        return torch.randn(shp, generator=g, device=dev).to(torch.bfloat16)
+
+    out = torch.empty(q_shape, dtype=torch.bfloat16, device=dev)
+    attn_events = []
+
+    def one_step(q, k_new, v_new, record):
+        """fork (if the workload has one) + append + attention [+ release of the step's forks]."""
+        kids = B.apar_fork(sess.ctx, step0.fork_parents, stream) if step0.fork_parents else []
+        live = B.int32_array(base_live + kids) if kids else base_live_arr
+        B.apar_append_kv(sess.ctx, live, None, k_new.data_ptr(), v_new.data_ptr(), stream)
+        if record:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        B.apar_tree_decode_attention(sess.ctx, live, q.data_ptr(), out.data_ptr(), sess.sm_scale,
+                                     stream)
+        if record:
+            e1.record()
+            attn_events.append((e0, e1))
+        if kids:
+            B.apar_release(sess.ctx, kids)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---------------- device-resident arm
+    inputs = [(fresh(q_shape), fresh(row_shape), fresh(row_shape)) for _ in range(min(4, steps_total))]
+    for i in range(args.warmup):
+        one_step(*inputs[i % len(inputs)], record=False)
+    barrier()
+    k0 = sess.stats()["kernels_total"]
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    host_t0 = time.perf_counter()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(args.steps):
+        one_step(*inputs[i % len(inputs)], record=True)
+    ev1.record()
+    host_issue_ms = 1e3 * (time.perf_counter() - host_t0)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = max_over_ranks(ev0.elapsed_time(ev1))
+    launches = sess.stats()["kernels_total"] - k0
+    attn_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_events)
+    st = sess.stats()
+
+    # ---------------- end-to-end arm: host buffers in, host buffer out, copies inside the timing
+    hq = [torch.empty(q_shape, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    hk = [torch.empty(row_shape, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    hv = [torch.empty(row_shape, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    hout = torch.empty(q_shape, dtype=torch.bfloat16).pin_memory()
+    for i in range(2):
+        hq[i].copy_(inputs[i % len(inputs)][0]); hk[i].copy_(inputs[i % len(inputs)][1])
+        hv[i].copy_(inputs[i % len(inputs)][2])
+    dq, dk, dv = (torch.empty(q_shape, dtype=torch.bfloat16, device=dev),
+                  torch.empty(row_shape, dtype=torch.bfloat16, device=dev),
+                  torch.empty(row_shape, dtype=torch.bfloat16, device=dev))
+
+    def e2e_step(i):
+        dq.copy_(hq[i % 2], non_blocking=True)
+        dk.copy_(hk[i % 2], non_blocking=True)
+        dv.copy_(hv[i % 2], non_blocking=True)
+        one_step(dq, dk, dv, record=False)
+        hout.copy_(out, non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, steps_total - 1))
+    e2e_step(0)
+    barrier()
+    ev0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    ev1.record()
+    barrier()
+    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1))
+    h2d = sum(t.numel() * 2 for t in (dq, dk, dv))
+    d2h = out.numel() * 2
+
+    # ---------------- numbers
+    units = torch.tensor([float(T)], device=dev, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(units)
+    total_T = float(units.item())
+    value = total_T * args.steps / (total_ms * 1e-3)
+    e2e_value = total_T * e2e_steps / (e2e_ms * 1e-3)
+    bpt = shape.bytes_per_token
+    unique_bytes = st["attn_unique_tokens"] * bpt
+    unshared_bytes = st["attn_attended_tokens"] * bpt
+    qo_bytes = 2 * T * shape.num_q_heads * shape.head_dim * 2
+    algo_bytes = unique_bytes + qo_bytes
+    peak, peak_kind = measured_peaks()
+    achieved = algo_bytes / (attn_ms * 1e-3) / 1e9
+
+    if rank == 0:
+        cpu_rate, cpu_threads, cores = oracle_sample(spec, 12.0) if world == 1 else (None, 0, 0)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {
+                "workload": args.workload, "threads_per_gpu": T, "requests": synth.DEFAULT_REQUESTS[cfg_id],
+                "num_q_heads": shape.num_q_heads, "num_kv_heads": shape.num_kv_heads,
+                "head_dim": shape.head_dim, "block_size": shape.block_size,
+                "step": ("fork+" if step0.fork_parents else "") + "append+attention, one layer",
+                "l2": "inputs larger than L2 (unique KV bytes per step >> 126 MB)"
+                      if unique_bytes > 4 * 126e6 else "KV smaller than L2: not flushed",
+                "parallelism": f"{world} independent shard(s), no collective",
+            },
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "gpu_launches": launches,
+            "roofline": {
+                "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None,
+                "peak_kind": f"of {peak_kind} copy bandwidth",
+                "kernel": "apar_tree_decode_attention call (table sync + attention + merge launches)",
+                "algorithmic_bytes": algo_bytes, "attention_ms": attn_ms,
+            },
+            "kv_bytes": {"unique_per_step": unique_bytes, "unshared_per_step": unshared_bytes,
+                         "sharing_ratio": unshared_bytes / max(1, unique_bytes),
+                         "attended_tokens_per_thread": st["attn_attended_tokens"] / T,
+                         "unique_tokens": st["attn_unique_tokens"]},
+            "plan": {"work_items": st["attn_work_items"], "vec_items": st["attn_vec_items"],
+                     "mma_items": st["attn_mma_items"], "partials": st["attn_partials"],
+                     "reused_last_step": st["attn_plan_reused"],
+                     "host_issue_ms_per_step": host_issue_ms / args.steps},
+            "setup_s": t_setup,
+        }
+        if cpu_rate is not None:
+            line["cpu_baseline"] = {
+                "value": cpu_rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": f"{cpu_threads} live threads of {args.workload}, one at a time "
+                          f"(fp64 chain materialisation + dense attention, all query heads)"}
+        print(json.dumps(line))
+    sess.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg4")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg_id = parse_workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, cfg_id)
+    else:
+        run_ours(args, cfg_id)
+
+
+if __name__ == "__main__":
+    main()

@@ -80,6 +80,8 @@ EXPORTS = tuple(_SIGS)
 
 
 def _arr(xs):
+    if isinstance(xs, tuple) and len(xs) == 2 and isinstance(xs[1], int):
+        return xs          # already marshalled by int32_array()
     xs = list(xs)
     return (C.c_int32 * len(xs))(*xs), len(xs)
 
@@ -129,7 +131,7 @@ def apar_append_kv(ctx, tid, n_tok, k_new: int, v_new: int, stream=0):
 
 
 def apar_tree_decode_attention(ctx, tid, q: int, out: int, sm_scale: float, stream=0):
-    tids, n = tid if isinstance(tid, tuple) else _arr(tid)
+    tids, n = _arr(tid)
     _check(lib.apar_tree_decode_attention(ctx, n, tids, q, out, sm_scale, stream))
 
 
