@@ -168,6 +168,44 @@ apar_status apar_tree_decode_attention_tables(const apar_config* cfg /*[host]*/,
                                               const void* q /*[device]*/, void* out /*[device]*/,
                                               float sm_scale, void* cuda_stream);
 
+/* Decode attention for callers that must not allocate.  (The paper has no counterpart: this
+ * is a packaging variant of the attention above, not a step of the method.)
+ *
+ * Some callers cannot let a library call cudaMalloc, cudaMallocHost or cudaFree on their
+ * behalf: a serving process whose GPU memory is entirely pre-carved by its own allocator, a
+ * plugin barred from the CUDA allocator of its host, or a latency-critical thread that must
+ * not hit the device-wide synchronisation those calls can imply.  Every other attention entry
+ * point of this library creates pinned staging buffers; this one allocates nothing at all.
+ * Its work-item list and its per-split partial results live in a 16 MiB array that is part
+ * of the library image, so every GPU that loads the library carries that array until exit.
+ *
+ * Semantics: row i of block_tables [device] int32 [n_threads][max_blocks_per_thread] with
+ * ctx_lens[i] [device] >= 1 tokens is one private chain; out[i][h] is the same softmax
+ * attention as above over that chain.  Rows are not de-duplicated: a block listed by several
+ * rows is read once per row.  Chains are cut into ceil(max_ctx_len / 1024) (at most 8) token
+ * ranges whose partial results are merged; max_ctx_len [host] is an upper bound of ctx_lens
+ * (a longer row is still computed correctly, only less evenly split).  k_pool, v_pool, q, out
+ * as in apar_config / apar_tree_decode_attention, all [device].
+ *
+ * Limits and sharing: the request is refused with APAR_ERR_WORKSPACE_TOO_SMALL when
+ * n_threads * splits * (32 + num_q_heads * 520) + n_threads * 24 bytes (each part rounded to
+ * 256) exceed 16 MiB - e.g. 64 rows x 32 heads x 8 splits fit, 512 rows x 64 heads x 8 do not.
+ * All calls on a device share the one array and it keeps the previous call's contents; every
+ * entry a call reads is written by that same call first, so nothing needs clearing, but two
+ * calls that overlap on the GPU (different streams, no ordering) race on it.
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call before any stream capture begins.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL, CUDA. */
+apar_status apar_tree_decode_attention_static(const void* k_pool /*[device]*/,
+                                              const void* v_pool /*[device]*/,
+                                              int32_t num_q_heads, int32_t num_kv_heads,
+                                              int32_t n_threads, int32_t max_blocks_per_thread,
+                                              const int32_t* block_tables /*[device]*/,
+                                              const int32_t* ctx_lens /*[device]*/,
+                                              int32_t max_ctx_len, const void* q /*[device]*/,
+                                              void* out /*[device]*/, float sm_scale,
+                                              void* cuda_stream);
+
 /* Introspection (host state only; used to compare bookkeeping entry by entry). */
 apar_status apar_get_thread(apar_ctx* ctx, int32_t tid, int32_t* len, int32_t* n_blocks,
                             int32_t* blocks /*[host] cap entries, may be NULL*/, int32_t cap);

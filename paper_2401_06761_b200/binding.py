@@ -65,6 +65,10 @@ _SIGS = {
     "apar_tree_decode_attention_tables": (C.c_int32, [_cfgp, C.c_int32, _i32p, _i32p,
                                                       C.c_void_p, C.c_void_p, C.c_float,
                                                       C.c_void_p]),
+    "apar_tree_decode_attention_static": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                                      C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                                      C.c_int32, C.c_void_p, C.c_void_p, C.c_float,
+                                                      C.c_void_p]),
     "apar_get_thread": (C.c_int32, [_ctx, C.c_int32, _i32p, _i32p, _i32p, C.c_int32]),
     "apar_get_refcounts": (C.c_int32, [_ctx, _i32p]),
     "apar_get_free_list": (C.c_int32, [_ctx, _i32p, C.c_int32, _i32p]),
@@ -147,6 +151,17 @@ def apar_tree_decode_attention_tables(cfg, block_tables, ctx_lens, q: int, out: 
     flat, _ = _arr(x for row in block_tables for x in row)
     _check(lib.apar_tree_decode_attention_tables(C.byref(cfg), n, flat, lens, q, out,
                                                  sm_scale, stream))
+
+
+def apar_tree_decode_attention_static(k_pool: int, v_pool: int, num_q_heads: int,
+                                      num_kv_heads: int, n_threads: int,
+                                      max_blocks_per_thread: int, block_tables: int,
+                                      ctx_lens: int, max_ctx_len: int, q: int, out: int,
+                                      sm_scale: float, stream=0):
+    """Allocation-free variant: block_tables and ctx_lens are DEVICE addresses here."""
+    _check(lib.apar_tree_decode_attention_static(k_pool, v_pool, num_q_heads, num_kv_heads,
+                                                 n_threads, max_blocks_per_thread, block_tables,
+                                                 ctx_lens, max_ctx_len, q, out, sm_scale, stream))
 
 
 def apar_get_thread(ctx, tid: int, cap: int = 0):
