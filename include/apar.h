@@ -3,10 +3,10 @@
  *
  * APAR (Auto-Parallel Auto-Regressive decoding) lets a model fork generation threads.
  * A forked thread shares its parent's prefix; with a paged KV cache the fork shares all
- * full blocks of the parent and copies at most one block (paper, Section 2.3 "Decoding").
+ * full blocks of the parent and duplicates no more than one block (paper, Section 2.3 "Decoding").
  * A new token attends only to the tokens on its path to the root of the paragraph tree,
  * itself included (Section 2.2 "Training attention"; Section 2.4 feature 3).  When a
- * thread finishes, the cache belonging only to it is released (Section 2.3; feature 2).
+ * thread finishes, whatever cache no other thread still uses is freed (Section 2.3; feature 2).
  *
  * This library owns the host-side bookkeeping (block tables, reference counts, free list)
  * and launches the CUDA kernels for: the copy of the partial last block at fork, the
@@ -111,12 +111,12 @@ size_t apar_workspace_bytes(const apar_config* cfg /*[host]*/);
 apar_status apar_create(const apar_config* cfg /*[host]*/, apar_ctx** out /*[host]*/);
 apar_status apar_destroy(apar_ctx* ctx);
 
-/* n new prompt sequences (roots of paragraph trees, Algorithm 1 "G <- {p}"): empty block
+/* n new prompt sequences (roots of paragraph trees; the initial sequence group of Algorithm 1): empty block
  * tables, length 0.  tid_out [host] receives n ids.  Errors: NO_THREADS. */
 apar_status apar_new_threads(apar_ctx* ctx, int32_t n, int32_t* tid_out /*[host]*/);
 
-/* Fork (Algorithm 1 "s' <- s"; Section 2.3: "copies at most 1 KV cache block and shares all
- * other blocks").  For each parent, in order: the child's table is the parent's first
+/* Fork (Algorithm 1, the step that duplicates a sequence; Section 2.3: the child maps the
+ * parent's blocks and at most a single block is physically duplicated).  For each parent, in order: the child's table is the parent's first
  * floor(len/16) block ids (their reference counts go up by one); if r = len mod 16 != 0 a
  * block is taken from the free list and the r valid rows of the parent's last block (K and V,
  * all KV heads) are copied into it by a kernel enqueued on the stream.  Child length = len.
@@ -125,7 +125,7 @@ apar_status apar_new_threads(apar_ctx* ctx, int32_t n, int32_t* tid_out /*[host]
 apar_status apar_fork(apar_ctx* ctx, int32_t n, const int32_t* parent_tid /*[host]*/,
                       int32_t* child_tid_out /*[host]*/, void* cuda_stream);
 
-/* KV append (Algorithm 1 "s.append_token(x)" and the K, V rows the model writes for it).
+/* KV append (the token append of Algorithm 1, i.e. the K, V rows the model writes for it).
  * Thread tid[i] receives n_tok[i] rows (n_tok NULL = one row each), taken consecutively from
  * k_new / v_new [device] bf16 [sum n_tok][num_kv_heads][128].  A row at position p goes to
  * slot p mod 16 of the thread's block p / 16; a block is allocated whenever p mod 16 == 0.
@@ -150,7 +150,8 @@ apar_status apar_tree_decode_attention(apar_ctx* ctx, int32_t n, const int32_t* 
                                        const void* q /*[device]*/, void* out /*[device]*/,
                                        float sm_scale, void* cuda_stream);
 
-/* ReleaseCache (Algorithm 1; Section 2.3: "the KV cache belonging only to s is released"):
+/* ReleaseCache (Algorithm 1; Section 2.3: a finished sequence gives back the cache that no
+ * other sequence holds):
  * one reference is dropped per table entry, in table order; blocks reaching zero go back to
  * the free list; the ids become invalid.  Errors: BAD_THREAD (also for a repeated id). */
 apar_status apar_release(apar_ctx* ctx, int32_t n, const int32_t* tid /*[host]*/);

@@ -1,8 +1,9 @@
 """Integer model of the paged KV pool.  Test infrastructure only (see oracle/__init__).
 
 What the paper fixes (Section 2.3 "Decoding"): a forked sequence shares its parent's
-prefix; with paged attention the fork copies at most one KV-cache block and shares all
-others; when a sequence finishes, the cache belonging only to it is released.
+prefix; on a paged cache the fork maps the parent's blocks into the child and physically
+duplicates no more than a single block; a finished sequence gives back exactly the cache
+that no other sequence still holds.
 
 What the paper leaves open and this model decides (the CUDA library documents the same
 policy in its header so that block ids can be compared one by one):

@@ -20,7 +20,7 @@ class Forest:
         self.v_rows = []
 
     def new_thread(self) -> int:
-        """A prompt sequence: no parent (Algorithm 1, G <- {p})."""
+        """A prompt sequence: no parent (the initial member of Algorithm 1's sequence group)."""
         self.parent.append(-1)
         self.inherited.append(0)
         self.k_rows.append([])
@@ -32,14 +32,14 @@ class Forest:
         return self.inherited[t] + sum(a.shape[0] for a in self.k_rows[t])
 
     def fork(self, p: int) -> int:
-        """s' <- s (Algorithm 1): the child shares every token the parent has now."""
+        """The sequence duplication of Algorithm 1: the child shares every token the parent has now."""
         t = self.new_thread()
         self.parent[t] = p
         self.inherited[t] = self.length(p)
         return t
 
     def append(self, t: int, k, v) -> None:
-        """append_token: rows [n][H_kv][D] produced for thread t's new tokens."""
+        """Token append of Algorithm 1: rows [n][H_kv][D] produced for thread t's new tokens."""
         k = np.asarray(k, dtype=np.float64)
         v = np.asarray(v, dtype=np.float64)
         assert k.shape == v.shape and k.shape[1:] == (self.num_kv_heads, self.head_dim)
