@@ -21,7 +21,7 @@ constexpr int kSlotsPerThread = 6;    // partial-result rows provisioned per liv
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {            // partition of the caller's workspace
-  size_t tables, lens, stage, plan_items, plan_users, plan_merges, part_ml, part_o, total;
+  size_t err, tables, lens, stage, plan_items, plan_users, plan_merges, part_ml, part_o, total;
   size_t stage_cap;        // bytes of the transient staging area
   int64_t slot_capacity;   // partial rows (before the head dimension)
   int64_t entry_capacity;  // (item, user) pairs a plan may hold
@@ -42,6 +42,7 @@ Layout make_layout(const apar_config* c) {
   L.stage_cap = std::min<size_t>(std::max<size_t>(table_bytes / 4 + (64 << 10), 1 << 20), 64 << 20);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  L.err = take(256);
   L.tables = take(table_bytes);
   L.lens = take((size_t)c->max_threads * 4);
   L.stage = take(L.stage_cap);
@@ -100,6 +101,7 @@ struct apar_ctx {
   int64_t plan_attended = 0;
   int plan_age = 0;
   int mma_min_rows = INT_MAX;
+  CUtensorMap tm_k, tm_v;
   int32_t last_cuda = 0;
   bool external_tables = false;        // the table-driven entry point owns no pool state
 
@@ -297,10 +299,13 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
   a.part_ml = (float2*)c->ws(c->lay.part_ml);
   a.shape = c->shape;
   a.scale_log2e = sm_scale * 1.4426950408889634f;
+  a.tm_k = &c->tm_k;
+  a.tm_v = &c->tm_v;
+  a.d_error = (int*)c->ws(c->lay.err);
   int launches = 0;
   if (p.n_mma) {
-    APAR_CUDA(c, launch_attention_mma(a, p.n_vec, p.n_mma, st));
-    ++launches;
+    APAR_CUDA(c, launch_attention_mma(a, p.n_vec, p.n_mma_tiles, st));
+    for (int k = 0; k < 4; ++k) launches += p.n_mma_tiles[k] > 0;
   }
   if (p.n_vec) {
     APAR_CUDA(c, launch_attention_vec(a, 0, p.n_vec, c->shape.group == 1 && c->mma_min_rows <= 2, st));
@@ -351,6 +356,13 @@ apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
   const char* path = getenv("APAR_ATTN_PATH");     // "vec": CUDA-core kernel for every item
   c->mma_min_rows = (path && !strcmp(path, "vec")) ? INT_MAX : 2;
   c->ring_bytes = lay.stage_cap;
+  if (make_pool_tensor_maps(cfg->k_pool, cfg->v_pool, cfg->num_blocks, cfg->num_kv_heads,
+                            &c->tm_k, &c->tm_v) != 0 ||
+      cudaMemset(c->ws(lay.err), 0, 256) != cudaSuccess) {
+    c->last_cuda = (int32_t)cudaGetLastError();
+    delete c;
+    return APAR_ERR_CUDA;
+  }
   for (int i = 0; i < kRing; ++i) {
     cudaError_t e = cudaMallocHost((void**)&c->ring[i].host, c->ring_bytes);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ring[i].done, cudaEventDisableTiming);
@@ -643,6 +655,12 @@ apar_status apar_get_stats(apar_ctx* c, apar_stats* out) {
   out->cow_blocks = c->cow_blocks;
   out->cow_rows = c->cow_rows;
   out->kernels_total = c->kernels_total;
+  int32_t flag = 0;   // synchronises with the device: introspection only
+  if (cudaMemcpy(&flag, c->ws(c->lay.err), 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    c->last_cuda = (int32_t)cudaGetLastError();
+    return APAR_ERR_CUDA;
+  }
+  out->device_wait_timeouts = flag;
   return APAR_OK;
 }
 

@@ -2,6 +2,7 @@
 // launchers.  Not part of the public boundary (include/apar.h).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -77,11 +78,20 @@ struct AttnArgs {
   float* part_o; float2* part_ml;     // [slots][num_q_heads][128], [slots][num_q_heads]
   Shape shape;
   float scale_log2e;                  // sm_scale * log2(e)
+  const CUtensorMap* tm_k = nullptr;  // [host] TMA descriptors of the pools (tensor-core path)
+  const CUtensorMap* tm_v = nullptr;
+  int* d_error = nullptr;             // [device] set to 1 when a bounded wait gave up
 };
 // single_row: every item carries exactly one query row.
 cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items, bool single_row,
                                  cudaStream_t st);
-cudaError_t launch_attention_mma(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st);
+// Tensor-core path.  Items start at item_begin, grouped by the number of 16-row query tiles
+// they need: first counts[3] items with 4 tiles, then counts[2] with 3, counts[1], counts[0].
+cudaError_t launch_attention_mma(const AttnArgs& a, int item_begin, const int32_t* counts,
+                                 cudaStream_t st);
+// Returns 0 on success.
+int make_pool_tensor_maps(void* k_pool, void* v_pool, int64_t num_blocks, int num_kv_heads,
+                          CUtensorMap* tm_k, CUtensorMap* tm_v);
 cudaError_t launch_merge(const AttnArgs& a, const MergeRef* d_merge, int n_merge, cudaStream_t st);
 
 // ---- planner (planner.cpp) ----
@@ -94,6 +104,7 @@ struct PlanQuery {
 struct Plan {
   std::vector<WorkItem> items;     // vec items first, then mma items; each class longest first
   int32_t n_vec = 0, n_mma = 0;
+  int32_t n_mma_tiles[4] = {0, 0, 0, 0};   // mma items needing 1, 2, 3, 4 query tiles
   std::vector<UserRef> users;
   std::vector<MergeRef> merges;
   int64_t total_slots = 0;         // partial rows (before the head dimension)
@@ -122,7 +133,7 @@ class Planner {
   std::vector<Seg> segs_;
   std::vector<SegUser> seg_users_;
   std::vector<int32_t> n_parts_, qbeg_, part_off_;
-  std::vector<WorkItem> vec_items_, mma_items_;
+  std::vector<WorkItem> vec_items_, mma_items_[4];
 };
 
 }  // namespace apar

@@ -151,7 +151,7 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
   // ---- items
   const int max_users = std::max(1, kMaxRowsPerItem / group_);
   vec_items_.clear();
-  mma_items_.clear();
+  for (auto& v : mma_items_) v.clear();
   for (const Seg& g : segs_) {
     const int32_t n_chunks = (int32_t)((g.tok_end - g.tok_begin + chunk - 1) / chunk);
     for (int u0 = 0; u0 < g.n_users; u0 += max_users) {
@@ -168,7 +168,8 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
         it.n_users = nu;
         it.slot_add = c;
         it.pad0 = it.pad1 = 0;
-        (nu * group_ >= mma_min_rows ? mma_items_ : vec_items_).push_back(it);
+        const int rows = nu * group_;
+        (rows >= mma_min_rows ? mma_items_[(rows + 15) / 16 - 1] : vec_items_).push_back(it);
       }
     }
   }
@@ -177,12 +178,16 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
   };
   auto by_cost = [&](const WorkItem& a, const WorkItem& b) { return cost(a) > cost(b); };
   std::stable_sort(vec_items_.begin(), vec_items_.end(), by_cost);
-  std::stable_sort(mma_items_.begin(), mma_items_.end(), by_cost);
   out->n_vec = (int32_t)vec_items_.size();
-  out->n_mma = (int32_t)mma_items_.size();
+  out->n_mma = 0;
   out->items.clear();
   out->items.insert(out->items.end(), vec_items_.begin(), vec_items_.end());
-  out->items.insert(out->items.end(), mma_items_.begin(), mma_items_.end());
+  for (int k = 3; k >= 0; --k) {          // widest items first
+    std::stable_sort(mma_items_[k].begin(), mma_items_[k].end(), by_cost);
+    out->n_mma_tiles[k] = (int32_t)mma_items_[k].size();
+    out->n_mma += out->n_mma_tiles[k];
+    out->items.insert(out->items.end(), mma_items_[k].begin(), mma_items_[k].end());
+  }
   out->total_slots = total_slots;
   out->unique_tokens = unique;
   out->attended_tokens = attended;
