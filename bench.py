@@ -168,7 +168,8 @@ def run_ours(args, cfg_id):
         dist.init_process_group("nccl", device_id=dev)
 
     # shard = the same workload with a rank-specific seed: independent requests, no exchange
-    spec = synth.forest_spec(cfg_id, seed=synth.default_seed(cfg_id, rank))
+    spec = synth.forest_spec(cfg_id, seed=synth.default_seed(cfg_id, rank),
+                             n_requests=args.requests)
     shape = spec.shape
     steps_total = args.warmup + args.steps
     nb, nt, mb = pool_requirements(spec)
@@ -296,14 +297,16 @@ def run_ours(args, cfg_id):
     achieved = algo_bytes / (attn_ms * 1e-3) / 1e9
 
     if rank == 0:
-        cpu_rate, cpu_threads, cores = oracle_sample(spec, 12.0) if world == 1 else (None, 0, 0)
+        cpu_rate, cpu_threads, cores = (oracle_sample(spec, 12.0)
+                                        if world == 1 and not args.skip_cpu_baseline
+                                        else (None, 0, 0))
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
             "config": {
-                "workload": args.workload, "threads_per_gpu": T, "requests": synth.DEFAULT_REQUESTS[cfg_id],
+                "workload": args.workload, "threads_per_gpu": T, "requests": args.requests or synth.DEFAULT_REQUESTS[cfg_id],
                 "num_q_heads": shape.num_q_heads, "num_kv_heads": shape.num_kv_heads,
                 "head_dim": shape.head_dim, "block_size": shape.block_size,
                 "step": ("fork+" if step0.fork_parents else "") + "append+attention, one layer",
@@ -350,6 +353,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--requests", type=int, default=None,
+                    help="shrink the workload to this many requests (profiling captures)")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg_id = parse_workload(args.workload)

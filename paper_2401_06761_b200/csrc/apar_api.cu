@@ -101,6 +101,7 @@ struct apar_ctx {
   int64_t plan_attended = 0;
   int plan_age = 0;
   int mma_min_rows = INT_MAX;
+  int umma_min_tiles = 2;               // items with at least this many 16-row tiles use tcgen05
   CUtensorMap tm_k, tm_v;
   int32_t last_cuda = 0;
   bool external_tables = false;        // the table-driven entry point owns no pool state
@@ -304,8 +305,19 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
   a.d_error = (int*)c->ws(c->lay.err);
   int launches = 0;
   if (p.n_mma) {
-    APAR_CUDA(c, launch_attention_mma(a, p.n_vec, p.n_mma_tiles, st));
-    for (int k = 0; k < 4; ++k) launches += p.n_mma_tiles[k] > 0;
+    // items are ordered 4, 3, 2, 1 query tiles: the first umma_min_tiles.. classes go to tcgen05
+    int32_t sync_counts[4], n_umma = 0;
+    for (int k = 0; k < 4; ++k) {
+      const bool umma = k + 1 >= c->umma_min_tiles;
+      sync_counts[k] = umma ? 0 : p.n_mma_tiles[k];
+      if (umma) n_umma += p.n_mma_tiles[k];
+    }
+    if (n_umma) {
+      APAR_CUDA(c, launch_attention_umma(a, p.n_vec, n_umma, st));
+      ++launches;
+    }
+    APAR_CUDA(c, launch_attention_mma(a, p.n_vec + n_umma, sync_counts, st));
+    for (int k = 0; k < 4; ++k) launches += sync_counts[k] > 0;
   }
   if (p.n_vec) {
     APAR_CUDA(c, launch_attention_vec(a, 0, p.n_vec, c->shape.group == 1 && c->mma_min_rows <= 2, st));
@@ -353,8 +365,11 @@ apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
   for (int i = 0; i < cfg->max_threads; ++i) c->free_slots[i] = cfg->max_threads - 1 - i;
   c->mark.assign(cfg->max_threads, 0);
   c->planner.init(cfg->num_blocks, c->shape.group, cfg->num_kv_heads);
-  const char* path = getenv("APAR_ATTN_PATH");     // "vec": CUDA-core kernel for every item
+  // APAR_ATTN_PATH (testing aid) forces one kernel family for every item it can take:
+  // "vec" CUDA cores, "mma" mma.sync, "umma" tcgen05.  Default: by row count.
+  const char* path = getenv("APAR_ATTN_PATH");
   c->mma_min_rows = (path && !strcmp(path, "vec")) ? INT_MAX : 2;
+  c->umma_min_tiles = (path && !strcmp(path, "mma")) ? 5 : (path && !strcmp(path, "umma")) ? 1 : 2;
   c->ring_bytes = lay.stage_cap;
   if (make_pool_tensor_maps(cfg->k_pool, cfg->v_pool, cfg->num_blocks, cfg->num_kv_heads,
                             &c->tm_k, &c->tm_v) != 0 ||

@@ -116,7 +116,10 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
   auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
   const uint32_t q_done_bar = bars + 8u * (2 * kStages);
 
-  if (*(volatile int*)a.d_error) return;   // an earlier CTA gave up a wait: do not pile up
+  // an earlier CTA gave up a wait: do not pile up (one reader, so the whole CTA agrees)
+  if (threadIdx.x == 0) *cta_abort = *(volatile int*)a.d_error;
+  __syncthreads();
+  if (*cta_abort) return;
   const WorkItem it = a.d_items[item_begin + blockIdx.x];
   const int kvh = blockIdx.y;
   const int G = a.shape.group, HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;
@@ -135,7 +138,6 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
       mbar_init(empty_bar(s), ACTIVE);
     }
     mbar_init(q_done_bar, 4);
-    *cta_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();

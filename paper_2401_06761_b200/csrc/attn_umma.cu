@@ -1,0 +1,439 @@
+// Blackwell tensor-core attention path (tcgen05 + TMEM) for work items with many query rows:
+// a run of blocks shared by up to 64 (query, head) rows.
+//
+// One CTA owns one (work item, kv head).  Roles:
+//   warps 0-3  softmax: thread i < 16 of warp w owns query row 16w + i, which is TMEM lane
+//              32w + i of an M = 64 accumulator.  They read S from TMEM, keep the running
+//              reference maximum and the row sum, write P = exp2(S - ref) as bf16 into shared
+//              memory in the K-major 128-byte-swizzled operand layout, rescale O in TMEM in the
+//              rare case the reference has to move, and write the results at the end.
+//   warp 4     producer: walks the block table, TMA tensor copies of 16-token K/V tiles into a
+//              ring of 64-token stages (same layout as the mma.sync path).
+//   warp 5     one elected thread issues S = Q K^T (M 64, N 64, K 128 as 8 MMAs) into one of two
+//              S buffers and O += P V (M 64, N 128, K 64 as 4 MMAs) with tcgen05.mma, and
+//              signals completion with tcgen05.commit on mbarriers.  Owns the TMEM allocation.
+// All waits are bounded; a wait that gives up raises an error word and every role unwinds to
+// the common exit where TMEM is released.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "apar_internal.h"
+
+namespace apar {
+namespace {
+
+constexpr int kTileTok = 64;                       // tokens per stage and per S tile
+constexpr int kTileBlocks = kTileTok / kBlock;     // 4
+constexpr int kNumStages = 2;
+constexpr int kHalf = kTileTok * 128;              // one 64-dim half of 64 rows: 8 KiB
+constexpr int kKV = 2 * kHalf;                     // K (or V) of a stage
+constexpr int kStage = 2 * kKV;                    // 32 KiB
+constexpr int kQOff = kNumStages * kStage;         // Q operand: [2 halves][64 rows][64 dims]
+constexpr int kPOff = kQOff + kKV;                 // P operand: [64 rows][64 tokens]
+constexpr int kBarOff = kPOff + kHalf;
+constexpr int kSmem = kBarOff + 256 + 1024;
+constexpr int kOutPitchU = kDim + 4;
+constexpr uint32_t kSpin = 1u << 20;
+constexpr int kTmemCols = 256;                     // S0 | S1 | O
+constexpr float kRefSlack = 8.f;                   // P stays below 2^8 before the reference moves
+
+enum Bar { FULL0 = 0, EMPTY0 = FULL0 + kNumStages, SFULL0 = EMPTY0 + kNumStages, SFREE0 = SFULL0 + 2,
+           PFULL = SFREE0 + 2, PFREE, QFULL, NBARS };
+
+__device__ __forceinline__ uint32_t s32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void bar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool bar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      " selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* cta_abort,
+                                         int* err_word) {
+  for (uint32_t i = 0; i < kSpin; ++i) {
+    if (bar_try(bar, parity)) return true;
+    if ((i & 255) == 255 && *cta_abort) return false;
+  }
+  *cta_abort = 1;
+  atomicExch(err_word, 1);
+  return false;
+}
+__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                       uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"((uint64_t)map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], bf16 operands, fp32 accumulate.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: D fp32, A and B bf16, A K-major, M = 64.
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(64 >> 4) << 24);
+}
+
+#define TMEM_LD_32(taddr, r, o)                                                                  \
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                         \
+               "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                          \
+               "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"         \
+               : "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), \
+                 "=r"(r[o + 5]), "=r"(r[o + 6]), "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), \
+                 "=r"(r[o + 10]), "=r"(r[o + 11]), "=r"(r[o + 12]), "=r"(r[o + 13]),             \
+                 "=r"(r[o + 14]), "=r"(r[o + 15]), "=r"(r[o + 16]), "=r"(r[o + 17]),             \
+                 "=r"(r[o + 18]), "=r"(r[o + 19]), "=r"(r[o + 20]), "=r"(r[o + 21]),             \
+                 "=r"(r[o + 22]), "=r"(r[o + 23]), "=r"(r[o + 24]), "=r"(r[o + 25]),             \
+                 "=r"(r[o + 26]), "=r"(r[o + 27]), "=r"(r[o + 28]), "=r"(r[o + 29]),             \
+                 "=r"(r[o + 30]), "=r"(r[o + 31])                                                \
+               : "r"(taddr))
+
+#define TMEM_ST_32(taddr, r)                                                                     \
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "                                   \
+               "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"                         \
+               "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"                \
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]),   \
+                 "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), \
+                 "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),         \
+                 "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),         \
+                 "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]),         \
+                 "r"(r[31])                                                                      \
+               : "memory")
+
+__device__ __forceinline__ void tmem_wait_ld() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() {
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ uint32_t swz_off(int row, int c) {   // as in the mma.sync path
+  return (uint32_t)((c >> 3) * kHalf + row * 128 + (((c & 7) ^ (row & 7)) << 4));
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *(uint32_t*)&v;
+}
+
+__global__ void __launch_bounds__(192, 2)
+attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                 const AttnArgs a, int item_begin) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (s32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* bp = smem_raw + (base - s32(smem_raw));
+  const uint32_t bars = base + kBarOff;
+  auto bar = [&](int i) { return bars + 8u * i; };
+  volatile int* cta_abort = (volatile int*)(bp + kBarOff + 8 * NBARS);
+  volatile uint32_t* tmem_slot = (volatile uint32_t*)(bp + kBarOff + 8 * NBARS + 8);
+
+  // an earlier CTA gave up a wait: do not pile up (one reader, so the whole CTA agrees)
+  if (threadIdx.x == 0) *cta_abort = *(volatile int*)a.d_error;
+  __syncthreads();
+  if (*cta_abort) return;
+  const WorkItem it = a.d_items[item_begin + blockIdx.x];
+  const int kvh = blockIdx.y;
+  const int G = a.shape.group, HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;
+  const int tok_end = it.tok_end < 0 ? a.d_lens[it.table_row] : it.tok_end;
+  const int n_tok = tok_end - it.tok_begin;
+  const int n_blk = (n_tok + kBlock - 1) / kBlock;
+  const int n_tiles = (n_tok + kTileTok - 1) / kTileTok;
+  const int32_t* table = a.d_tables + (size_t)it.table_row * a.shape.table_stride +
+                         it.tok_begin / kBlock;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int R = it.n_users * G;
+  const int n_active = (R + 15) >> 4;              // softmax warps that own real rows
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kNumStages; ++s) {
+      bar_init(bar(FULL0 + s), 1);
+      bar_init(bar(EMPTY0 + s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      bar_init(bar(SFULL0 + b), 1);
+      bar_init(bar(SFREE0 + b), n_active);
+    }
+    bar_init(bar(PFULL), n_active);
+    bar_init(bar(PFREE), 1);
+    bar_init(bar(QFULL), 4);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(s32((const void*)tmem_slot)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tm_o = tmem + 128u;      // S buffer b sits at columns [64 b, 64 b + 64)
+
+  if (warp == 4) {
+    // ---------------------------------------------------------------- TMA producer
+    for (int t = 0; t < n_tiles; ++t) {
+      const int s = t % kNumStages;
+      const int blk = t * kTileBlocks + (lane >> 2);
+      const bool mine = lane < 4 * kTileBlocks && blk < n_blk;
+      const int bid = mine ? table[blk] : 0;
+      if (t >= kNumStages &&
+          !bar_wait(bar(EMPTY0 + s), ((t / kNumStages) - 1) & 1, cta_abort, a.d_error))
+        break;
+      if (lane == 0) {
+        const int nb = min(kTileBlocks, n_blk - t * kTileBlocks);
+        bar_expect_tx(bar(FULL0 + s), (uint32_t)nb * 2u * kTileBytes);
+      }
+      __syncwarp();
+      if (mine) {
+        const int which = lane & 3;                         // K lo, K hi, V lo, V hi
+        const uint32_t dst = base + s * kStage + (which >> 1) * kKV + (which & 1) * kHalf +
+                             (lane >> 2) * (kBlock * 128);
+        tma_2d(dst, (which >> 1) ? &tm_v : &tm_k, (which & 1) * 64, (bid * HKV + kvh) * kBlock,
+               bar(FULL0 + s));
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------------------------------------------------------- MMA issuer
+    constexpr uint32_t kIdescQK = instr_desc(kTileTok, false);
+    constexpr uint32_t kIdescPV = instr_desc(kDim, true);
+    bool ok = bar_wait(bar(QFULL), 0, cta_abort, a.d_error);
+    tc_fence_after();
+    auto issue_qk = [&](int t) -> bool {
+      const int s = t % kNumStages, b = t & 1;
+      if (!bar_wait(bar(FULL0 + s), (t / kNumStages) & 1, cta_abort, a.d_error)) return false;
+      if (t >= 2 && !bar_wait(bar(SFREE0 + b), ((t >> 1) - 1) & 1, cta_abort, a.d_error))
+        return false;
+      tc_fence_after();
+      if (lane == 0) {
+        const uint32_t kb = base + s * kStage, qb = base + kQOff;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t off = (ks >> 2) * kHalf + (ks & 3) * 32;
+          umma_bf16(tmem + 64u * b, smem_desc(qb + off, 16, 1024), smem_desc(kb + off, 16, 1024),
+                    kIdescQK, ks > 0);
+        }
+        umma_commit(bar(SFULL0 + b));
+      }
+      __syncwarp();
+      return true;
+    };
+    if (ok && n_tiles > 0) ok = issue_qk(0);
+    for (int t = 0; ok && t < n_tiles; ++t) {
+      if (t + 1 < n_tiles && !issue_qk(t + 1)) break;
+      if (!bar_wait(bar(PFULL), t & 1, cta_abort, a.d_error)) break;
+      tc_fence_after();
+      if (lane == 0) {
+        const int s = t % kNumStages;
+        const uint32_t vb = base + s * kStage + kKV, pb = base + kPOff;
+        // blocks past the end of the item were never loaded: leave their k-steps out
+        const int nk = min(kTileBlocks, (n_tok - t * kTileTok + kBlock - 1) / kBlock);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          if (kk < nk)
+            umma_bf16(tm_o, smem_desc(pb + kk * 32, 16, 1024),
+                    smem_desc(vb + kk * (kBlock * 128), kHalf, 1024), kIdescPV, (t | kk) != 0);
+        umma_commit(bar(PFREE));
+        umma_commit(bar(EMPTY0 + s));
+      }
+      __syncwarp();
+    }
+  } else {
+    // ---------------------------------------------------------------- softmax warps 0-3
+    // query rows into the A-operand layout (rows past R are zero)
+    for (int i = threadIdx.x; i < 64 * 16; i += 128) {
+      const int row = i >> 4, c = i & 15;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (row < R) {
+        const int query = a.d_users[it.user_begin + row / G].query;
+        v = *((const uint4*)a.q + ((size_t)query * HQ + kvh * G + row % G) * 16 + c);
+      }
+      *(uint4*)(bp + kQOff + swz_off(row, c)) = v;
+    }
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) bar_arrive(bar(QFULL));
+
+    const bool active = warp < n_active;
+    const int row = warp * 16 + (lane & 15);
+    const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+    const float c = a.scale_log2e;
+    float ref = -INFINITY, l = 0.f;
+    bool alive = true;
+    if (active) {
+      for (int t = 0; t < n_tiles; ++t) {
+        const int b = t & 1;
+        if (!bar_wait(bar(SFULL0 + b), (t >> 1) & 1, cta_abort, a.d_error)) { alive = false; break; }
+        tc_fence_after();
+        uint32_t sr[64];
+        TMEM_LD_32((tmem + 64u * b) | lane_sel, sr, 0);
+        TMEM_LD_32((tmem + 64u * b + 32u) | lane_sel, sr, 32);
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) bar_arrive(bar(SFREE0 + b));
+        const int tile_tok = min(kTileTok, n_tok - t * kTileTok);
+        float mx = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 64; ++j) {
+          const float x = j < tile_tok ? __uint_as_float(sr[j]) * c : -INFINITY;
+          sr[j] = __float_as_uint(x);
+          mx = fmaxf(mx, x);
+        }
+        // P(t) overwrites the buffer P V(t-1) reads, and a rescale touches the O that P V(t-1)
+        // accumulates into: both need that MMA to have completed
+        if (t > 0 && !bar_wait(bar(PFREE), (t - 1) & 1, cta_abort, a.d_error)) { alive = false; break; }
+        const bool move = mx > ref + kRefSlack || ref == -INFINITY;
+        const float new_ref = move ? mx : ref;
+        if (t > 0 && __any_sync(0xffffffffu, move && lane < 16)) {
+          tc_fence_after();
+          const float f = move ? exp2f(ref - new_ref) : 1.f;
+          l *= f;
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint32_t orow[32];
+            TMEM_LD_32((tm_o + 32u * q4) | lane_sel, orow, 0);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) orow[j] = __float_as_uint(__uint_as_float(orow[j]) * f);
+            TMEM_ST_32((tm_o + 32u * q4) | lane_sel, orow);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+        }
+        ref = new_ref;
+        float ps = 0.f;
+        uint8_t* prow = bp + kPOff + row * 128;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          float p[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            p[e] = exp2f(__uint_as_float(sr[8 * ch + e]) - ref);
+            ps += p[e];
+          }
+          if (lane < 16)
+            *(uint4*)(prow + ((ch ^ (row & 7)) << 4)) =
+                make_uint4(pack2(p[0], p[1]), pack2(p[2], p[3]), pack2(p[4], p[5]),
+                           pack2(p[6], p[7]));
+        }
+        l += ps;
+        // rows of V past the valid length hold unspecified bits: zero them before P V
+        if (tile_tok < kTileTok && warp == 0) {
+          uint8_t* vptr = bp + (t % kNumStages) * kStage + kKV;
+          const int first = tile_tok, last = ((tile_tok + kBlock - 1) / kBlock) * kBlock;
+          for (int x = lane; x < (last - first) * 16; x += 32)
+            *(uint4*)(vptr + swz_off(first + (x >> 4), x & 15)) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) bar_arrive(bar(PFULL));
+      }
+      if (alive && n_tiles > 0)
+        alive = bar_wait(bar(PFREE), (n_tiles - 1) & 1, cta_abort, a.d_error);
+      tc_fence_after();
+    }
+    // ---- O rows out of TMEM, staged through shared memory for coalesced writes
+    asm volatile("bar.sync 1, 128;" ::: "memory");     // stage memory is free: all MMAs are done
+    float* so = (float*)bp;                                  // [64][kOutPitchU]
+    float* sml = so + 64 * kOutPitchU;                       // [64][2]
+    if (active) {
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        uint32_t orow[32];
+        TMEM_LD_32((tm_o + 32u * q4) | lane_sel, orow, 0);
+        tmem_wait_ld();
+        if (lane < 16) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4)
+            *(float4*)(so + row * kOutPitchU + 32 * q4 + j) =
+                make_float4(__uint_as_float(orow[j]), __uint_as_float(orow[j + 1]),
+                            __uint_as_float(orow[j + 2]), __uint_as_float(orow[j + 3]));
+        }
+      }
+      if (lane < 16) { sml[row * 2] = ref; sml[row * 2 + 1] = l; }
+    }
+    tc_fence_before();
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (alive) {
+      const int d = threadIdx.x;
+      for (int r = 0; r < R; ++r) {
+        const float M = sml[r * 2], L = sml[r * 2 + 1], O = so[r * kOutPitchU + d];
+        const UserRef ur = a.d_users[it.user_begin + r / G];
+        const int head = kvh * G + r % G;
+        if (ur.slot < 0) {
+          ((__nv_bfloat16*)a.out)[((size_t)ur.query * HQ + head) * kDim + d] =
+              __float2bfloat16_rn(O / L);
+        } else {
+          const size_t prow = (size_t)(ur.slot + it.slot_add) * HQ + head;
+          a.part_o[prow * kDim + d] = O;
+          if (d == 0) a.part_ml[prow] = make_float2(M, L);
+        }
+      }
+    }
+  }
+  // ---- common exit: every role arrives here, then the allocating warp frees TMEM
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem),
+                 "r"(kTmemCols) : "memory");
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items,
+                                  cudaStream_t st) {
+  if (n_items <= 0) return cudaSuccess;
+  static bool configured[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(attn_umma_kernel,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  attn_umma_kernel<<<dim3(n_items, a.shape.num_kv_heads), 192, kSmem, st>>>(*a.tm_k, *a.tm_v, a,
+                                                                            item_begin);
+  return cudaGetLastError();
+}
+
+}  // namespace apar

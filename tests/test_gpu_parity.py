@@ -65,7 +65,7 @@ def _make(spec, path, monkeypatch, extra_blocks=0):
     return sess, orc, Both(sess, orc)
 
 
-@pytest.mark.parametrize("path", ["vec", "auto"])
+@pytest.mark.parametrize("path", ["vec", "mma", "umma", "auto"])
 @pytest.mark.parametrize("config,nreq", [(1, 1), (2, 3), (3, 6), (4, 2), (5, 24)])
 def test_config_step_parity(config, nreq, path, monkeypatch):
     spec = synth.forest_spec(config, n_requests=nreq)
@@ -93,7 +93,7 @@ def test_config_step_parity(config, nreq, path, monkeypatch):
     sess.close()
 
 
-@pytest.mark.parametrize("path", ["vec", "auto"])
+@pytest.mark.parametrize("path", ["vec", "mma", "umma", "auto"])
 def test_random_event_replay_with_plan_reuse(path, monkeypatch):
     shape = synth.LayerShape(8, 2)
     monkeypatch.setenv("APAR_ATTN_PATH", path)
@@ -139,7 +139,7 @@ def test_random_event_replay_with_plan_reuse(path, monkeypatch):
     sess.close()
 
 
-@pytest.mark.parametrize("path", ["vec", "auto"])
+@pytest.mark.parametrize("path", ["vec", "mma", "umma", "auto"])
 @pytest.mark.parametrize("hq,hkv,n_children,prompt", [(4, 4, 40, 100), (16, 2, 12, 333),
                                                       (8, 8, 2, 1), (8, 1, 70, 48)])
 def test_wide_forks(hq, hkv, n_children, prompt, path, monkeypatch):
@@ -166,7 +166,7 @@ def test_wide_forks(hq, hkv, n_children, prompt, path, monkeypatch):
     sess.close()
 
 
-@pytest.mark.parametrize("path", ["vec", "auto"])
+@pytest.mark.parametrize("path", ["vec", "mma", "umma", "auto"])
 def test_long_thread_is_split_and_merged(path, monkeypatch):
     shape = synth.LayerShape(8, 2)
     monkeypatch.setenv("APAR_ATTN_PATH", path)
@@ -283,4 +283,44 @@ def test_error_codes_match_the_model_and_change_nothing():
     assert sess.attention([], q[:0]).shape[0] == 0
     bad = B.make_config(6, 8, 3, 4, 4)
     assert B.apar_workspace_bytes(bad) == 0
+    sess.close()
+
+
+@pytest.mark.parametrize("path", ["vec", "mma", "umma", "auto"])
+@pytest.mark.parametrize("hq,hkv,kids", [(4, 4, 5), (16, 2, 6), (8, 8, 1)])
+def test_scores_that_keep_growing_move_the_softmax_reference(hq, hkv, kids, path, monkeypatch):
+    """Every later token scores far higher than all earlier ones, so the running maximum rises by
+    many powers of two from tile to tile (and the early tokens end up with negligible weight)."""
+    shape = synth.LayerShape(hq, hkv)
+    monkeypatch.setenv("APAR_ATTN_PATH", path)
+    sess = _session(shape, 200, kids + 3, 40, poison=True)
+    orc = OracleBackend(shape, 200, kids + 3, 40)
+    both = Both(sess, orc)
+    g = torch.Generator(device="cuda").manual_seed(21)
+    u = torch.randn((128,), generator=g, device="cuda")
+    u = u / u.norm()
+    n_prompt, n_tail = 330, 45
+
+    def rows(n, start):
+        ramp = (torch.arange(start, start + n, device="cuda", dtype=torch.float32) * 0.35)
+        k = ramp[:, None, None] * u[None, None, :] + 0.05 * torch.randn((n, hkv, 128), generator=g,
+                                                                        device="cuda")
+        v = torch.randn((n, hkv, 128), generator=g, device="cuda")
+        return k.to(torch.bfloat16), v.to(torch.bfloat16)
+
+    (p,) = both.new_threads(1)
+    both.append([p], [n_prompt], *rows(n_prompt, 0))
+    tids = both.fork([p] * kids) if kids > 1 else [p]
+    for i, t in enumerate(tids):
+        both.append([t], [n_tail + i], *rows(n_tail + i, n_prompt))
+    q = (8.0 * u[None, None, :] + 0.1 * torch.randn((len(tids), hq, 128), generator=g,
+                                                    device="cuda")).to(torch.bfloat16)
+    out = sess.attention(tids, q, sm_scale=1.0)
+    ref = orc.attention(tids, q, 1.0)
+    # The softmax is nearly one-hot here, so outputs are single V rows of magnitude ~1 and the
+    # bf16 rounding of the output alone (half an ulp = 2^-9 relative) is of the order of the
+    # usual mean tolerance; allow for it explicitly.
+    err = np.abs(out.cpu().to(torch.float64).numpy() - ref)
+    assert np.isfinite(err).all() and err.max() <= 2e-2, (path, err.max())
+    assert err.mean() <= 1e-3 + 2.0 ** -9 * np.abs(ref).mean(), (path, err.mean())
     sess.close()
