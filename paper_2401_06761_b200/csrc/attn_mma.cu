@@ -23,7 +23,8 @@ constexpr int kStages = 3;
 constexpr int kHalfBytes = kStageTokens * 128;                 // 64 tokens x 64 dims x 2 B = 8 KiB
 constexpr int kKVBytes = 2 * kHalfBytes;                       // K (or V) of a stage: 16 KiB
 constexpr int kStageBytes = 2 * kKVBytes;                      // 32 KiB
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment*/ + 256 /*barriers*/;
+constexpr int kUsersOff = kStages * kStageBytes + 256;        // the item's UserRef entries (<= 64)
+constexpr int kSmemBytes = kUsersOff + 64 * 8 + 1024 /*alignment*/;
 constexpr int kOutPitch = kDim + 4;                            // floats per staged output row
 constexpr uint32_t kSpinLimit = 1u << 20;
 
@@ -85,6 +86,11 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
       "{%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2(float x) {   // 2^x, flushes to zero, 2^-inf = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -173,14 +179,18 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
 
   // -------------------------------------------------------------------- consumer warps
   // query rows -> shared memory (tile layout of a K stage, rows = query rows), zero padded
+  UserRef* s_users = (UserRef*)(base_ptr + kUsersOff);
+  if (threadIdx.x < it.n_users) s_users[threadIdx.x] = a.d_users[it.user_begin + threadIdx.x];
+  consumer_sync();
   {
     const uint32_t qbase = base + (kStages - 1) * kStageBytes;
     uint8_t* qptr = base_ptr + (kStages - 1) * kStageBytes;
+#pragma unroll
     for (int i = threadIdx.x; i < MT * 16 * 16; i += 128) {
       const int row = i >> 4, c = i & 15;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
       if (row < R) {
-        const int query = a.d_users[it.user_begin + row / G].query;
+        const int query = s_users[row / G].query;
         v = *((const uint4*)a.q + ((size_t)query * HQ + kvh * G + row % G) * 16 + c);
       }
       *(uint4*)(qptr + tile_off(row, c)) = v;
@@ -264,7 +274,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
         mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
         mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
         const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: token 0 is valid
-        const float cr0 = exp2f(m0 - mn0), cr1 = exp2f(m1 - mn1);
+        const float cr0 = ex2(m0 - mn0), cr1 = ex2(m1 - mn1);
         m0 = mn0; m1 = mn1;
         float ps0 = 0.f, ps1 = 0.f;
         uint32_t pa[NBW][4];
@@ -273,10 +283,10 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
           float p[2][4];
 #pragma unroll
           for (int n = 0; n < 2; ++n) {
-            p[n][0] = exp2f(sc[2 * i + n][0] - mn0);
-            p[n][1] = exp2f(sc[2 * i + n][1] - mn0);
-            p[n][2] = exp2f(sc[2 * i + n][2] - mn1);
-            p[n][3] = exp2f(sc[2 * i + n][3] - mn1);
+            p[n][0] = ex2(sc[2 * i + n][0] - mn0);
+            p[n][1] = ex2(sc[2 * i + n][1] - mn0);
+            p[n][2] = ex2(sc[2 * i + n][2] - mn1);
+            p[n][3] = ex2(sc[2 * i + n][3] - mn1);
             ps0 += p[n][0] + p[n][1];
             ps1 += p[n][2] + p[n][3];
           }
@@ -343,11 +353,11 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
     for (int sp = 0; sp < SPLITS; ++sp) {
       const int w = rmt + MT * sp;
       const float mw = sml[(w * 16 + ri) * 2];
-      const float wgt = mw == -INFINITY ? 0.f : exp2f(mw - M);
+      const float wgt = mw == -INFINITY ? 0.f : ex2(mw - M);
       L += sml[(w * 16 + ri) * 2 + 1] * wgt;
       O += so[(w * 16 + ri) * kOutPitch + d] * wgt;
     }
-    const UserRef ur = a.d_users[it.user_begin + r / G];
+    const UserRef ur = s_users[r / G];
     const int head = kvh * G + r % G;
     if (ur.slot < 0) {
       ((__nv_bfloat16*)a.out)[((size_t)ur.query * HQ + head) * kDim + d] =

@@ -30,16 +30,17 @@ constexpr int kHalf = kTileTok * 128;              // one 64-dim half of 64 rows
 constexpr int kKV = 2 * kHalf;                     // K (or V) of a stage
 constexpr int kStage = 2 * kKV;                    // 32 KiB
 constexpr int kQOff = kNumStages * kStage;         // Q operand: [2 halves][64 rows][64 dims]
-constexpr int kPOff = kQOff + kKV;                 // P operand: [64 rows][64 tokens]
-constexpr int kBarOff = kPOff + kHalf;
-constexpr int kSmem = kBarOff + 256 + 1024;
+constexpr int kPOff = kQOff + kKV;                 // P operand, two buffers of [64 rows][64 tokens]
+constexpr int kBarOff = kPOff + 2 * kHalf;
+constexpr int kUserOff = kBarOff + 256;             // the item's UserRef entries (at most 64)
+constexpr int kSmem = kUserOff + 64 * 8 + 1024;
 constexpr int kOutPitchU = kDim + 4;
 constexpr uint32_t kSpin = 1u << 20;
 constexpr int kTmemCols = 256;                     // S0 | S1 | O
 constexpr float kRefSlack = 8.f;                   // P stays below 2^8 before the reference moves
 
 enum Bar { FULL0 = 0, EMPTY0 = FULL0 + kNumStages, SFULL0 = EMPTY0 + kNumStages, SFREE0 = SFULL0 + 2,
-           PFULL = SFREE0 + 2, PFREE, QFULL, NBARS };
+           PFULL0 = SFREE0 + 2, PFREE0 = PFULL0 + 2, QFULL = PFREE0 + 2, NBARS };
 
 __device__ __forceinline__ uint32_t s32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -147,6 +148,11 @@ __device__ __forceinline__ void tmem_wait_st() {
 __device__ __forceinline__ uint32_t swz_off(int row, int c) {   // as in the mma.sync path
   return (uint32_t)((c >> 3) * kHalf + row * 128 + (((c & 7) ^ (row & 7)) << 4));
 }
+__device__ __forceinline__ float ex2(float x) {   // 2^x, flushes to zero, 2^-inf = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *(uint32_t*)&v;
@@ -188,9 +194,9 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     for (int b = 0; b < 2; ++b) {
       bar_init(bar(SFULL0 + b), 1);
       bar_init(bar(SFREE0 + b), n_active);
+      bar_init(bar(PFULL0 + b), n_active);
+      bar_init(bar(PFREE0 + b), 1);
     }
-    bar_init(bar(PFULL), n_active);
-    bar_init(bar(PFREE), 1);
     bar_init(bar(QFULL), 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -232,55 +238,73 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     // ---------------------------------------------------------------- MMA issuer
     constexpr uint32_t kIdescQK = instr_desc(kTileTok, false);
     constexpr uint32_t kIdescPV = instr_desc(kDim, true);
-    bool ok = bar_wait(bar(QFULL), 0, cta_abort, a.d_error);
-    tc_fence_after();
-    auto issue_qk = [&](int t) -> bool {
-      const int s = t % kNumStages, b = t & 1;
-      if (!bar_wait(bar(FULL0 + s), (t / kNumStages) & 1, cta_abort, a.d_error)) return false;
-      if (t >= 2 && !bar_wait(bar(SFREE0 + b), ((t >> 1) - 1) & 1, cta_abort, a.d_error))
-        return false;
+    // One thread issues everything.  It polls for whichever step can go next - Q K^T of the
+    // next tile as soon as its K has landed and an S buffer is free, P V of the oldest pending
+    // tile as soon as the softmax warps have published P - so that neither waits for the other.
+    if (lane == 0 && bar_wait(bar(QFULL), 0, cta_abort, a.d_error)) {
       tc_fence_after();
-      if (lane == 0) {
-        const uint32_t kb = base + s * kStage, qb = base + kQOff;
+      int qk_next = 0, pv_next = 0;
+      uint32_t idle = 0;
+      while (pv_next < n_tiles) {
+        bool did = false;
+        if (qk_next < n_tiles) {
+          const int t = qk_next, s = t % kNumStages, b = t & 1;
+          if (bar_try(bar(FULL0 + s), (t / kNumStages) & 1) &&
+              (t < 2 || bar_try(bar(SFREE0 + b), ((t >> 1) - 1) & 1))) {
+            tc_fence_after();
+            const uint32_t kb = base + s * kStage, qb = base + kQOff;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t off = (ks >> 2) * kHalf + (ks & 3) * 32;
-          umma_bf16(tmem + 64u * b, smem_desc(qb + off, 16, 1024), smem_desc(kb + off, 16, 1024),
-                    kIdescQK, ks > 0);
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint32_t off = (ks >> 2) * kHalf + (ks & 3) * 32;
+              umma_bf16(tmem + 64u * b, smem_desc(qb + off, 16, 1024),
+                        smem_desc(kb + off, 16, 1024), kIdescQK, ks > 0);
+            }
+            umma_commit(bar(SFULL0 + b));
+            ++qk_next;
+            did = true;
+          }
         }
-        umma_commit(bar(SFULL0 + b));
-      }
-      __syncwarp();
-      return true;
-    };
-    if (ok && n_tiles > 0) ok = issue_qk(0);
-    for (int t = 0; ok && t < n_tiles; ++t) {
-      if (t + 1 < n_tiles && !issue_qk(t + 1)) break;
-      if (!bar_wait(bar(PFULL), t & 1, cta_abort, a.d_error)) break;
-      tc_fence_after();
-      if (lane == 0) {
-        const int s = t % kNumStages;
-        const uint32_t vb = base + s * kStage + kKV, pb = base + kPOff;
-        // blocks past the end of the item were never loaded: leave their k-steps out
-        const int nk = min(kTileBlocks, (n_tok - t * kTileTok + kBlock - 1) / kBlock);
+        if (pv_next < qk_next) {
+          const int t = pv_next, s = t % kNumStages;
+          if (bar_try(bar(PFULL0 + (t & 1)), (t >> 1) & 1)) {
+            tc_fence_after();
+            const uint32_t vb = base + s * kStage + kKV, pb = base + kPOff + (t & 1) * kHalf;
+            // blocks past the end of the item were never loaded: leave their k-steps out
+            const int nk = min(kTileBlocks, (n_tok - t * kTileTok + kBlock - 1) / kBlock);
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
-          if (kk < nk)
-            umma_bf16(tm_o, smem_desc(pb + kk * 32, 16, 1024),
-                    smem_desc(vb + kk * (kBlock * 128), kHalf, 1024), kIdescPV, (t | kk) != 0);
-        umma_commit(bar(PFREE));
-        umma_commit(bar(EMPTY0 + s));
+            for (int kk = 0; kk < 4; ++kk)
+              if (kk < nk)
+                umma_bf16(tm_o, smem_desc(pb + kk * 32, 16, 1024),
+                          smem_desc(vb + kk * (kBlock * 128), kHalf, 1024), kIdescPV,
+                          (t | kk) != 0);
+            umma_commit(bar(PFREE0 + (t & 1)));
+            umma_commit(bar(EMPTY0 + s));
+            ++pv_next;
+            did = true;
+          }
+        }
+        if (did) {
+          idle = 0;
+        } else if (++idle > kSpin || ((idle & 255) == 0 && *cta_abort)) {
+          *cta_abort = 1;
+          atomicExch(a.d_error, 1);
+          break;
+        }
       }
-      __syncwarp();
     }
+    __syncwarp();
   } else {
     // ---------------------------------------------------------------- softmax warps 0-3
-    // query rows into the A-operand layout (rows past R are zero)
+    // the item's users once, then the query rows into the A-operand layout (rows past R zero)
+    UserRef* s_users = (UserRef*)(bp + kUserOff);
+    if (threadIdx.x < it.n_users) s_users[threadIdx.x] = a.d_users[it.user_begin + threadIdx.x];
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+#pragma unroll
     for (int i = threadIdx.x; i < 64 * 16; i += 128) {
       const int row = i >> 4, c = i & 15;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
       if (row < R) {
-        const int query = a.d_users[it.user_begin + row / G].query;
+        const int query = s_users[row / G].query;
         v = *((const uint4*)a.q + ((size_t)query * HQ + kvh * G + row % G) * 16 + c);
       }
       *(uint4*)(bp + kQOff + swz_off(row, c)) = v;
@@ -315,14 +339,16 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           sr[j] = __float_as_uint(x);
           mx = fmaxf(mx, x);
         }
-        // P(t) overwrites the buffer P V(t-1) reads, and a rescale touches the O that P V(t-1)
-        // accumulates into: both need that MMA to have completed
-        if (t > 0 && !bar_wait(bar(PFREE), (t - 1) & 1, cta_abort, a.d_error)) { alive = false; break; }
         const bool move = mx > ref + kRefSlack || ref == -INFINITY;
         const float new_ref = move ? mx : ref;
         if (t > 0 && __any_sync(0xffffffffu, move && lane < 16)) {
+          // rare: the reference moves, so O (which P V(t-1) still accumulates into) is rescaled
+          if (!bar_wait(bar(PFREE0 + ((t - 1) & 1)), ((t - 1) >> 1) & 1, cta_abort, a.d_error)) {
+            alive = false;
+            break;
+          }
           tc_fence_after();
-          const float f = move ? exp2f(ref - new_ref) : 1.f;
+          const float f = move ? ex2(ref - new_ref) : 1.f;
           l *= f;
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
@@ -338,21 +364,27 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
         ref = new_ref;
         float ps = 0.f;
-        uint8_t* prow = bp + kPOff + row * 128;
+        uint32_t pk[32];
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          float p[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            p[e] = exp2f(__uint_as_float(sr[8 * ch + e]) - ref);
-            ps += p[e];
-          }
-          if (lane < 16)
-            *(uint4*)(prow + ((ch ^ (row & 7)) << 4)) =
-                make_uint4(pack2(p[0], p[1]), pack2(p[2], p[3]), pack2(p[4], p[5]),
-                           pack2(p[6], p[7]));
+        for (int j = 0; j < 32; ++j) {
+          const float p0 = ex2(__uint_as_float(sr[2 * j]) - ref);
+          const float p1 = ex2(__uint_as_float(sr[2 * j + 1]) - ref);
+          ps += p0 + p1;
+          pk[j] = pack2(p0, p1);
         }
         l += ps;
+        // P(t) goes into the buffer that P V(t-2) read
+        if (t >= 2 && !bar_wait(bar(PFREE0 + b), ((t >> 1) - 1) & 1, cta_abort, a.d_error)) {
+          alive = false;
+          break;
+        }
+        if (lane < 16) {
+          uint8_t* prow = bp + kPOff + b * kHalf + row * 128;
+#pragma unroll
+          for (int ch = 0; ch < 8; ++ch)
+            *(uint4*)(prow + ((ch ^ (row & 7)) << 4)) =
+                make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+        }
         // rows of V past the valid length hold unspecified bits: zero them before P V
         if (tile_tok < kTileTok && warp == 0) {
           uint8_t* vptr = bp + (t % kNumStages) * kStage + kKV;
@@ -362,10 +394,11 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) bar_arrive(bar(PFULL));
+        if (lane == 0) bar_arrive(bar(PFULL0 + b));
       }
       if (alive && n_tiles > 0)
-        alive = bar_wait(bar(PFREE), (n_tiles - 1) & 1, cta_abort, a.d_error);
+        alive = bar_wait(bar(PFREE0 + ((n_tiles - 1) & 1)), ((n_tiles - 1) >> 1) & 1, cta_abort,
+                         a.d_error);
       tc_fence_after();
     }
     // ---- O rows out of TMEM, staged through shared memory for coalesced writes
@@ -394,7 +427,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       const int d = threadIdx.x;
       for (int r = 0; r < R; ++r) {
         const float M = sml[r * 2], L = sml[r * 2 + 1], O = so[r * kOutPitchU + d];
-        const UserRef ur = a.d_users[it.user_begin + r / G];
+        const UserRef ur = s_users[r / G];
         const int head = kvh * G + r % G;
         if (ur.slot < 0) {
           ((__nv_bfloat16*)a.out)[((size_t)ur.query * HQ + head) * kDim + d] =
