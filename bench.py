@@ -249,6 +249,9 @@ def run_ours(args, cfg_id):
     launches = sess.stats()["kernels_total"] - k0
     attn_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_events)
     st = sess.stats()
+    if st["device_wait_timeouts"]:
+        raise SystemExit(f"a kernel gave up a bounded wait (code {st['device_wait_timeouts']}): "
+                         "the timed results are invalid")
 
     # ---------------- end-to-end arm: host buffers in, host buffer out, copies inside the timing
     hq = [torch.empty(q_shape, dtype=torch.bfloat16).pin_memory() for _ in range(2)]

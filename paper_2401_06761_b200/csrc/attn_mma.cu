@@ -122,11 +122,11 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
   auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
   const uint32_t q_done_bar = bars + 8u * (2 * kStages);
 
+  const WorkItem it = a.d_items[item_begin + blockIdx.x];
   // an earlier CTA gave up a wait: do not pile up (one reader, so the whole CTA agrees)
   if (threadIdx.x == 0) *cta_abort = *(volatile int*)a.d_error;
   __syncthreads();
   if (*cta_abort) return;
-  const WorkItem it = a.d_items[item_begin + blockIdx.x];
   const int kvh = blockIdx.y;
   const int G = a.shape.group, HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;
   const int tok_end = it.tok_end < 0 ? a.d_lens[it.table_row] : it.tok_end;
@@ -150,11 +150,20 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
 
   if (warp == 4) {
     // ------------------------------------------------------------------ producer warp
+    // block ids are fetched 32 at a time (eight tiles), one batch ahead of their use, so that
+    // no table read sits between two tiles
+    int ids_cur = lane < n_blk ? table[lane] : 0;
+    int ids_next = 32 + lane < n_blk ? table[32 + lane] : 0;
     for (int t = 0; t < n_tiles; ++t) {
       const int s = t % kStages;
+      if (t > 0 && (t & 7) == 0) {
+        ids_cur = ids_next;
+        const int nxt = (t + 8) * kStageBlocks + lane;
+        ids_next = nxt < n_blk ? table[nxt] : 0;
+      }
       const int blk = t * kStageBlocks + (lane >> 2);
       const bool mine = lane < 4 * kStageBlocks && blk < n_blk;
-      const int bid = mine ? table[blk] : 0;
+      const int bid = __shfl_sync(0xffffffffu, ids_cur, blk & 31);
       if (t >= kStages) {
         if (!mbar_wait(empty_bar(s), ((t / kStages) - 1) & 1, cta_abort, a.d_error)) break;
       } else if (s == kStages - 1) {
@@ -343,6 +352,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
   }
   consumer_sync();
   const int d = threadIdx.x;                                 // one output dim per thread
+#pragma unroll 4
   for (int r = 0; r < R; ++r) {
     const int rmt = r >> 4, ri = r & 15;
     float M = -INFINITY;

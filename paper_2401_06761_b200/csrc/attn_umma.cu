@@ -7,8 +7,10 @@
 //              reference maximum and the row sum, write P = exp2(S - ref) as bf16 into shared
 //              memory in the K-major 128-byte-swizzled operand layout, rescale O in TMEM in the
 //              rare case the reference has to move, and write the results at the end.
-//   warp 4     producer: walks the block table, TMA tensor copies of 16-token K/V tiles into a
-//              ring of 64-token stages (same layout as the mma.sync path).
+//   warp 4     producer: walks the block table, TMA tensor copies of 16-token K/V tiles into
+//              two rings of 64-token stages - K (two deep, released as soon as Q K^T has
+//              read it) and V (three deep, released after P V) - same tile layout as the
+//              mma.sync path.
 //   warp 5     one elected thread issues S = Q K^T (M 64, N 64, K 128 as 8 MMAs) into one of two
 //              S buffers and O += P V (M 64, N 128, K 64 as 4 MMAs) with tcgen05.mma, and
 //              signals completion with tcgen05.commit on mbarriers.  Owns the TMEM allocation.
@@ -25,13 +27,13 @@ namespace {
 
 constexpr int kTileTok = 64;                       // tokens per stage and per S tile
 constexpr int kTileBlocks = kTileTok / kBlock;     // 4
-constexpr int kNumStages = 2;
+constexpr int kKStages = 2, kVStages = 3;
 constexpr int kHalf = kTileTok * 128;              // one 64-dim half of 64 rows: 8 KiB
-constexpr int kKV = 2 * kHalf;                     // K (or V) of a stage
-constexpr int kStage = 2 * kKV;                    // 32 KiB
-constexpr int kQOff = kNumStages * kStage;         // Q operand: [2 halves][64 rows][64 dims]
-constexpr int kPOff = kQOff + kKV;                 // P operand, two buffers of [64 rows][64 tokens]
-constexpr int kBarOff = kPOff + 2 * kHalf;
+constexpr int kKV = 2 * kHalf;                     // K (or V) of a stage: 16 KiB
+constexpr int kVOff = kKStages * kKV;              // V ring after the K ring
+constexpr int kQOff = kVOff + kVStages * kKV;      // Q operand: [2 halves][64 rows][64 dims]
+constexpr int kPOff = kQOff + kKV;                 // P operand: [64 rows][64 tokens]
+constexpr int kBarOff = kPOff + kHalf;
 constexpr int kUserOff = kBarOff + 256;             // the item's UserRef entries (at most 64)
 constexpr int kSmem = kUserOff + 64 * 8 + 1024;
 constexpr int kOutPitchU = kDim + 4;
@@ -39,8 +41,9 @@ constexpr uint32_t kSpin = 1u << 20;
 constexpr int kTmemCols = 256;                     // S0 | S1 | O
 constexpr float kRefSlack = 8.f;                   // P stays below 2^8 before the reference moves
 
-enum Bar { FULL0 = 0, EMPTY0 = FULL0 + kNumStages, SFULL0 = EMPTY0 + kNumStages, SFREE0 = SFULL0 + 2,
-           PFULL0 = SFREE0 + 2, PFREE0 = PFULL0 + 2, QFULL = PFREE0 + 2, NBARS };
+enum Bar { KFULL0 = 0, KEMPTY0 = KFULL0 + kKStages, VFULL0 = KEMPTY0 + kKStages,
+           VEMPTY0 = VFULL0 + kVStages, SFULL0 = VEMPTY0 + kVStages, SFREE0 = SFULL0 + 2,
+           PFULL = SFREE0 + 2, PFREE, QFULL, NBARS };
 
 __device__ __forceinline__ uint32_t s32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -63,14 +66,15 @@ __device__ __forceinline__ bool bar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// Bounded wait.  On giving up it records where (code = wait site * 1000 + tile) in the error word.
 __device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* cta_abort,
-                                         int* err_word) {
+                                         int* err_word, int code) {
   for (uint32_t i = 0; i < kSpin; ++i) {
     if (bar_try(bar, parity)) return true;
     if ((i & 255) == 255 && *cta_abort) return false;
   }
   *cta_abort = 1;
-  atomicExch(err_word, 1);
+  atomicCAS(err_word, 0, code);
   return false;
 }
 __device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
@@ -169,11 +173,11 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   volatile int* cta_abort = (volatile int*)(bp + kBarOff + 8 * NBARS);
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(bp + kBarOff + 8 * NBARS + 8);
 
+  const WorkItem it = a.d_items[item_begin + blockIdx.x];
   // an earlier CTA gave up a wait: do not pile up (one reader, so the whole CTA agrees)
   if (threadIdx.x == 0) *cta_abort = *(volatile int*)a.d_error;
   __syncthreads();
   if (*cta_abort) return;
-  const WorkItem it = a.d_items[item_begin + blockIdx.x];
   const int kvh = blockIdx.y;
   const int G = a.shape.group, HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;
   const int tok_end = it.tok_end < 0 ? a.d_lens[it.table_row] : it.tok_end;
@@ -187,16 +191,20 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   const int n_active = (R + 15) >> 4;              // softmax warps that own real rows
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kNumStages; ++s) {
-      bar_init(bar(FULL0 + s), 1);
-      bar_init(bar(EMPTY0 + s), 1);
+    for (int s = 0; s < kKStages; ++s) {
+      bar_init(bar(KFULL0 + s), 1);
+      bar_init(bar(KEMPTY0 + s), 1);
+    }
+    for (int s = 0; s < kVStages; ++s) {
+      bar_init(bar(VFULL0 + s), 1);
+      bar_init(bar(VEMPTY0 + s), 1);
     }
     for (int b = 0; b < 2; ++b) {
       bar_init(bar(SFULL0 + b), 1);
       bar_init(bar(SFREE0 + b), n_active);
-      bar_init(bar(PFULL0 + b), n_active);
-      bar_init(bar(PFREE0 + b), 1);
     }
+    bar_init(bar(PFULL), n_active);
+    bar_init(bar(PFREE), 1);
     bar_init(bar(QFULL), 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -213,25 +221,69 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 
   if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
-    for (int t = 0; t < n_tiles; ++t) {
-      const int s = t % kNumStages;
-      const int blk = t * kTileBlocks + (lane >> 2);
-      const bool mine = lane < 4 * kTileBlocks && blk < n_blk;
-      const int bid = mine ? table[blk] : 0;
-      if (t >= kNumStages &&
-          !bar_wait(bar(EMPTY0 + s), ((t / kNumStages) - 1) & 1, cta_abort, a.d_error))
-        break;
-      if (lane == 0) {
-        const int nb = min(kTileBlocks, n_blk - t * kTileBlocks);
-        bar_expect_tx(bar(FULL0 + s), (uint32_t)nb * 2u * kTileBytes);
+    // K and V tiles are two independent sequences; each is issued as soon as its ring slot has
+    // been released.  Block ids are fetched 32 at a time (eight tiles), one batch ahead.
+    int kid_cur = lane < n_blk ? table[lane] : 0, vid_cur = kid_cur;
+    int kid_next = 32 + lane < n_blk ? table[32 + lane] : 0, vid_next = kid_next;
+    int k_next = 0, v_next = 0;
+    uint32_t idle = 0;
+    while (k_next < n_tiles || v_next < n_tiles) {
+      bool did = false;
+      if (k_next < n_tiles) {
+        const int t = k_next, s = t % kKStages;
+        int ready = t < kKStages || bar_try(bar(KEMPTY0 + s), ((t / kKStages) - 1) & 1);
+        ready = __shfl_sync(0xffffffffu, ready, 0);
+        if (ready) {
+          if (t > 0 && (t & 7) == 0) {
+            kid_cur = kid_next;
+            const int nxt = (t + 8) * kTileBlocks + lane;
+            kid_next = nxt < n_blk ? table[nxt] : 0;
+          }
+          const int blk = t * kTileBlocks + (lane >> 1);
+          const int bid = __shfl_sync(0xffffffffu, kid_cur, blk & 31);
+          if (lane == 0)
+            bar_expect_tx(bar(KFULL0 + s),
+                          (uint32_t)min(kTileBlocks, n_blk - t * kTileBlocks) * kTileBytes);
+          __syncwarp();
+          if (lane < 2 * kTileBlocks && blk < n_blk)
+            tma_2d(base + s * kKV + (lane & 1) * kHalf + (lane >> 1) * (kBlock * 128), &tm_k,
+                   (lane & 1) * 64, (bid * HKV + kvh) * kBlock, bar(KFULL0 + s));
+          ++k_next;
+          did = true;
+        }
       }
-      __syncwarp();
-      if (mine) {
-        const int which = lane & 3;                         // K lo, K hi, V lo, V hi
-        const uint32_t dst = base + s * kStage + (which >> 1) * kKV + (which & 1) * kHalf +
-                             (lane >> 2) * (kBlock * 128);
-        tma_2d(dst, (which >> 1) ? &tm_v : &tm_k, (which & 1) * 64, (bid * HKV + kvh) * kBlock,
-               bar(FULL0 + s));
+      if (v_next < n_tiles) {
+        const int t = v_next, s = t % kVStages;
+        int ready = t < kVStages || bar_try(bar(VEMPTY0 + s), ((t / kVStages) - 1) & 1);
+        ready = __shfl_sync(0xffffffffu, ready, 0);
+        if (ready) {
+          if (t > 0 && (t & 7) == 0) {
+            vid_cur = vid_next;
+            const int nxt = (t + 8) * kTileBlocks + lane;
+            vid_next = nxt < n_blk ? table[nxt] : 0;
+          }
+          const int blk = t * kTileBlocks + (lane >> 1);
+          const int bid = __shfl_sync(0xffffffffu, vid_cur, blk & 31);
+          if (lane == 0)
+            bar_expect_tx(bar(VFULL0 + s),
+                          (uint32_t)min(kTileBlocks, n_blk - t * kTileBlocks) * kTileBytes);
+          __syncwarp();
+          if (lane < 2 * kTileBlocks && blk < n_blk)
+            tma_2d(base + kVOff + s * kKV + (lane & 1) * kHalf + (lane >> 1) * (kBlock * 128),
+                   &tm_v, (lane & 1) * 64, (bid * HKV + kvh) * kBlock, bar(VFULL0 + s));
+          ++v_next;
+          did = true;
+        }
+      }
+      if (did) {
+        idle = 0;
+      } else {
+        ++idle;
+        int stop = idle > kSpin || ((idle & 255) == 0 && *cta_abort);
+        if (__shfl_sync(0xffffffffu, stop, 0)) {
+          if (lane == 0 && idle > kSpin) { *cta_abort = 1; atomicCAS(a.d_error, 0, 6000 + k_next * 40 + v_next % 40); }
+          break;
+        }
       }
     }
   } else if (warp == 5) {
@@ -241,18 +293,18 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     // One thread issues everything.  It polls for whichever step can go next - Q K^T of the
     // next tile as soon as its K has landed and an S buffer is free, P V of the oldest pending
     // tile as soon as the softmax warps have published P - so that neither waits for the other.
-    if (lane == 0 && bar_wait(bar(QFULL), 0, cta_abort, a.d_error)) {
+    if (lane == 0 && bar_wait(bar(QFULL), 0, cta_abort, a.d_error, 1000)) {
       tc_fence_after();
       int qk_next = 0, pv_next = 0;
       uint32_t idle = 0;
       while (pv_next < n_tiles) {
         bool did = false;
         if (qk_next < n_tiles) {
-          const int t = qk_next, s = t % kNumStages, b = t & 1;
-          if (bar_try(bar(FULL0 + s), (t / kNumStages) & 1) &&
+          const int t = qk_next, s = t % kKStages, b = t & 1;
+          if (bar_try(bar(KFULL0 + s), (t / kKStages) & 1) &&
               (t < 2 || bar_try(bar(SFREE0 + b), ((t >> 1) - 1) & 1))) {
             tc_fence_after();
-            const uint32_t kb = base + s * kStage, qb = base + kQOff;
+            const uint32_t kb = base + s * kKV, qb = base + kQOff;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
               const uint32_t off = (ks >> 2) * kHalf + (ks & 3) * 32;
@@ -260,15 +312,16 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         smem_desc(kb + off, 16, 1024), kIdescQK, ks > 0);
             }
             umma_commit(bar(SFULL0 + b));
+            umma_commit(bar(KEMPTY0 + s));
             ++qk_next;
             did = true;
           }
         }
         if (pv_next < qk_next) {
-          const int t = pv_next, s = t % kNumStages;
-          if (bar_try(bar(PFULL0 + (t & 1)), (t >> 1) & 1)) {
+          const int t = pv_next, s = t % kVStages;
+          if (bar_try(bar(PFULL), t & 1) && bar_try(bar(VFULL0 + s), (t / kVStages) & 1)) {
             tc_fence_after();
-            const uint32_t vb = base + s * kStage + kKV, pb = base + kPOff + (t & 1) * kHalf;
+            const uint32_t vb = base + kVOff + s * kKV, pb = base + kPOff;
             // blocks past the end of the item were never loaded: leave their k-steps out
             const int nk = min(kTileBlocks, (n_tok - t * kTileTok + kBlock - 1) / kBlock);
 #pragma unroll
@@ -277,8 +330,8 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 umma_bf16(tm_o, smem_desc(pb + kk * 32, 16, 1024),
                           smem_desc(vb + kk * (kBlock * 128), kHalf, 1024), kIdescPV,
                           (t | kk) != 0);
-            umma_commit(bar(PFREE0 + (t & 1)));
-            umma_commit(bar(EMPTY0 + s));
+            umma_commit(bar(PFREE));
+            umma_commit(bar(VEMPTY0 + s));
             ++pv_next;
             did = true;
           }
@@ -286,8 +339,8 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         if (did) {
           idle = 0;
         } else if (++idle > kSpin || ((idle & 255) == 0 && *cta_abort)) {
+          if (idle > kSpin) atomicCAS(a.d_error, 0, 7000 + qk_next * 40 + pv_next % 40);
           *cta_abort = 1;
-          atomicExch(a.d_error, 1);
           break;
         }
       }
@@ -322,7 +375,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     if (active) {
       for (int t = 0; t < n_tiles; ++t) {
         const int b = t & 1;
-        if (!bar_wait(bar(SFULL0 + b), (t >> 1) & 1, cta_abort, a.d_error)) { alive = false; break; }
+        if (!bar_wait(bar(SFULL0 + b), (t >> 1) & 1, cta_abort, a.d_error, 2000 + t)) { alive = false; break; }
         tc_fence_after();
         uint32_t sr[64];
         TMEM_LD_32((tmem + 64u * b) | lane_sel, sr, 0);
@@ -341,9 +394,10 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
         const bool move = mx > ref + kRefSlack || ref == -INFINITY;
         const float new_ref = move ? mx : ref;
-        if (t > 0 && __any_sync(0xffffffffu, move && lane < 16)) {
+        const bool rescale = t > 0 && __any_sync(0xffffffffu, move && lane < 16);
+        if (rescale) {
           // rare: the reference moves, so O (which P V(t-1) still accumulates into) is rescaled
-          if (!bar_wait(bar(PFREE0 + ((t - 1) & 1)), ((t - 1) >> 1) & 1, cta_abort, a.d_error)) {
+          if (!bar_wait(bar(PFREE), (t - 1) & 1, cta_abort, a.d_error, 3000 + t)) {
             alive = false;
             break;
           }
@@ -373,13 +427,13 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           pk[j] = pack2(p0, p1);
         }
         l += ps;
-        // P(t) goes into the buffer that P V(t-2) read
-        if (t >= 2 && !bar_wait(bar(PFREE0 + b), ((t >> 1) - 1) & 1, cta_abort, a.d_error)) {
+        // P(t) overwrites the buffer that P V(t-1) reads
+        if (t > 0 && !rescale && !bar_wait(bar(PFREE), (t - 1) & 1, cta_abort, a.d_error, 3000 + t)) {
           alive = false;
           break;
         }
         if (lane < 16) {
-          uint8_t* prow = bp + kPOff + b * kHalf + row * 128;
+          uint8_t* prow = bp + kPOff + row * 128;
 #pragma unroll
           for (int ch = 0; ch < 8; ++ch)
             *(uint4*)(prow + ((ch ^ (row & 7)) << 4)) =
@@ -387,18 +441,22 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
         // rows of V past the valid length hold unspecified bits: zero them before P V
         if (tile_tok < kTileTok && warp == 0) {
-          uint8_t* vptr = bp + (t % kNumStages) * kStage + kKV;
+          const int vs = t % kVStages;
+          if (!bar_wait(bar(VFULL0 + vs), (t / kVStages) & 1, cta_abort, a.d_error, 4000 + t)) {
+            alive = false;
+            break;
+          }
+          uint8_t* vptr = bp + kVOff + vs * kKV;
           const int first = tile_tok, last = ((tile_tok + kBlock - 1) / kBlock) * kBlock;
           for (int x = lane; x < (last - first) * 16; x += 32)
             *(uint4*)(vptr + swz_off(first + (x >> 4), x & 15)) = make_uint4(0u, 0u, 0u, 0u);
         }
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) bar_arrive(bar(PFULL0 + b));
+        if (lane == 0) bar_arrive(bar(PFULL));
       }
       if (alive && n_tiles > 0)
-        alive = bar_wait(bar(PFREE0 + ((n_tiles - 1) & 1)), ((n_tiles - 1) >> 1) & 1, cta_abort,
-                         a.d_error);
+        alive = bar_wait(bar(PFREE), (n_tiles - 1) & 1, cta_abort, a.d_error, 5000);
       tc_fence_after();
     }
     // ---- O rows out of TMEM, staged through shared memory for coalesced writes
@@ -425,6 +483,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     asm volatile("bar.sync 1, 128;" ::: "memory");
     if (alive) {
       const int d = threadIdx.x;
+#pragma unroll 4
       for (int r = 0; r < R; ++r) {
         const float M = sml[r * 2], L = sml[r * 2 + 1], O = so[r * kOutPitchU + d];
         const UserRef ur = s_users[r / G];
