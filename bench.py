@@ -24,7 +24,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2401_06761_b200 import synth  # noqa: E402
+from paper_2401_06761_b200 import sharding, synth  # noqa: E402
 
 METRIC = "tree decode-attention thread-tokens/s"
 UNIT = "thread-tokens/s"
@@ -168,8 +168,7 @@ def run_ours(args, cfg_id):
         dist.init_process_group("nccl", device_id=dev)
 
     # shard = the same workload with a rank-specific seed: independent requests, no exchange
-    spec = synth.forest_spec(cfg_id, seed=synth.default_seed(cfg_id, rank),
-                             n_requests=args.requests)
+    spec = sharding.shard_spec(cfg_id, rank, n_requests=args.requests)
     shape = spec.shape
     steps_total = args.warmup + args.steps
     nb, nt, mb = pool_requirements(spec)
@@ -221,11 +220,7 @@ def run_ours(args, cfg_id):
         torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return sharding.reduce_timing(ms, 0.0, dist, dev)[0]
 
     # ---------------- device-resident arm
     inputs = [(fresh(q_shape), fresh(row_shape), fresh(row_shape)) for _ in range(min(4, steps_total))]
@@ -285,10 +280,7 @@ def run_ours(args, cfg_id):
     d2h = out.numel() * 2
 
     # ---------------- numbers
-    units = torch.tensor([float(T)], device=dev, dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(units)
-    total_T = float(units.item())
+    total_T = sharding.reduce_timing(0.0, float(T), dist, dev)[1]
     value = total_T * args.steps / (total_ms * 1e-3)
     e2e_value = total_T * e2e_steps / (e2e_ms * 1e-3)
     bpt = shape.bytes_per_token
