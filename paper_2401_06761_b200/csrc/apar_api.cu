@@ -102,6 +102,7 @@ struct apar_ctx {
   int plan_age = 0;
   int mma_min_rows = INT_MAX;
   int umma_min_tiles = 2;               // items with at least this many 16-row tiles use tcgen05
+  bool use_ws = true;                   // single-tile items use the warp-stream kernel
   CUtensorMap tm_k, tm_v;
   int32_t last_cuda = 0;
   bool external_tables = false;        // the table-driven entry point owns no pool state
@@ -316,6 +317,13 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
       APAR_CUDA(c, launch_attention_umma(a, p.n_vec, n_umma, st));
       ++launches;
     }
+    if (c->use_ws && sync_counts[0] > 0) {
+      // single-tile items are last in the list: whole items (all kv heads) per CTA
+      const int first = p.n_vec + p.n_mma - sync_counts[0];
+      APAR_CUDA(c, launch_attention_ws(a, first, sync_counts[0], st));
+      sync_counts[0] = 0;
+      ++launches;
+    }
     APAR_CUDA(c, launch_attention_mma(a, p.n_vec + n_umma, sync_counts, st));
     for (int k = 0; k < 4; ++k) launches += sync_counts[k] > 0;
   }
@@ -366,10 +374,12 @@ apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
   c->mark.assign(cfg->max_threads, 0);
   c->planner.init(cfg->num_blocks, c->shape.group, cfg->num_kv_heads);
   // APAR_ATTN_PATH (testing aid) forces one kernel family for every item it can take:
-  // "vec" CUDA cores, "mma" mma.sync, "umma" tcgen05.  Default: by row count.
+  // "vec" CUDA cores, "mma" mma.sync, "umma" tcgen05.  Default ("auto"): 1 row vec, up to 16
+  // rows warp-stream (mma.sync, whole item per CTA), more rows tcgen05.
   const char* path = getenv("APAR_ATTN_PATH");
   c->mma_min_rows = (path && !strcmp(path, "vec")) ? INT_MAX : 2;
   c->umma_min_tiles = (path && !strcmp(path, "mma")) ? 5 : (path && !strcmp(path, "umma")) ? 1 : 2;
+  c->use_ws = !(path && (!strcmp(path, "mma") || !strcmp(path, "umma")));
   c->ring_bytes = lay.stage_cap;
   if (make_pool_tensor_maps(cfg->k_pool, cfg->v_pool, cfg->num_blocks, cfg->num_kv_heads,
                             &c->tm_k, &c->tm_v) != 0 ||

@@ -91,6 +91,8 @@ cudaError_t launch_attention_mma(const AttnArgs& a, int item_begin, const int32_
                                  cudaStream_t st);
 // Blackwell tcgen05/TMEM path for items with up to 64 rows (any number of query tiles).
 cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st);
+// Warp-stream path for items with at most 16 rows per kv head; one CTA per item, all kv heads.
+cudaError_t launch_attention_ws(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st);
 // Returns 0 on success.
 int make_pool_tensor_maps(void* k_pool, void* v_pool, int64_t num_blocks, int num_kv_heads,
                           CUtensorMap* tm_k, CUtensorMap* tm_v);

@@ -1,0 +1,333 @@
+// Warp-stream attention path for work items with at most 16 query rows per kv head (the tails of
+// GQA threads, small sets of siblings): one CTA owns a whole work item, *all* kv heads.
+//
+// The four consumer warps each stream different kv heads, independently of one another: warp w
+// takes heads w, w+4, ...  Every warp has its own ring of four 16-token slots (K and V tile of
+// one block, 8 KiB) filled by the producer warp with TMA tensor copies, its own mbarriers, and
+// keeps Q (as mma.sync A-fragments, fetched straight from global memory one head ahead), the
+// online-softmax state and O in registers.  There is no CTA-wide synchronisation inside the
+// loop, no folding between warps, and the fixed cost of a CTA (item, users, first TMA round
+// trip, write-out) is paid once per item instead of once per (item, head), which is what the
+// short tails of decode batches are sensitive to.  One CTA per SM keeps 128 KiB in flight.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "apar_internal.h"
+
+namespace apar {
+namespace {
+
+constexpr int kSlots = 4;                           // ring depth per consumer warp
+constexpr int kSlotBytes = 2 * kTileBytes;          // K tile + V tile of one block: 8 KiB
+constexpr int kRingBytes = 4 * kSlots * kSlotBytes; // 128 KiB
+constexpr int kUsersOffW = kRingBytes;              // UserRef[16]
+constexpr int kBarsOffW = kUsersOffW + 16 * 8;      // full[4][kSlots], empty[4][kSlots]
+constexpr int kSmemW = kBarsOffW + 2 * 4 * kSlots * 8 + 64 + 1024;
+constexpr uint32_t kSpinW = 1u << 20;
+constexpr float kSlack = 8.f;                       // the reference max moves only past 2^8
+
+__device__ __forceinline__ uint32_t sm32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void wb_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void wb_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void wb_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool wb_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      " selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait; records (site * 1000 + detail) in the error word when it gives up.
+__device__ __forceinline__ bool wb_wait(uint32_t bar, uint32_t parity, volatile int* cta_abort,
+                                        int* err_word, int code) {
+  for (uint32_t i = 0; i < kSpinW; ++i) {
+    if (wb_try(bar, parity)) return true;
+    if ((i & 255) == 255 && *cta_abort) return false;
+  }
+  *cta_abort = 1;
+  atomicCAS(err_word, 0, code);
+  return false;
+}
+__device__ __forceinline__ void tma2d(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                      uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"((uint64_t)map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm4t(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+      "{%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2f(float x) {   // 2^x, flushes to zero, 2^-inf = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t packbf(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *(uint32_t*)&v;
+}
+// (row of the block, 16-byte chunk c of 16) inside a [2 halves][16 rows][64 dims] tile written
+// by TMA with the 128-byte swizzle.
+__device__ __forceinline__ uint32_t blk_off(int row, int c) {
+  return (uint32_t)((c >> 3) * 2048 + row * 128 + (((c & 7) ^ (row & 7)) << 4));
+}
+
+__global__ void __launch_bounds__(160, 1)
+attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+               const AttnArgs a, int item_begin) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (sm32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* bp = smem_raw + (base - sm32(smem_raw));
+  UserRef* s_users = (UserRef*)(bp + kUsersOffW);
+  const uint32_t bars = base + kBarsOffW;
+  auto full_bar = [&](int w, int s) { return bars + 8u * (w * kSlots + s); };
+  auto empty_bar = [&](int w, int s) { return bars + 8u * (4 * kSlots + w * kSlots + s); };
+  volatile int* cta_abort = (volatile int*)(bp + kBarsOffW + 2 * 4 * kSlots * 8);
+
+  const WorkItem it = a.d_items[item_begin + blockIdx.x];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    *cta_abort = *(volatile int*)a.d_error;   // an earlier CTA gave up a wait: do not pile up
+    for (int i = 0; i < 4 * kSlots; ++i) {
+      wb_init(bars + 8u * i, 1);
+      wb_init(bars + 8u * (4 * kSlots + i), 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (threadIdx.x < it.n_users) s_users[threadIdx.x] = a.d_users[it.user_begin + threadIdx.x];
+  __syncthreads();
+  if (*cta_abort) return;
+
+  const int G = a.shape.group, HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;
+  const int tok_end = it.tok_end < 0 ? a.d_lens[it.table_row] : it.tok_end;
+  const int n_tok = tok_end - it.tok_begin;
+  const int n_blk = (n_tok + kBlock - 1) / kBlock;
+  const int32_t* table = a.d_tables + (size_t)it.table_row * a.shape.table_stride +
+                         it.tok_begin / kBlock;
+  const int R = it.n_users * G;                    // rows per kv head, <= 16
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ producer warp
+    // Lanes 0-15 work on their own: lane = 4 * stream + op, op = K lo, K hi, V lo, V hi.  The
+    // four lanes of a stream poll the same "slot free" barrier and each issues its own copy;
+    // the op-0 lane also posts the byte count.
+    if (lane < 16) {
+      const int w = lane >> 2, op = lane & 3;
+      const int heads_w = (HKV - w + 3) >> 2;
+      const int total = heads_w * n_blk;
+      const CUtensorMap* map = (op >> 1) ? &tm_v : &tm_k;
+      int bid_next = total > 0 ? table[0] : 0;
+      for (int c = 0, hi = 0, b = 0; c < total; ++c) {
+        const int bid = bid_next;
+        const int b1 = b + 1 == n_blk ? 0 : b + 1;
+        if (c + 1 < total) bid_next = table[b1];            // one block ahead of its use
+        const int s = c % kSlots;
+        if (c >= kSlots &&
+            !wb_wait(empty_bar(w, s), ((c / kSlots) - 1) & 1, cta_abort, a.d_error, 8000 + w))
+          break;
+        if (op == 0) wb_expect_tx(full_bar(w, s), kSlotBytes);
+        const int h = w + 4 * hi;
+        tma2d(base + (w * kSlots + s) * kSlotBytes + (op >> 1) * kTileBytes + (op & 1) * 2048, map,
+              (op & 1) * 64, (bid * HKV + h) * kBlock, full_bar(w, s));
+        b = b1;
+        if (b == 0) ++hi;
+      }
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- consumer warps
+  const int w = warp;
+  const int heads_w = (HKV - w + 3) >> 2;
+  const int g = lane >> 2, tq = lane & 3;
+  const int jm = lane >> 3, jr = lane & 7;
+  const float cs = a.scale_log2e;
+
+  // Q rows g and g+8 of head h as A-fragments, straight from global memory.
+  auto load_q = [&](int h, uint32_t (&qa)[8][4]) {
+    const uint32_t* p0 = nullptr;
+    const uint32_t* p1 = nullptr;
+    if (g < R)
+      p0 = (const uint32_t*)a.q + ((size_t)s_users[g / G].query * HQ + h * G + g % G) * 64;
+    if (g + 8 < R)
+      p1 = (const uint32_t*)a.q +
+           ((size_t)s_users[(g + 8) / G].query * HQ + h * G + (g + 8) % G) * 64;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      qa[ks][0] = p0 ? __ldg(p0 + ks * 8 + tq) : 0u;
+      qa[ks][2] = p0 ? __ldg(p0 + ks * 8 + 4 + tq) : 0u;
+      qa[ks][1] = p1 ? __ldg(p1 + ks * 8 + tq) : 0u;
+      qa[ks][3] = p1 ? __ldg(p1 + ks * 8 + 4 + tq) : 0u;
+    }
+  };
+
+  uint32_t qa[8][4], qn[8][4];
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) qn[ks][0] = qn[ks][1] = qn[ks][2] = qn[ks][3] = 0u;
+  if (heads_w > 0) load_q(w, qa);
+  int c = 0;                                       // blocks consumed so far by this warp
+  bool alive = true;
+  for (int hi = 0; hi < heads_w && alive; ++hi) {
+    const int h = w + 4 * hi;
+    if (hi + 1 < heads_w) load_q(h + 4, qn);       // lands while this head streams
+    float o[16][4];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
+    float ref0 = -INFINITY, ref1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+
+    for (int b = 0; b < n_blk; ++b, ++c) {
+      const int s = c % kSlots;
+      if (!wb_wait(full_bar(w, s), (c / kSlots) & 1, cta_abort, a.d_error, 9000 + w)) {
+        alive = false;
+        break;
+      }
+      const uint32_t kb = base + (w * kSlots + s) * kSlotBytes, vb = kb + kTileBytes;
+      const int nv = min(kBlock, n_tok - b * kBlock);
+      // S = Q K^T for the 16 tokens of the block
+      float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
+      {
+        const int row = (jm >> 1) * 8 + jr;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          uint32_t kf[4];
+          ldsm4(kb + blk_off(row, 2 * ks + (jm & 1)), kf);
+          mma16816(acc0, qa[ks], kf[0], kf[1]);
+          mma16816(acc1, qa[ks], kf[2], kf[3]);
+        }
+      }
+      if (nv < kBlock) {   // rows of V past the valid length hold unspecified bits: zero them
+        uint8_t* vptr = bp + (w * kSlots + s) * kSlotBytes + kTileBytes;
+        for (int x = lane; x < (kBlock - nv) * 16; x += 32)
+          *(uint4*)(vptr + blk_off(nv + (x >> 4), x & 15)) = make_uint4(0u, 0u, 0u, 0u);
+        __syncwarp();
+      }
+      float sc[2][4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int t0 = 2 * tq + (e & 1);
+        sc[0][e] = t0 < nv ? acc0[e] * cs : -INFINITY;
+        sc[1][e] = t0 + 8 < nv ? acc1[e] * cs : -INFINITY;
+      }
+      float mx0 = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
+      float mx1 = fmaxf(fmaxf(sc[0][2], sc[0][3]), fmaxf(sc[1][2], sc[1][3]));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      // the reference only moves when the maximum outgrows it by 2^8 (P stays below 256)
+      const bool mv0 = mx0 > ref0 + kSlack || ref0 == -INFINITY;
+      const bool mv1 = mx1 > ref1 + kSlack || ref1 == -INFINITY;
+      if (__any_sync(0xffffffffu, mv0 || mv1)) {
+        const float f0 = mv0 ? ex2f(ref0 - mx0) : 1.f, f1 = mv1 ? ex2f(ref1 - mx1) : 1.f;
+        if (mv0) ref0 = mx0;
+        if (mv1) ref1 = mx1;
+        l0 *= f0;
+        l1 *= f1;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          o[j][0] *= f0; o[j][1] *= f0; o[j][2] *= f1; o[j][3] *= f1;
+        }
+      }
+      float p[2][4];
+#pragma unroll
+      for (int n = 0; n < 2; ++n) {
+        p[n][0] = ex2f(sc[n][0] - ref0);
+        p[n][1] = ex2f(sc[n][1] - ref0);
+        p[n][2] = ex2f(sc[n][2] - ref1);
+        p[n][3] = ex2f(sc[n][3] - ref1);
+      }
+      l0 += p[0][0] + p[0][1] + p[1][0] + p[1][1];
+      l1 += p[0][2] + p[0][3] + p[1][2] + p[1][3];
+      uint32_t pa[4] = {packbf(p[0][0], p[0][1]), packbf(p[0][2], p[0][3]),
+                        packbf(p[1][0], p[1][1]), packbf(p[1][2], p[1][3])};
+      {
+        const int row = (jm & 1) * 8 + jr;
+#pragma unroll
+        for (int jp = 0; jp < 8; ++jp) {
+          uint32_t vf[4];
+          ldsm4t(vb + blk_off(row, 2 * jp + (jm >> 1)), vf);
+          mma16816(o[2 * jp], pa, vf[0], vf[1]);
+          mma16816(o[2 * jp + 1], pa, vf[2], vf[3]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) wb_arrive(empty_bar(w, s));
+    }
+    if (!alive) break;
+    // ---- this head's rows: straight from the accumulator fragments
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int r = g + 8 * half;
+      if (r < R) {
+        const UserRef ur = s_users[r / G];
+        const int head = h * G + r % G;
+        const float L = half ? l1 : l0, M = half ? ref1 : ref0;
+        if (ur.slot < 0) {
+          const float inv = 1.f / L;
+          uint32_t* dst = (uint32_t*)a.out + ((size_t)ur.query * HQ + head) * 64 + tq;
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            dst[4 * j] = packbf(o[j][2 * half] * inv, o[j][2 * half + 1] * inv);
+        } else {
+          const size_t prow = (size_t)(ur.slot + it.slot_add) * HQ + head;
+          float2* dst = (float2*)(a.part_o + prow * kDim) + tq;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) dst[4 * j] = make_float2(o[j][2 * half], o[j][2 * half + 1]);
+          if (tq == 0) a.part_ml[prow] = make_float2(M, L);
+        }
+      }
+    }
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) qa[ks][e] = qn[ks][e];
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_attention_ws(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st) {
+  if (n_items <= 0) return cudaSuccess;
+  static bool configured[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(attn_ws_kernel,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemW);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
+  }
+  attn_ws_kernel<<<n_items, 160, kSmemW, st>>>(*a.tm_k, *a.tm_v, a, item_begin);
+  return cudaGetLastError();
+}
+
+}  // namespace apar
