@@ -36,7 +36,6 @@ constexpr int kPOff = kQOff + kKV;                 // P operand: [64 rows][64 to
 constexpr int kBarOff = kPOff + kHalf;
 constexpr int kUserOff = kBarOff + 256;             // the item's UserRef entries (at most 64)
 constexpr int kSmem = kUserOff + 64 * 8 + 1024;
-constexpr int kOutPitchU = kDim + 4;
 constexpr uint32_t kSpin = 1u << 20;
 constexpr int kTmemCols = 256;                     // S0 | S1 | O
 constexpr float kRefSlack = 8.f;                   // P stays below 2^8 before the reference moves
@@ -352,15 +351,23 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     UserRef* s_users = (UserRef*)(bp + kUserOff);
     if (threadIdx.x < it.n_users) s_users[threadIdx.x] = a.d_users[it.user_begin + threadIdx.x];
     asm volatile("bar.sync 1, 128;" ::: "memory");
+    {
+      // all eight loads of a thread are issued before the first store, so that their
+      // latencies overlap
+      uint4 qv[8];
 #pragma unroll
-    for (int i = threadIdx.x; i < 64 * 16; i += 128) {
-      const int row = i >> 4, c = i & 15;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (row < R) {
-        const int query = s_users[row / G].query;
-        v = *((const uint4*)a.q + ((size_t)query * HQ + kvh * G + row % G) * 16 + c);
+      for (int k = 0; k < 8; ++k) {
+        const int i = threadIdx.x + 128 * k, row = i >> 4, c = i & 15;
+        qv[k] = make_uint4(0u, 0u, 0u, 0u);
+        if (row < R)
+          qv[k] = __ldg((const uint4*)a.q +
+                        ((size_t)s_users[row / G].query * HQ + kvh * G + row % G) * 16 + c);
       }
-      *(uint4*)(bp + kQOff + swz_off(row, c)) = v;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int i = threadIdx.x + 128 * k;
+        *(uint4*)(bp + kQOff + swz_off(i >> 4, i & 15)) = qv[k];
+      }
     }
     fence_async_smem();
     __syncwarp();
@@ -459,44 +466,40 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         alive = bar_wait(bar(PFREE), (n_tiles - 1) & 1, cta_abort, a.d_error, 5000);
       tc_fence_after();
     }
-    // ---- O rows out of TMEM, staged through shared memory for coalesced writes
-    asm volatile("bar.sync 1, 128;" ::: "memory");     // stage memory is free: all MMAs are done
-    float* so = (float*)bp;                                  // [64][kOutPitchU]
-    float* sml = so + 64 * kOutPitchU;                       // [64][2]
-    if (active) {
+    // ---- O rows out of TMEM: the thread that owns a row writes it, 32 columns at a time
+    if (active && alive) {
+      const bool mine = lane < 16 && row < R;
+      UserRef ur = UserRef{0, -1};
+      if (mine) ur = s_users[row / G];
+      const int head = kvh * G + row % G;
+      const float inv = 1.f / l;
+      uint4* dst_out = (uint4*)((__nv_bfloat16*)a.out + ((size_t)ur.query * HQ + head) * kDim);
+      const size_t prow = (size_t)(ur.slot + it.slot_add) * HQ + head;
+      float4* dst_part = (float4*)(a.part_o + prow * kDim);
 #pragma unroll
       for (int q4 = 0; q4 < 4; ++q4) {
         uint32_t orow[32];
         TMEM_LD_32((tm_o + 32u * q4) | lane_sel, orow, 0);
         tmem_wait_ld();
-        if (lane < 16) {
+        if (mine) {
+          if (ur.slot < 0) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 4)
-            *(float4*)(so + row * kOutPitchU + 32 * q4 + j) =
-                make_float4(__uint_as_float(orow[j]), __uint_as_float(orow[j + 1]),
-                            __uint_as_float(orow[j + 2]), __uint_as_float(orow[j + 3]));
+            for (int j = 0; j < 32; j += 8)
+              dst_out[4 * q4 + (j >> 3)] = make_uint4(
+                  pack2(__uint_as_float(orow[j]) * inv, __uint_as_float(orow[j + 1]) * inv),
+                  pack2(__uint_as_float(orow[j + 2]) * inv, __uint_as_float(orow[j + 3]) * inv),
+                  pack2(__uint_as_float(orow[j + 4]) * inv, __uint_as_float(orow[j + 5]) * inv),
+                  pack2(__uint_as_float(orow[j + 6]) * inv, __uint_as_float(orow[j + 7]) * inv));
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              dst_part[8 * q4 + (j >> 2)] =
+                  make_float4(__uint_as_float(orow[j]), __uint_as_float(orow[j + 1]),
+                              __uint_as_float(orow[j + 2]), __uint_as_float(orow[j + 3]));
+          }
         }
       }
-      if (lane < 16) { sml[row * 2] = ref; sml[row * 2 + 1] = l; }
-    }
-    tc_fence_before();
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    if (alive) {
-      const int d = threadIdx.x;
-#pragma unroll 4
-      for (int r = 0; r < R; ++r) {
-        const float M = sml[r * 2], L = sml[r * 2 + 1], O = so[r * kOutPitchU + d];
-        const UserRef ur = s_users[r / G];
-        const int head = kvh * G + r % G;
-        if (ur.slot < 0) {
-          ((__nv_bfloat16*)a.out)[((size_t)ur.query * HQ + head) * kDim + d] =
-              __float2bfloat16_rn(O / L);
-        } else {
-          const size_t prow = (size_t)(ur.slot + it.slot_add) * HQ + head;
-          a.part_o[prow * kDim + d] = O;
-          if (d == 0) a.part_ml[prow] = make_float2(M, L);
-        }
-      }
+      if (mine && ur.slot >= 0) a.part_ml[prow] = make_float2(ref, l);
     }
   }
   // ---- common exit: every role arrives here, then the allocating warp frees TMEM
