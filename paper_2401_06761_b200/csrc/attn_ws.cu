@@ -1,5 +1,6 @@
 // Warp-stream attention path for work items with at most 16 query rows per kv head (the tails of
-// GQA threads, small sets of siblings): one CTA owns a whole work item, *all* kv heads.
+// GQA threads, small sets of siblings): one CTA owns a whole work item, *all* kv heads (or a
+// group of them when there are too few items to fill the machine).
 //
 // The four consumer warps each stream different kv heads, independently of one another: warp w
 // takes heads w, w+4, ...  Every warp has its own ring of four 16-token slots (K and V tile of
@@ -99,7 +100,7 @@ __device__ __forceinline__ uint32_t blk_off(int row, int c) {
 
 __global__ void __launch_bounds__(160, 1)
 attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-               const AttnArgs a, int item_begin) {
+               const AttnArgs a, int item_begin, int heads_per_cta) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (sm32(smem_raw) + 1023u) & ~1023u;
   uint8_t* bp = smem_raw + (base - sm32(smem_raw));
@@ -130,6 +131,9 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   const int32_t* table = a.d_tables + (size_t)it.table_row * a.shape.table_stride +
                          it.tok_begin / kBlock;
   const int R = it.n_users * G;                    // rows per kv head, <= 16
+  // this CTA's kv heads: [h_begin, h_begin + n_heads); warp w takes h_begin + w, + w + 4, ...
+  const int h_begin = blockIdx.y * heads_per_cta;
+  const int n_heads = min(heads_per_cta, HKV - h_begin);
 
   if (warp == 4) {
     // ------------------------------------------------------------------ producer warp
@@ -138,7 +142,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     // the op-0 lane also posts the byte count.
     if (lane < 16) {
       const int w = lane >> 2, op = lane & 3;
-      const int heads_w = (HKV - w + 3) >> 2;
+      const int heads_w = max(0, n_heads - w + 3) >> 2;
       const int total = heads_w * n_blk;
       const CUtensorMap* map = (op >> 1) ? &tm_v : &tm_k;
       int bid_next = total > 0 ? table[0] : 0;
@@ -151,7 +155,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             !wb_wait(empty_bar(w, s), ((c / kSlots) - 1) & 1, cta_abort, a.d_error, 8000 + w))
           break;
         if (op == 0) wb_expect_tx(full_bar(w, s), kSlotBytes);
-        const int h = w + 4 * hi;
+        const int h = h_begin + w + 4 * hi;
         tma2d(base + (w * kSlots + s) * kSlotBytes + (op >> 1) * kTileBytes + (op & 1) * 2048, map,
               (op & 1) * 64, (bid * HKV + h) * kBlock, full_bar(w, s));
         b = b1;
@@ -163,7 +167,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
   // -------------------------------------------------------------------- consumer warps
   const int w = warp;
-  const int heads_w = (HKV - w + 3) >> 2;
+  const int heads_w = max(0, n_heads - w + 3) >> 2;
   const int g = lane >> 2, tq = lane & 3;
   const int jm = lane >> 3, jr = lane & 7;
   const float cs = a.scale_log2e;
@@ -189,11 +193,11 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   uint32_t qa[8][4], qn[8][4];
 #pragma unroll
   for (int ks = 0; ks < 8; ++ks) qn[ks][0] = qn[ks][1] = qn[ks][2] = qn[ks][3] = 0u;
-  if (heads_w > 0) load_q(w, qa);
+  if (heads_w > 0) load_q(h_begin + w, qa);
   int c = 0;                                       // blocks consumed so far by this warp
   bool alive = true;
   for (int hi = 0; hi < heads_w && alive; ++hi) {
-    const int h = w + 4 * hi;
+    const int h = h_begin + w + 4 * hi;
     if (hi + 1 < heads_w) load_q(h + 4, qn);       // lands while this head streams
     float o[16][4];
 #pragma unroll
@@ -326,7 +330,16 @@ cudaError_t launch_attention_ws(const AttnArgs& a, int item_begin, int n_items, 
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  attn_ws_kernel<<<n_items, 160, kSmemW, st>>>(*a.tm_k, *a.tm_v, a, item_begin);
+  // Whole items per CTA when there are enough of them to fill the machine; otherwise the kv
+  // heads are dealt out over several CTAs (in multiples of the four consumer warps).
+  const int hkv = a.shape.num_kv_heads;
+  const int max_groups = (hkv + 3) / 4;
+  const int want = (2 * 148 + n_items - 1) / n_items;
+  const int groups = want < 1 ? 1 : (want > max_groups ? max_groups : want);
+  const int heads_per_cta = ((hkv + groups - 1) / groups + 3) / 4 * 4;
+  const int grid_y = (hkv + heads_per_cta - 1) / heads_per_cta;
+  attn_ws_kernel<<<dim3(n_items, grid_y), 160, kSmemW, st>>>(*a.tm_k, *a.tm_v, a, item_begin,
+                                                             heads_per_cta);
   return cudaGetLastError();
 }
 
