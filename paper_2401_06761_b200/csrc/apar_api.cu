@@ -377,7 +377,7 @@ apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
   // "vec" CUDA cores, "mma" mma.sync, "umma" tcgen05.  Default ("auto"): 1 row vec, up to 16
   // rows warp-stream (mma.sync, whole item per CTA), more rows tcgen05.
   const char* path = getenv("APAR_ATTN_PATH");
-  c->mma_min_rows = (path && !strcmp(path, "vec")) ? INT_MAX : 2;
+  c->mma_min_rows = (path && !strcmp(path, "vec")) ? INT_MAX : (path && !strcmp(path, "ws")) ? 1 : 2;
   c->umma_min_tiles = (path && !strcmp(path, "mma")) ? 5 : (path && !strcmp(path, "umma")) ? 1 : 2;
   c->use_ws = !(path && (!strcmp(path, "mma") || !strcmp(path, "umma")));
   c->ring_bytes = lay.stage_cap;

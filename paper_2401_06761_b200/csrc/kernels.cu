@@ -258,12 +258,137 @@ __global__ void __launch_bounds__(128) attn_vec_kernel(const AttnArgs a, int ite
   }
 }
 
+// Single-row items (a private tail read by one query, MHA): one CTA per item, and each of its
+// four warps walks whole kv heads on its own - warp w takes heads w, w+4, ... of the CTA's
+// group - so there is nothing to fold between warps, no shared memory and no CTA barrier, and
+// the fixed cost of a CTA is paid once per item instead of once per (item, head).  Loads are
+// the same coalesced 16-byte pattern as above; the block id of the next tile is fetched one
+// tile ahead.
+__global__ void __launch_bounds__(128) attn_vec_heads_kernel(const AttnArgs a, int item_begin,
+                                                             int heads_per_cta) {
+  const WorkItem it = a.d_items[item_begin + blockIdx.x];
+  const int HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;   // equal: group == 1
+  const int tok_end = it.tok_end < 0 ? a.d_lens[it.table_row] : it.tok_end;
+  const int n_tok = tok_end - it.tok_begin;
+  const int n_blk = (n_tok + kBlock - 1) / kBlock;
+  const int32_t* table = a.d_tables + (size_t)it.table_row * a.shape.table_stride +
+                         it.tok_begin / kBlock;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int half = lane >> 4, c = lane & 15;
+  const UserRef ur = a.d_users[it.user_begin];
+  const int h_begin = blockIdx.y * heads_per_cta;
+  const int h_end = min(HKV, h_begin + heads_per_cta);
+
+  for (int h = h_begin + warp; h < h_end; h += 4) {
+    float qf[8], o[8];
+    {
+      const uint4 qv = __ldg((const uint4*)a.q + ((size_t)ur.query * HQ + h) * 16 + c);
+      bf16x8_to_float(qv, qf);
+#pragma unroll
+      for (int d = 0; d < 8; ++d) { qf[d] *= a.scale_log2e; o[d] = 0.f; }
+    }
+    float m = -INFINITY, l = 0.f;
+    int bid = n_blk > 0 ? table[0] : 0;
+    for (int b = 0; b < n_blk; ++b) {
+      const int bid_next = b + 1 < n_blk ? table[b + 1] : 0;
+      const size_t tile = ((size_t)bid * HKV + h) * (kTileBytes / 16);
+      const uint4* kt = (const uint4*)a.k_pool + tile + half * 16 + c;
+      const uint4* vt = (const uint4*)a.v_pool + tile + half * 16 + c;
+      const int nv = min(kBlock, n_tok - b * kBlock);
+      uint4 kk[8], vv[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) kk[j] = ld_stream(kt + j * 32);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) vv[j] = ld_stream(vt + j * 32);
+      float s[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float kf[8];
+        bf16x8_to_float(kk[j], kf);
+        float acc = 0.f;
+#pragma unroll
+        for (int d = 0; d < 8; ++d) acc = fmaf(qf[d], kf[d], acc);
+        s[j] = acc;
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float x = s[j];
+        x += __shfl_xor_sync(0xffffffffu, x, 8);
+        x += __shfl_xor_sync(0xffffffffu, x, 4);
+        x += __shfl_xor_sync(0xffffffffu, x, 2);
+        x += __shfl_xor_sync(0xffffffffu, x, 1);
+        s[j] = (2 * j + half < nv) ? x : -INFINITY;      // rows past the length are never used
+      }
+      float bm = s[0];
+#pragma unroll
+      for (int j = 1; j < 8; ++j) bm = fmaxf(bm, s[j]);
+      bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));   // token 0 is always valid
+      const float mn = fmaxf(m, bm);
+      const float corr = exp2f(m - mn);
+      m = mn;
+      float ps = 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        s[j] = exp2f(s[j] - mn);
+        ps += s[j];
+      }
+      l = l * corr + ps;
+#pragma unroll
+      for (int d = 0; d < 8; ++d) o[d] *= corr;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float vf[8];
+        bf16x8_to_float(vv[j], vf);
+        if (2 * j + half >= nv) {          // unspecified bits (possibly NaN patterns): drop them
+#pragma unroll
+          for (int d = 0; d < 8; ++d) vf[d] = 0.f;
+        }
+#pragma unroll
+        for (int d = 0; d < 8; ++d) o[d] = fmaf(s[j], vf[d], o[d]);
+      }
+      bid = bid_next;
+    }
+    l += __shfl_xor_sync(0xffffffffu, l, 16);
+#pragma unroll
+    for (int d = 0; d < 8; ++d) o[d] += __shfl_xor_sync(0xffffffffu, o[d], 16);
+    if (half == 0) {
+      if (ur.slot < 0) {
+        const float inv = 1.f / l;
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(o[0] * inv, o[1] * inv);
+        __nv_bfloat162 p1 = __floats2bfloat162_rn(o[2] * inv, o[3] * inv);
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(o[4] * inv, o[5] * inv);
+        __nv_bfloat162 p3 = __floats2bfloat162_rn(o[6] * inv, o[7] * inv);
+        uint4 packed;
+        packed.x = *(uint32_t*)&p0; packed.y = *(uint32_t*)&p1;
+        packed.z = *(uint32_t*)&p2; packed.w = *(uint32_t*)&p3;
+        ((uint4*)((__nv_bfloat16*)a.out + ((size_t)ur.query * HQ + h) * kDim))[c] = packed;
+      } else {
+        const size_t prow = (size_t)(ur.slot + it.slot_add) * HQ + h;
+        float4* dst = (float4*)(a.part_o + prow * kDim) + 2 * c;
+        dst[0] = make_float4(o[0], o[1], o[2], o[3]);
+        dst[1] = make_float4(o[4], o[5], o[6], o[7]);
+        if (c == 0) a.part_ml[prow] = make_float2(m, l);
+      }
+    }
+  }
+}
+
 cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items, bool single_row,
                                  cudaStream_t st) {
   if (n_items <= 0) return cudaSuccess;
-  const dim3 grid(n_items, a.shape.num_kv_heads);
-  if (single_row) attn_vec_kernel<1><<<grid, 128, 0, st>>>(a, item_begin);
-  else attn_vec_kernel<4><<<grid, 128, 0, st>>>(a, item_begin);
+  if (single_row) {
+    // whole items per CTA when there are enough of them; otherwise heads are dealt out over
+    // several CTAs (multiples of the four warps) until the machine is full
+    const int hkv = a.shape.num_kv_heads;
+    const int max_groups = (hkv + 3) / 4;
+    const int want = (5 * 148 + n_items - 1) / n_items;
+    const int groups = want < 1 ? 1 : (want > max_groups ? max_groups : want);
+    const int heads_per_cta = ((hkv + groups - 1) / groups + 3) / 4 * 4;
+    const dim3 grid(n_items, (hkv + heads_per_cta - 1) / heads_per_cta);
+    attn_vec_heads_kernel<<<grid, 128, 0, st>>>(a, item_begin, heads_per_cta);
+  } else {
+    attn_vec_kernel<4><<<dim3(n_items, a.shape.num_kv_heads), 128, 0, st>>>(a, item_begin);
+  }
   return cudaGetLastError();
 }
 
