@@ -244,7 +244,10 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
     c->pq.resize(n);
     for (int i = 0; i < n; ++i)
       c->pq[i] = PlanQuery{c->row(qslots[i]), qslots[i], c->slots[qslots[i]].len};
+    // finishing items land in the single-row vector kernel or the warp-stream kernel
+    const bool fuse_final = c->use_ws && c->mma_min_rows <= 2;
     if (!c->planner.build(c->pq.data(), n, c->lay.slot_capacity, cacheable, c->mma_min_rows,
+                          fuse_final,
                           &c->plan))
       return APAR_ERR_WORKSPACE_TOO_SMALL;
     if ((int64_t)c->plan.users.size() > c->lay.entry_capacity ||
@@ -318,17 +321,31 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
       ++launches;
     }
     if (c->use_ws && sync_counts[0] > 0) {
-      // single-tile items are last in the list: whole items (all kv heads) per CTA
+      // single-tile items are last in the list: whole items (all kv heads) per CTA; the
+      // finishing ones wait until every other item has been launched
       const int first = p.n_vec + p.n_mma - sync_counts[0];
-      APAR_CUDA(c, launch_attention_ws(a, first, sync_counts[0], st));
+      const int n_plain = sync_counts[0] - p.n_mma1_final;
+      if (n_plain > 0) {
+        APAR_CUDA(c, launch_attention_ws(a, first, n_plain, st));
+        ++launches;
+      }
       sync_counts[0] = 0;
-      ++launches;
     }
     APAR_CUDA(c, launch_attention_mma(a, p.n_vec + n_umma, sync_counts, st));
     for (int k = 0; k < 4; ++k) launches += sync_counts[k] > 0;
   }
-  if (p.n_vec) {
-    APAR_CUDA(c, launch_attention_vec(a, 0, p.n_vec, c->shape.group == 1 && c->mma_min_rows <= 2, st));
+  const bool single_row = c->shape.group == 1 && c->mma_min_rows <= 2;
+  if (p.n_vec - p.n_vec_final > 0) {
+    APAR_CUDA(c, launch_attention_vec(a, 0, p.n_vec - p.n_vec_final, single_row, st));
+    ++launches;
+  }
+  // finishing items: everything they fold has been enqueued before them on this stream
+  if (p.n_mma1_final > 0) {
+    APAR_CUDA(c, launch_attention_ws(a, p.n_vec + p.n_mma - p.n_mma1_final, p.n_mma1_final, st));
+    ++launches;
+  }
+  if (p.n_vec_final > 0) {
+    APAR_CUDA(c, launch_attention_vec(a, p.n_vec - p.n_vec_final, p.n_vec_final, single_row, st));
     ++launches;
   }
   if (!p.merges.empty()) {

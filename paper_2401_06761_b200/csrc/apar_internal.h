@@ -25,7 +25,10 @@ struct WorkItem {
   int32_t user_begin;  // first entry of this item's users in the UserRef array
   int32_t n_users;     // queries sharing the run (rows = n_users * group)
   int32_t slot_add;    // added to every user's partial slot (chunk ordinal inside the run)
-  int32_t pad0, pad1;
+  // fin_n > 0: this is the last item of its (single) query's chain; instead of writing a
+  // partial it folds partial slots [fin_begin, fin_begin + fin_n), which earlier launches of
+  // the same call completed, into its own state and writes the final output.
+  int32_t fin_n, fin_begin;
 };
 
 // A query that reads a work item.  slot < 0: the item covers the query's whole chain and
@@ -106,8 +109,11 @@ struct PlanQuery {
 };
 
 struct Plan {
-  std::vector<WorkItem> items;     // vec items first, then mma items; each class longest first
+  // vec items (finishing ones last), then mma items by tile count 4, 3, 2, 1 (in the 1-tile
+  // class the finishing ones last); each group longest first
+  std::vector<WorkItem> items;
   int32_t n_vec = 0, n_mma = 0;
+  int32_t n_vec_final = 0, n_mma1_final = 0;   // finishing items at the end of their class
   int32_t n_mma_tiles[4] = {0, 0, 0, 0};   // mma items needing 1, 2, 3, 4 query tiles
   std::vector<UserRef> users;
   std::vector<MergeRef> merges;
@@ -123,8 +129,10 @@ class Planner {
   // from the length array), so the plan stays valid while threads only grow.
   // Items with at least mma_min_rows query rows go to the tensor-core kernel.
   // Returns false if the partial rows cannot fit `slot_capacity` even without splitting.
+  // fuse_final: the last item of a query whose chain ends in a private run of at most 16 rows
+  // finishes the query itself (see WorkItem::fin_n); such queries need no merge entry.
   bool build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_tails,
-             int mma_min_rows, Plan* out);
+             int mma_min_rows, bool fuse_final, Plan* out);
 
  private:
   int num_blocks_ = 0, group_ = 1, hint_kv_heads_ = 1;
@@ -137,7 +145,8 @@ class Planner {
   std::vector<Seg> segs_;
   std::vector<SegUser> seg_users_;
   std::vector<int32_t> n_parts_, qbeg_, part_off_;
-  std::vector<WorkItem> vec_items_, mma_items_[4];
+  std::vector<WorkItem> vec_items_, mma_items_[4], vec_final_, mma1_final_;
+  std::vector<uint8_t> fused_;
 };
 
 }  // namespace apar

@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(128) static_plan_kernel(WorkItem* items, UserR
   it.user_begin = i;
   it.n_users = 1;
   it.slot_add = s;
-  it.pad0 = it.pad1 = 0;
+  it.fin_n = it.fin_begin = 0;
   items[idx] = it;
   if (s == 0) {
     users[i] = UserRef{i, splits > 1 ? i * splits : -1};

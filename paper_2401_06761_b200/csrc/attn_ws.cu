@@ -294,8 +294,25 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       if (r < R) {
         const UserRef ur = s_users[r / G];
         const int head = h * G + r % G;
-        const float L = half ? l1 : l0, M = half ? ref1 : ref0;
-        if (ur.slot < 0) {
+        float L = half ? l1 : l0, M = half ? ref1 : ref0;
+        // a finishing item folds the partial results of the rest of the chain into its own
+        for (int pj = 0; pj < it.fin_n; ++pj) {
+          const size_t prow = (size_t)(it.fin_begin + pj) * HQ + head;
+          const float2 ml = a.part_ml[prow];
+          const float2* src = (const float2*)(a.part_o + prow * kDim) + tq;
+          const float mn = fmaxf(M, ml.x);
+          const float f0 = M == -INFINITY ? 0.f : ex2f(M - mn);
+          const float f1 = ml.x == -INFINITY ? 0.f : ex2f(ml.x - mn);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float2 x = src[4 * j];
+            o[j][2 * half] = o[j][2 * half] * f0 + x.x * f1;
+            o[j][2 * half + 1] = o[j][2 * half + 1] * f0 + x.y * f1;
+          }
+          L = L * f0 + ml.y * f1;
+          M = mn;
+        }
+        if (ur.slot < 0 || it.fin_n > 0) {
           const float inv = 1.f / L;
           uint32_t* dst = (uint32_t*)a.out + ((size_t)ur.query * HQ + head) * 64 + tq;
 #pragma unroll

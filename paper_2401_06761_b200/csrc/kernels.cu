@@ -352,7 +352,23 @@ __global__ void __launch_bounds__(128) attn_vec_heads_kernel(const AttnArgs a, i
 #pragma unroll
     for (int d = 0; d < 8; ++d) o[d] += __shfl_xor_sync(0xffffffffu, o[d], 16);
     if (half == 0) {
-      if (ur.slot < 0) {
+      // a finishing item folds the partial results of the rest of the chain into its own
+      for (int j = 0; j < it.fin_n; ++j) {
+        const size_t prow = (size_t)(it.fin_begin + j) * HQ + h;
+        const float2 ml = a.part_ml[prow];
+        const float4* src = (const float4*)(a.part_o + prow * kDim) + 2 * c;
+        const float4 x0 = src[0], x1 = src[1];
+        const float mn = fmaxf(m, ml.x);
+        const float f0 = m == -INFINITY ? 0.f : exp2f(m - mn);
+        const float f1 = ml.x == -INFINITY ? 0.f : exp2f(ml.x - mn);
+        o[0] = o[0] * f0 + x0.x * f1; o[1] = o[1] * f0 + x0.y * f1;
+        o[2] = o[2] * f0 + x0.z * f1; o[3] = o[3] * f0 + x0.w * f1;
+        o[4] = o[4] * f0 + x1.x * f1; o[5] = o[5] * f0 + x1.y * f1;
+        o[6] = o[6] * f0 + x1.z * f1; o[7] = o[7] * f0 + x1.w * f1;
+        l = l * f0 + ml.y * f1;
+        m = mn;
+      }
+      if (ur.slot < 0 || it.fin_n > 0) {
         const float inv = 1.f / l;
         __nv_bfloat162 p0 = __floats2bfloat162_rn(o[0] * inv, o[1] * inv);
         __nv_bfloat162 p1 = __floats2bfloat162_rn(o[2] * inv, o[3] * inv);

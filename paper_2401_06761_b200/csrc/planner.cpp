@@ -30,7 +30,7 @@ void Planner::init(int num_blocks, int group, int num_kv_heads) {
 static inline int64_t round_up16(int64_t x) { return (x + 15) / 16 * 16; }
 
 bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_tails,
-                    int mma_min_rows, Plan* out) {
+                    int mma_min_rows, bool fuse_final, Plan* out) {
   if (++epoch_ == 0) {
     std::fill(stamp_.begin(), stamp_.end(), 0u);
     epoch_ = 1;
@@ -128,10 +128,14 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
   out->merges.clear();
   part_off_.assign(n, -1);
   int32_t off = 0;
+  fused_.assign(n, 0);
   for (int i = 0; i < n; ++i) {
     if (n_parts_[i] >= 2) {
       part_off_[i] = off;
-      out->merges.push_back(MergeRef{i, off, n_parts_[i], 0});
+      // the chain ends in a private run: its last item can finish the query on its own
+      const Seg& last = segs_[seg_users_[qbeg_[i + 1] - 1].seg];
+      if (fuse_final && last.priv && group_ <= 16) fused_[i] = 1;
+      if (!fused_[i]) out->merges.push_back(MergeRef{i, off, n_parts_[i], 0});
       off += n_parts_[i];
     }
   }
@@ -151,6 +155,8 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
   // ---- items
   const int max_users = std::max(1, kMaxRowsPerItem / group_);
   vec_items_.clear();
+  vec_final_.clear();
+  mma1_final_.clear();
   for (auto& v : mma_items_) v.clear();
   for (const Seg& g : segs_) {
     const int32_t n_chunks = (int32_t)((g.tok_end - g.tok_begin + chunk - 1) / chunk);
@@ -167,9 +173,20 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
         it.user_begin = g.user_off + u0;
         it.n_users = nu;
         it.slot_add = c;
-        it.pad0 = it.pad1 = 0;
+        it.fin_n = it.fin_begin = 0;
         const int rows = nu * group_;
-        (rows >= mma_min_rows ? mma_items_[(rows + 15) / 16 - 1] : vec_items_).push_back(it);
+        const bool to_mma = rows >= mma_min_rows;
+        if (g.priv && g.n_users == 1 && c == n_chunks - 1) {
+          // private runs hold exactly one query; is this the end of a fused query's chain?
+          const int qi = out->users[g.user_off].query;
+          if (fused_[qi] && g.tok_end == q[qi].len) {
+            it.fin_n = n_parts_[qi] - 1;
+            it.fin_begin = part_off_[qi];
+            (to_mma ? mma1_final_ : vec_final_).push_back(it);
+            continue;
+          }
+        }
+        (to_mma ? mma_items_[(rows + 15) / 16 - 1] : vec_items_).push_back(it);
       }
     }
   }
@@ -178,16 +195,22 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
   };
   auto by_cost = [&](const WorkItem& a, const WorkItem& b) { return cost(a) > cost(b); };
   std::stable_sort(vec_items_.begin(), vec_items_.end(), by_cost);
-  out->n_vec = (int32_t)vec_items_.size();
+  std::stable_sort(vec_final_.begin(), vec_final_.end(), by_cost);
+  std::stable_sort(mma1_final_.begin(), mma1_final_.end(), by_cost);
+  out->n_vec_final = (int32_t)vec_final_.size();
+  out->n_mma1_final = (int32_t)mma1_final_.size();
+  out->n_vec = (int32_t)(vec_items_.size() + vec_final_.size());
   out->n_mma = 0;
   out->items.clear();
   out->items.insert(out->items.end(), vec_items_.begin(), vec_items_.end());
+  out->items.insert(out->items.end(), vec_final_.begin(), vec_final_.end());
   for (int k = 3; k >= 0; --k) {          // widest items first
     std::stable_sort(mma_items_[k].begin(), mma_items_[k].end(), by_cost);
-    out->n_mma_tiles[k] = (int32_t)mma_items_[k].size();
+    out->n_mma_tiles[k] = (int32_t)mma_items_[k].size() + (k == 0 ? out->n_mma1_final : 0);
     out->n_mma += out->n_mma_tiles[k];
     out->items.insert(out->items.end(), mma_items_[k].begin(), mma_items_[k].end());
   }
+  out->items.insert(out->items.end(), mma1_final_.begin(), mma1_final_.end());
   out->total_slots = total_slots;
   out->unique_tokens = unique;
   out->attended_tokens = attended;
