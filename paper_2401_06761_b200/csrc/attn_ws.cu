@@ -3,13 +3,15 @@
 // group of them when there are too few items to fill the machine).
 //
 // The four consumer warps each stream different kv heads, independently of one another: warp w
-// takes heads w, w+4, ...  Every warp has its own ring of four 16-token slots (K and V tile of
+// takes heads w, w+4, ...  Every warp has its own ring of three 16-token slots (K and V tile of
 // one block, 8 KiB) filled by the producer warp with TMA tensor copies, its own mbarriers, and
 // keeps Q (as mma.sync A-fragments, fetched straight from global memory one head ahead), the
 // online-softmax state and O in registers.  There is no CTA-wide synchronisation inside the
 // loop, no folding between warps, and the fixed cost of a CTA (item, users, first TMA round
 // trip, write-out) is paid once per item instead of once per (item, head), which is what the
-// short tails of decode batches are sensitive to.  One CTA per SM keeps 128 KiB in flight.
+// short tails of decode batches are sensitive to.  Two CTAs per SM, each with four rings of
+// three 8 KiB slots, keep up to 192 KiB in flight and overlap one CTA's start-up and
+// write-out with the other's streaming.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -19,7 +21,7 @@
 namespace apar {
 namespace {
 
-constexpr int kSlots = 4;                           // ring depth per consumer warp
+constexpr int kSlots = 3;                           // ring depth per consumer warp
 constexpr int kSlotBytes = 2 * kTileBytes;          // K tile + V tile of one block: 8 KiB
 constexpr int kRingBytes = 4 * kSlots * kSlotBytes; // 128 KiB
 constexpr int kUsersOffW = kRingBytes;              // UserRef[16]
@@ -98,7 +100,7 @@ __device__ __forceinline__ uint32_t blk_off(int row, int c) {
   return (uint32_t)((c >> 3) * 2048 + row * 128 + (((c & 7) ^ (row & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(160, 1)
+__global__ void __launch_bounds__(160, 2)
 attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                const AttnArgs a, int item_begin, int heads_per_cta) {
   extern __shared__ uint8_t smem_raw[];
@@ -351,7 +353,7 @@ cudaError_t launch_attention_ws(const AttnArgs& a, int item_begin, int n_items, 
   // heads are dealt out over several CTAs (in multiples of the four consumer warps).
   const int hkv = a.shape.num_kv_heads;
   const int max_groups = (hkv + 3) / 4;
-  const int want = (2 * 148 + n_items - 1) / n_items;
+  const int want = (4 * 148 + n_items - 1) / n_items;
   const int groups = want < 1 ? 1 : (want > max_groups ? max_groups : want);
   const int heads_per_cta = ((hkv + groups - 1) / groups + 3) / 4 * 4;
   const int grid_y = (hkv + heads_per_cta - 1) / heads_per_cta;
