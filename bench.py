@@ -197,7 +197,7 @@ def run_ours(args, cfg_id):
     out = torch.empty(q_shape, dtype=torch.bfloat16, device=dev)
     attn_events = []
 
-    def one_step(q, k_new, v_new, record):
+    def one_step(q, k_new, v_new, record, stream=stream, out=out):
         """fork (if the workload has one) + append + attention [+ release of the step's forks]."""
         kids = B.apar_fork(sess.ctx, step0.fork_parents, stream) if step0.fork_parents else []
         live = B.int32_array(base_live + kids) if kids else base_live_arr
@@ -256,16 +256,38 @@ def run_ours(args, cfg_id):
     for i in range(2):
         hq[i].copy_(inputs[i % len(inputs)][0]); hk[i].copy_(inputs[i % len(inputs)][1])
         hv[i].copy_(inputs[i % len(inputs)][2])
-    dq, dk, dv = (torch.empty(q_shape, dtype=torch.bfloat16, device=dev),
-                  torch.empty(row_shape, dtype=torch.bfloat16, device=dev),
-                  torch.empty(row_shape, dtype=torch.bfloat16, device=dev))
+    # A serving loop would overlap the copies of neighbouring steps with compute, so the end-to-
+    # end arm does: inputs of step i+1 go up (copy stream) and the result of step i-1 comes
+    # down (second copy stream) while step i computes, with two device buffers of each kind.
+    # Every step's own copies are inside the timed region.
+    dq = [torch.empty(q_shape, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    dk = [torch.empty(row_shape, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    dv = [torch.empty(row_shape, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    dout = [torch.empty(q_shape, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    s_cmp = torch.cuda.current_stream()
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_cmp = [torch.cuda.Event() for _ in range(2)]
+    ev_out = [torch.cuda.Event() for _ in range(2)]
 
     def e2e_step(i):
-        dq.copy_(hq[i % 2], non_blocking=True)
-        dk.copy_(hk[i % 2], non_blocking=True)
-        dv.copy_(hv[i % 2], non_blocking=True)
-        one_step(dq, dk, dv, record=False)
-        hout.copy_(out, non_blocking=True)
+        b = i % 2
+        with torch.cuda.stream(s_in):
+            if i >= 2:
+                s_in.wait_event(ev_cmp[b])          # step i-2 has consumed these input buffers
+            dq[b].copy_(hq[b], non_blocking=True)
+            dk[b].copy_(hk[b], non_blocking=True)
+            dv[b].copy_(hv[b], non_blocking=True)
+            ev_in[b].record(s_in)
+        s_cmp.wait_event(ev_in[b])
+        if i >= 2:
+            s_cmp.wait_event(ev_out[b])             # the result of step i-2 has left dout[b]
+        one_step(dq[b], dk[b], dv[b], record=False, out=dout[b])
+        ev_cmp[b].record(s_cmp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_cmp[b])
+            hout.copy_(dout[b], non_blocking=True)
+            ev_out[b].record(s_out)
 
     e2e_steps = max(1, min(args.steps, steps_total - 1))
     e2e_step(0)
@@ -273,10 +295,13 @@ def run_ours(args, cfg_id):
     ev0.record()
     for i in range(e2e_steps):
         e2e_step(i)
+    s_cmp.wait_event(ev_out[(e2e_steps - 1) % 2])
+    if e2e_steps >= 2:
+        s_cmp.wait_event(ev_out[e2e_steps % 2])
     ev1.record()
     barrier()
     e2e_ms = max_over_ranks(ev0.elapsed_time(ev1))
-    h2d = sum(t.numel() * 2 for t in (dq, dk, dv))
+    h2d = sum(t[0].numel() * 2 for t in (dq, dk, dv))
     d2h = out.numel() * 2
 
     # ---------------- numbers
