@@ -100,6 +100,8 @@ typedef struct {
   int64_t attn_vec_items;         /* items on the CUDA-core vector path                          */
   int64_t attn_mma_items;         /* items on the tensor-core path                               */
   int64_t kernels_total;          /* kernels launched by this context since creation             */
+  int64_t peak_used_blocks;       /* most blocks ever in use at once (x16 = "max cached tokens",
+                                     Section 3.4, in block granularity)                           */
   int64_t device_wait_timeouts;   /* non-zero once a kernel gave up a bounded wait (results of
                                      that call are invalid); reading it synchronises the device   */
 } apar_stats;

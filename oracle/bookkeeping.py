@@ -37,12 +37,14 @@ class BlockModel:
         self.next_tid = 0
         self.cow_blocks = 0   # blocks copied by forks so far
         self.cow_rows = 0     # token rows copied by forks so far
+        self.peak_used = 0    # most blocks in use at once so far
 
     # ------------------------------------------------------------ helpers
     def _alloc(self) -> int:
         b = self.free.pop()
         assert self.refcount[b] == 0
         self.refcount[b] = 1
+        self.peak_used = max(self.peak_used, self.num_blocks - len(self.free))
         return b
 
     def _check_live(self, tids):

@@ -41,7 +41,7 @@ class apar_stats(C.Structure):
         "live_threads", "free_blocks", "used_blocks", "forks", "cow_blocks", "cow_rows",
         "attn_threads", "attn_attended_tokens", "attn_unique_tokens", "attn_work_items",
         "attn_partials", "attn_kernels", "attn_plan_reused", "attn_vec_items",
-        "attn_mma_items", "kernels_total", "device_wait_timeouts")]
+        "attn_mma_items", "kernels_total", "peak_used_blocks", "device_wait_timeouts")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}

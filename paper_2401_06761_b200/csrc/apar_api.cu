@@ -84,7 +84,7 @@ struct apar_ctx {
   std::vector<int32_t> tid_slot;       // tid -> slot or -1
   int32_t next_tid = 0;
   int64_t live = 0;
-  int64_t forks = 0, cow_blocks = 0, cow_rows = 0, kernels_total = 0;
+  int64_t forks = 0, cow_blocks = 0, cow_rows = 0, kernels_total = 0, peak_used = 0;
   apar_stats last = {};
   std::vector<uint32_t> mark;          // per slot, duplicate detection
   uint32_t mark_epoch = 0;
@@ -169,6 +169,7 @@ int32_t alloc_block(apar_ctx* c) {
   const int32_t b = c->free_stack.back();
   c->free_stack.pop_back();
   c->refcnt[b] = 1;
+  c->peak_used = std::max<int64_t>(c->peak_used, c->cfg.num_blocks - (int64_t)c->free_stack.size());
   return b;
 }
 
@@ -697,6 +698,7 @@ apar_status apar_get_stats(apar_ctx* c, apar_stats* out) {
   out->cow_blocks = c->cow_blocks;
   out->cow_rows = c->cow_rows;
   out->kernels_total = c->kernels_total;
+  out->peak_used_blocks = c->peak_used;
   int32_t flag = 0;   // synchronises with the device: introspection only
   if (cudaMemcpy(&flag, c->ws(c->lay.err), 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
     c->last_cuda = (int32_t)cudaGetLastError();

@@ -294,3 +294,87 @@ def run_step_forks(step: StepInputs, backend) -> None:
         for n, h in zip(step.fork_nodes, backend.fork(step.fork_parents)):
             step.handles[n.index] = h
         step.live_handles = [step.handles[n.index] for n in step.live_nodes]
+
+
+# ------------------------------------------------------------------ request lifecycle replay
+
+@dataclass
+class LifecycleStep:
+    """Events of one decode step, in the order of Algorithm 1: new requests are admitted, threads
+    whose last token was the fork token are duplicated, every live thread appends one token (and
+    attends), threads that produced the end token finish."""
+    arrive: List[tuple] = field(default_factory=list)   # (thread key, request, prompt length)
+    fork: List[tuple] = field(default_factory=list)     # (parent key, child key)
+    finish: List[int] = field(default_factory=list)     # thread keys
+
+
+def lifecycle_schedule(seed: int, n_requests: int, n_steps: int, max_live: int = 48):
+    """A token-free replay of Algorithm 1 for a stream of requests: which thread forks and which
+    one finishes at which step.  Thread keys are small integers private to the schedule.
+    Returns (steps, request_of_thread)."""
+    rng = np.random.default_rng(seed)
+    steps: List[LifecycleStep] = []
+    remaining = {}            # live thread key -> tokens still to generate
+    request_of = {}
+    next_key, admitted = 0, 0
+    for _ in range(n_steps):
+        st = LifecycleStep()
+        while admitted < n_requests and len(remaining) < max_live // 2 and rng.random() < 0.5:
+            st.arrive.append((next_key, admitted, int(rng.integers(5, 90))))
+            remaining[next_key] = int(rng.integers(20, 120))
+            request_of[next_key] = admitted
+            next_key += 1
+            admitted += 1
+        for key in list(remaining):
+            if len(remaining) < max_live and remaining[key] > 8 and rng.random() < 0.06:
+                st.fork.append((key, next_key))            # the child writes the detail paragraph
+                remaining[next_key] = int(rng.integers(4, 60))
+                request_of[next_key] = request_of[key]
+                next_key += 1
+        for key in list(remaining):
+            remaining[key] -= 1
+            if remaining[key] <= 0:
+                st.finish.append(key)
+                del remaining[key]
+        steps.append(st)
+    return steps, request_of
+
+
+def run_lifecycle(steps, request_of, backend, rows, early_release: bool = True, on_step=None):
+    """Drive `backend` through the schedule.  `rows(n)` supplies (k, v) for n new token rows.
+    With early_release a thread's cache is released the moment it finishes (Section 2.3);
+    otherwise only when its whole request has finished.  on_step(step_index, live_handles) runs
+    after the step's appends."""
+    handle, live, finished_of_request, alive_of_request = {}, [], {}, {}
+    for i, st in enumerate(steps):
+        if st.arrive:
+            hs = backend.new_threads(len(st.arrive))
+            counts = [p for _, _, p in st.arrive]
+            backend.append(hs, counts, *rows(sum(counts)))
+            for (key, req, _), h in zip(st.arrive, hs):
+                handle[key] = h
+                live.append(key)
+                alive_of_request[req] = alive_of_request.get(req, 0) + 1
+        if st.fork:
+            hs = backend.fork([handle[p] for p, _ in st.fork])
+            for (_, child), h in zip(st.fork, hs):
+                handle[child] = h
+                live.append(child)
+                alive_of_request[request_of[child]] += 1
+        if live:
+            backend.append([handle[k] for k in live], None, *rows(len(live)))
+            if on_step is not None:
+                on_step(i, [handle[k] for k in live])
+        for key in st.finish:
+            live.remove(key)
+            req = request_of[key]
+            alive_of_request[req] -= 1
+            if early_release:
+                backend.release([handle[key]])
+            else:
+                finished_of_request.setdefault(req, []).append(handle[key])
+                if alive_of_request[req] == 0:
+                    backend.release(finished_of_request.pop(req))
+    leftovers = [handle[k] for k in live] + [h for hs in finished_of_request.values() for h in hs]
+    if leftovers:
+        backend.release(leftovers)
