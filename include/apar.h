@@ -27,8 +27,9 @@
  *     There is no CPU fallback: without a usable CUDA device calls fail with APAR_ERR_CUDA.
  *
  * Layout of the KV pool (fixed): K pool and V pool are each
- *       bf16 [num_blocks][num_kv_heads][block_size = 16][head_dim = 128],
- *   so the rows of one (block, kv head) form a contiguous 4 KiB tile.  Q, out:
+ *       bf16 [num_layers][num_blocks][num_kv_heads][block_size = 16][head_dim = 128],
+ *   so the rows of one (layer, block, kv head) form a contiguous 4 KiB tile.  All layers share
+ *   one set of block tables: block b of layer l is the same logical block in every layer.  Q, out:
  *   bf16 [n][num_q_heads][128].  k_new, v_new: bf16 [rows][num_kv_heads][128].
  *   Query head h reads KV head h / (num_q_heads / num_kv_heads).
  *
@@ -76,8 +77,9 @@ typedef struct {
   int32_t head_dim;               /* must be 128                                                 */
   int32_t max_threads;            /* live generation threads at any time                         */
   int32_t max_blocks_per_thread;  /* longest chain, in blocks                                    */
-  void*   k_pool;                 /* [device] caller-owned, 1024-byte aligned                    */
-  void*   v_pool;                 /* [device] caller-owned, 1024-byte aligned                    */
+  int32_t num_layers;             /* attention layers that share the block tables; 0 means 1     */
+  void*   k_pool;                 /* [device] caller-owned, 256-byte aligned                     */
+  void*   v_pool;                 /* [device] caller-owned, 256-byte aligned                     */
   void*   workspace;              /* [device] caller-owned scratch, 256-byte aligned             */
   size_t  workspace_bytes;        /* >= apar_workspace_bytes(cfg)                                */
 } apar_config;
@@ -153,6 +155,26 @@ apar_status apar_append_kv(apar_ctx* ctx, int32_t n, const int32_t* tid /*[host]
 apar_status apar_tree_decode_attention(apar_ctx* ctx, int32_t n, const int32_t* tid /*[host]*/,
                                        const void* q /*[device]*/, void* out /*[device]*/,
                                        float sm_scale, void* cuda_stream);
+
+/* The same decode step for the other attention layers of a model (Algorithm 1's Sample runs
+ * every layer over the same sequences; the paper states nothing per layer).  Both calls reuse
+ * what the most recent apar_append_kv / apar_tree_decode_attention of this context prepared on
+ * the device - the slot of every new row, the work plan - and do no bookkeeping, no planning
+ * and no host-to-device copy: they only launch kernels on layer `layer` (0 <= layer <
+ * num_layers) of the pools.
+ *   apar_append_kv_layer: k_new / v_new [device] hold the same rows, in the same order, as in
+ *     that apar_append_kv call (which itself wrote layer 0).  At most 262144 rows are retained
+ *     per call; a larger call cannot be replayed (APAR_ERR_WORKSPACE_TOO_SMALL).
+ *   apar_tree_decode_attention_layer: same queries, in the same order, as in that attention
+ *     call (which itself ran on layer 0).  Fails with APAR_ERR_INVALID_ARG if any bookkeeping
+ *     call (new_threads, fork, append, release) came after it.
+ * apar_fork copies the partial block in every layer.
+ * Errors: INVALID_ARG, WORKSPACE_TOO_SMALL, CUDA. */
+apar_status apar_append_kv_layer(apar_ctx* ctx, int32_t layer, const void* k_new /*[device]*/,
+                                 const void* v_new /*[device]*/, void* cuda_stream);
+apar_status apar_tree_decode_attention_layer(apar_ctx* ctx, int32_t layer,
+                                             const void* q /*[device]*/, void* out /*[device]*/,
+                                             float sm_scale, void* cuda_stream);
 
 /* ReleaseCache (Algorithm 1; Section 2.3: a finished sequence gives back the cache that no
  * other sequence holds):

@@ -31,7 +31,7 @@ class apar_config(C.Structure):
     _fields_ = [("num_blocks", C.c_int32), ("block_size", C.c_int32),
                 ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("max_threads", C.c_int32),
-                ("max_blocks_per_thread", C.c_int32),
+                ("max_blocks_per_thread", C.c_int32), ("num_layers", C.c_int32),
                 ("k_pool", C.c_void_p), ("v_pool", C.c_void_p),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
 
@@ -61,6 +61,9 @@ _SIGS = {
                                    C.c_void_p]),
     "apar_tree_decode_attention": (C.c_int32, [_ctx, C.c_int32, _i32p, C.c_void_p, C.c_void_p,
                                                C.c_float, C.c_void_p]),
+    "apar_append_kv_layer": (C.c_int32, [_ctx, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "apar_tree_decode_attention_layer": (C.c_int32, [_ctx, C.c_int32, C.c_void_p, C.c_void_p,
+                                                     C.c_float, C.c_void_p]),
     "apar_release": (C.c_int32, [_ctx, C.c_int32, _i32p]),
     "apar_tree_decode_attention_tables": (C.c_int32, [_cfgp, C.c_int32, _i32p, _i32p,
                                                       C.c_void_p, C.c_void_p, C.c_float,
@@ -96,9 +99,11 @@ def _check(status: int):
 
 
 def make_config(num_blocks, num_q_heads, num_kv_heads, max_threads, max_blocks_per_thread,
-                k_pool=0, v_pool=0, workspace=0, workspace_bytes=0, block_size=16, head_dim=128):
+                k_pool=0, v_pool=0, workspace=0, workspace_bytes=0, block_size=16, head_dim=128,
+                num_layers=1):
     return apar_config(num_blocks, block_size, num_q_heads, num_kv_heads, head_dim, max_threads,
-                       max_blocks_per_thread, k_pool, v_pool, workspace, workspace_bytes)
+                       max_blocks_per_thread, num_layers, k_pool, v_pool, workspace,
+                       workspace_bytes)
 
 
 def apar_workspace_bytes(cfg: apar_config) -> int:
@@ -137,6 +142,14 @@ def apar_append_kv(ctx, tid, n_tok, k_new: int, v_new: int, stream=0):
 def apar_tree_decode_attention(ctx, tid, q: int, out: int, sm_scale: float, stream=0):
     tids, n = _arr(tid)
     _check(lib.apar_tree_decode_attention(ctx, n, tids, q, out, sm_scale, stream))
+
+
+def apar_append_kv_layer(ctx, layer: int, k_new: int, v_new: int, stream=0):
+    _check(lib.apar_append_kv_layer(ctx, layer, k_new, v_new, stream))
+
+
+def apar_tree_decode_attention_layer(ctx, layer: int, q: int, out: int, sm_scale: float, stream=0):
+    _check(lib.apar_tree_decode_attention_layer(ctx, layer, q, out, sm_scale, stream))
 
 
 def apar_release(ctx, tid):

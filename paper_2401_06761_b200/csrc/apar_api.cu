@@ -17,11 +17,12 @@ namespace {
 
 constexpr int kRing = 4;              // pinned staging buffers in flight
 constexpr int kSlotsPerThread = 6;    // partial-result rows provisioned per live thread
+constexpr int kSlotMapRows = 262144;  // new-row slots of the last append kept for other layers
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {            // partition of the caller's workspace
-  size_t err, tables, lens, stage, plan_items, plan_users, plan_merges, part_ml, part_o, total;
+  size_t err, tables, lens, stage, slot_map, plan_items, plan_users, plan_merges, part_ml, part_o, total;
   size_t stage_cap;        // bytes of the transient staging area
   int64_t slot_capacity;   // partial rows (before the head dimension)
   int64_t entry_capacity;  // (item, user) pairs a plan may hold
@@ -30,8 +31,9 @@ struct Layout {            // partition of the caller's workspace
 bool supported(const apar_config* c) {
   return c && c->block_size == kBlock && c->head_dim == kDim && c->num_blocks > 0 &&
          c->num_kv_heads > 0 && c->num_q_heads > 0 && c->num_q_heads % c->num_kv_heads == 0 &&
-         c->max_threads > 0 && c->max_blocks_per_thread > 0 &&
-         (int64_t)c->num_blocks * kBlock < INT32_MAX;
+         c->max_threads > 0 && c->max_blocks_per_thread > 0 && c->num_layers >= 0 &&
+         (int64_t)c->num_blocks * kBlock < INT32_MAX &&
+         (int64_t)std::max(1, c->num_layers) * c->num_blocks * c->num_kv_heads * kBlock < INT32_MAX;
 }
 
 Layout make_layout(const apar_config* c) {
@@ -46,6 +48,7 @@ Layout make_layout(const apar_config* c) {
   L.tables = take(table_bytes);
   L.lens = take((size_t)c->max_threads * 4);
   L.stage = take(L.stage_cap);
+  L.slot_map = take((size_t)kSlotMapRows * 4);
   L.plan_items = take((size_t)L.entry_capacity * sizeof(WorkItem));
   L.plan_users = take((size_t)L.entry_capacity * sizeof(UserRef));
   L.plan_merges = take((size_t)c->max_threads * sizeof(MergeRef));
@@ -103,7 +106,11 @@ struct apar_ctx {
   int mma_min_rows = INT_MAX;
   int umma_min_tiles = 2;               // items with at least this many 16-row tiles use tcgen05
   bool use_ws = true;                   // single-tile items use the warp-stream kernel
-  CUtensorMap tm_k, tm_v;
+  std::vector<CUtensorMap> tm_k, tm_v;   // one pair per layer
+  size_t layer_bytes = 0;                // bytes of one layer of a pool
+  int num_layers = 1;
+  uint64_t book_seq = 1, attn_book_seq = 0;   // bookkeeping calls so far / at the last plan
+  int64_t last_append_rows = -1;              // rows of the last append kept in the slot map
   int32_t last_cuda = 0;
   bool external_tables = false;        // the table-driven entry point owns no pool state
 
@@ -228,6 +235,74 @@ apar_status sync_device_tables(apar_ctx* c, const int32_t* slots, int n, cudaStr
   return APAR_OK;
 }
 
+// Launch sequence of the current plan on one layer of the pools.
+apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float sm_scale,
+                        cudaStream_t st, int* launches_out) {
+  const Plan& p = c->plan;
+  AttnArgs a;
+  a.q = q;
+  a.out = out;
+  a.k_pool = (const char*)c->cfg.k_pool + (size_t)layer * c->layer_bytes;
+  a.v_pool = (const char*)c->cfg.v_pool + (size_t)layer * c->layer_bytes;
+  a.d_tables = (const int32_t*)c->ws(c->lay.tables);
+  a.d_lens = (const int32_t*)c->ws(c->lay.lens);
+  a.d_items = (const WorkItem*)c->ws(c->lay.plan_items);
+  a.d_users = (const UserRef*)c->ws(c->lay.plan_users);
+  a.part_o = (float*)c->ws(c->lay.part_o);
+  a.part_ml = (float2*)c->ws(c->lay.part_ml);
+  a.shape = c->shape;
+  a.scale_log2e = sm_scale * 1.4426950408889634f;
+  a.tm_k = &c->tm_k[layer];
+  a.tm_v = &c->tm_v[layer];
+  a.d_error = (int*)c->ws(c->lay.err);
+  if (p.n_mma) {
+    // items are ordered 4, 3, 2, 1 query tiles: the first umma_min_tiles.. classes go to tcgen05
+    int32_t sync_counts[4], n_umma = 0;
+    for (int k = 0; k < 4; ++k) {
+      const bool umma = k + 1 >= c->umma_min_tiles;
+      sync_counts[k] = umma ? 0 : p.n_mma_tiles[k];
+      if (umma) n_umma += p.n_mma_tiles[k];
+    }
+    if (n_umma) {
+      APAR_CUDA(c, launch_attention_umma(a, p.n_vec, n_umma, st));
+      ++*launches_out;
+    }
+    if (c->use_ws && sync_counts[0] > 0) {
+      // single-tile items are last in the list: whole items (all kv heads) per CTA; the
+      // finishing ones wait until every other item has been launched
+      const int first = p.n_vec + p.n_mma - sync_counts[0];
+      const int n_plain = sync_counts[0] - p.n_mma1_final;
+      if (n_plain > 0) {
+        APAR_CUDA(c, launch_attention_ws(a, first, n_plain, st));
+        ++*launches_out;
+      }
+      sync_counts[0] = 0;
+    }
+    APAR_CUDA(c, launch_attention_mma(a, p.n_vec + n_umma, sync_counts, st));
+    for (int k = 0; k < 4; ++k) (*launches_out) += sync_counts[k] > 0;
+  }
+  const bool single_row = c->shape.group == 1 && c->mma_min_rows <= 2;
+  if (p.n_vec - p.n_vec_final > 0) {
+    APAR_CUDA(c, launch_attention_vec(a, 0, p.n_vec - p.n_vec_final, single_row, st));
+    ++*launches_out;
+  }
+  // finishing items: everything they fold has been enqueued before them on this stream
+  if (p.n_mma1_final > 0) {
+    APAR_CUDA(c, launch_attention_ws(a, p.n_vec + p.n_mma - p.n_mma1_final, p.n_mma1_final, st));
+    ++*launches_out;
+  }
+  if (p.n_vec_final > 0) {
+    APAR_CUDA(c, launch_attention_vec(a, p.n_vec - p.n_vec_final, p.n_vec_final, single_row, st));
+    ++*launches_out;
+  }
+  if (!p.merges.empty()) {
+    APAR_CUDA(c, launch_merge(a, (const MergeRef*)c->ws(c->lay.plan_merges),
+                              (int)p.merges.size(), st));
+    ++*launches_out;
+  }
+  return APAR_OK;
+}
+
 // The attention launch sequence for queries given as slots (already validated, len > 0).
 apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32_t* tids,
                           bool has_dups, const void* q, void* out, float sm_scale,
@@ -292,68 +367,10 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
     ++c->plan_age;
   }
 
-  AttnArgs a;
-  a.q = q;
-  a.out = out;
-  a.k_pool = c->cfg.k_pool;
-  a.v_pool = c->cfg.v_pool;
-  a.d_tables = (const int32_t*)c->ws(c->lay.tables);
-  a.d_lens = (const int32_t*)c->ws(c->lay.lens);
-  a.d_items = (const WorkItem*)c->ws(c->lay.plan_items);
-  a.d_users = (const UserRef*)c->ws(c->lay.plan_users);
-  a.part_o = (float*)c->ws(c->lay.part_o);
-  a.part_ml = (float2*)c->ws(c->lay.part_ml);
-  a.shape = c->shape;
-  a.scale_log2e = sm_scale * 1.4426950408889634f;
-  a.tm_k = &c->tm_k;
-  a.tm_v = &c->tm_v;
-  a.d_error = (int*)c->ws(c->lay.err);
   int launches = 0;
-  if (p.n_mma) {
-    // items are ordered 4, 3, 2, 1 query tiles: the first umma_min_tiles.. classes go to tcgen05
-    int32_t sync_counts[4], n_umma = 0;
-    for (int k = 0; k < 4; ++k) {
-      const bool umma = k + 1 >= c->umma_min_tiles;
-      sync_counts[k] = umma ? 0 : p.n_mma_tiles[k];
-      if (umma) n_umma += p.n_mma_tiles[k];
-    }
-    if (n_umma) {
-      APAR_CUDA(c, launch_attention_umma(a, p.n_vec, n_umma, st));
-      ++launches;
-    }
-    if (c->use_ws && sync_counts[0] > 0) {
-      // single-tile items are last in the list: whole items (all kv heads) per CTA; the
-      // finishing ones wait until every other item has been launched
-      const int first = p.n_vec + p.n_mma - sync_counts[0];
-      const int n_plain = sync_counts[0] - p.n_mma1_final;
-      if (n_plain > 0) {
-        APAR_CUDA(c, launch_attention_ws(a, first, n_plain, st));
-        ++launches;
-      }
-      sync_counts[0] = 0;
-    }
-    APAR_CUDA(c, launch_attention_mma(a, p.n_vec + n_umma, sync_counts, st));
-    for (int k = 0; k < 4; ++k) launches += sync_counts[k] > 0;
-  }
-  const bool single_row = c->shape.group == 1 && c->mma_min_rows <= 2;
-  if (p.n_vec - p.n_vec_final > 0) {
-    APAR_CUDA(c, launch_attention_vec(a, 0, p.n_vec - p.n_vec_final, single_row, st));
-    ++launches;
-  }
-  // finishing items: everything they fold has been enqueued before them on this stream
-  if (p.n_mma1_final > 0) {
-    APAR_CUDA(c, launch_attention_ws(a, p.n_vec + p.n_mma - p.n_mma1_final, p.n_mma1_final, st));
-    ++launches;
-  }
-  if (p.n_vec_final > 0) {
-    APAR_CUDA(c, launch_attention_vec(a, p.n_vec - p.n_vec_final, p.n_vec_final, single_row, st));
-    ++launches;
-  }
-  if (!p.merges.empty()) {
-    APAR_CUDA(c, launch_merge(a, (const MergeRef*)c->ws(c->lay.plan_merges),
-                              (int)p.merges.size(), st));
-    ++launches;
-  }
+  rc = launch_plan(c, 0, q, out, sm_scale, st, &launches);
+  if (rc) return rc;
+  c->attn_book_seq = c->book_seq;
   c->kernels_total += launches;
   c->last.attn_kernels += launches;
   c->last.attn_threads = n;
@@ -371,7 +388,7 @@ apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
   if (!cfg || !out) return APAR_ERR_INVALID_ARG;
   if (!supported(cfg)) return APAR_ERR_UNSUPPORTED;
   if (!cfg->k_pool || !cfg->v_pool || !cfg->workspace) return APAR_ERR_INVALID_ARG;
-  if (((uintptr_t)cfg->k_pool | (uintptr_t)cfg->v_pool) & 1023) return APAR_ERR_INVALID_ARG;
+  if (((uintptr_t)cfg->k_pool | (uintptr_t)cfg->v_pool) & 255) return APAR_ERR_INVALID_ARG;
   if ((uintptr_t)cfg->workspace & 255) return APAR_ERR_INVALID_ARG;
   const Layout lay = make_layout(cfg);
   if (cfg->workspace_bytes < lay.total) return APAR_ERR_WORKSPACE_TOO_SMALL;
@@ -399,9 +416,16 @@ apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
   c->umma_min_tiles = (path && !strcmp(path, "mma")) ? 5 : (path && !strcmp(path, "umma")) ? 1 : 2;
   c->use_ws = !(path && (!strcmp(path, "mma") || !strcmp(path, "umma")));
   c->ring_bytes = lay.stage_cap;
-  if (make_pool_tensor_maps(cfg->k_pool, cfg->v_pool, cfg->num_blocks, cfg->num_kv_heads,
-                            &c->tm_k, &c->tm_v) != 0 ||
-      cudaMemset(c->ws(lay.err), 0, 256) != cudaSuccess) {
+  c->num_layers = std::max(1, cfg->num_layers);
+  c->layer_bytes = (size_t)cfg->num_blocks * cfg->num_kv_heads * kTileBytes;
+  c->tm_k.resize(c->num_layers);
+  c->tm_v.resize(c->num_layers);
+  bool maps_ok = true;
+  for (int l = 0; l < c->num_layers && maps_ok; ++l)
+    maps_ok = make_pool_tensor_maps((char*)cfg->k_pool + l * c->layer_bytes,
+                                    (char*)cfg->v_pool + l * c->layer_bytes, cfg->num_blocks,
+                                    cfg->num_kv_heads, &c->tm_k[l], &c->tm_v[l]) == 0;
+  if (!maps_ok || cudaMemset(c->ws(lay.err), 0, 256) != cudaSuccess) {
     c->last_cuda = (int32_t)cudaGetLastError();
     delete c;
     return APAR_ERR_CUDA;
@@ -447,6 +471,7 @@ apar_status apar_new_threads(apar_ctx* c, int32_t n, int32_t* tid_out) {
   if (c->live + n > c->cfg.max_threads) return APAR_ERR_NO_THREADS;
   for (int i = 0; i < n; ++i) tid_out[i] = c->slots[new_slot(c)].tid;
   if (n) ++c->struct_epoch;
+  ++c->book_seq;
   return APAR_OK;
 }
 
@@ -495,13 +520,17 @@ apar_status apar_fork(apar_ctx* c, int32_t n, const int32_t* parent_tid, int32_t
     ++c->forks;
   }
   if (n) ++c->struct_epoch;
+  ++c->book_seq;
   if (nc) {
     char* d_stage = c->ws(c->lay.stage);
     apar_status rc = send(c, stg, d_stage, (size_t)nc * sizeof(CowCopy), st);
     if (rc) return rc;
-    APAR_CUDA(c, launch_cow_copy(c->cfg.k_pool, c->cfg.v_pool, (const CowCopy*)d_stage, nc,
-                                 c->cfg.num_kv_heads, st));
-    ++c->kernels_total;
+    for (int l = 0; l < c->num_layers; ++l) {
+      APAR_CUDA(c, launch_cow_copy((char*)c->cfg.k_pool + l * c->layer_bytes,
+                                   (char*)c->cfg.v_pool + l * c->layer_bytes,
+                                   (const CowCopy*)d_stage, nc, c->cfg.num_kv_heads, st));
+      ++c->kernels_total;
+    }
   }
   return APAR_OK;
 }
@@ -529,7 +558,11 @@ apar_status apar_append_kv(apar_ctx* c, int32_t n, const int32_t* tid, const int
   }
   if (need > (int64_t)c->free_stack.size()) return APAR_ERR_NO_BLOCKS;
   if (rows > INT32_MAX) return APAR_ERR_INVALID_ARG;
-  // bookkeeping and slot list, streamed to the device in staging-sized pieces
+  // bookkeeping and slot list, streamed to the device in staging-sized pieces; calls that fit
+  // leave their slots in the slot map so that the other layers can replay the scatter
+  const bool keep = rows <= kSlotMapRows;
+  c->last_append_rows = keep ? rows : -1;
+  ++c->book_seq;
   const size_t cap_rows = c->lay.stage_cap / 4;
   Staging* stg = nullptr;
   int32_t* slots = nullptr;
@@ -537,7 +570,7 @@ apar_status apar_append_kv(apar_ctx* c, int32_t n, const int32_t* tid, const int
   int64_t first_row = 0;
   auto flush = [&]() -> apar_status {
     if (!filled) return APAR_OK;
-    char* d_stage = c->ws(c->lay.stage);
+    char* d_stage = keep ? c->ws(c->lay.slot_map) + (size_t)first_row * 4 : c->ws(c->lay.stage);
     apar_status rc = send(c, stg, d_stage, filled * 4, st);
     if (rc) return rc;
     APAR_CUDA(c, launch_append(c->cfg.k_pool, c->cfg.v_pool, k_new, v_new,
@@ -599,6 +632,30 @@ apar_status apar_tree_decode_attention(apar_ctx* c, int32_t n, const int32_t* ti
                        (cudaStream_t)cuda_stream);
 }
 
+apar_status apar_append_kv_layer(apar_ctx* c, int32_t layer, const void* k_new, const void* v_new,
+                                 void* cuda_stream) {
+  if (!c || layer < 0 || layer >= c->num_layers || !k_new || !v_new) return APAR_ERR_INVALID_ARG;
+  if (c->last_append_rows < 0) return APAR_ERR_WORKSPACE_TOO_SMALL;
+  if (c->last_append_rows == 0) return APAR_OK;
+  APAR_CUDA(c, launch_append((char*)c->cfg.k_pool + layer * c->layer_bytes,
+                             (char*)c->cfg.v_pool + layer * c->layer_bytes, k_new, v_new,
+                             (const int32_t*)c->ws(c->lay.slot_map), 0, (int)c->last_append_rows,
+                             c->cfg.num_kv_heads, (cudaStream_t)cuda_stream));
+  ++c->kernels_total;
+  return APAR_OK;
+}
+
+apar_status apar_tree_decode_attention_layer(apar_ctx* c, int32_t layer, const void* q, void* out,
+                                             float sm_scale, void* cuda_stream) {
+  if (!c || layer < 0 || layer >= c->num_layers || !q || !out) return APAR_ERR_INVALID_ARG;
+  // the device-resident plan, tables and lengths must still describe the pool
+  if (c->attn_book_seq != c->book_seq || c->plan.items.empty()) return APAR_ERR_INVALID_ARG;
+  int launches = 0;
+  apar_status rc = launch_plan(c, layer, q, out, sm_scale, (cudaStream_t)cuda_stream, &launches);
+  c->kernels_total += launches;
+  return rc;
+}
+
 apar_status apar_release(apar_ctx* c, int32_t n, const int32_t* tid) {
   if (!c || n < 0 || (n > 0 && !tid)) return APAR_ERR_INVALID_ARG;
   const uint32_t mk = next_mark(c);
@@ -619,6 +676,7 @@ apar_status apar_release(apar_ctx* c, int32_t n, const int32_t* tid) {
     --c->live;
   }
   if (n) ++c->struct_epoch;
+  ++c->book_seq;
   return APAR_OK;
 }
 

@@ -21,12 +21,15 @@ def pool_requirements(spec: ForestSpec, slack: float = 0.05):
 
 class PagedSession:
     def __init__(self, shape: LayerShape, num_blocks: int, max_threads: int,
-                 max_blocks_per_thread: int, device="cuda", poison: bool = False):
+                 max_blocks_per_thread: int, device="cuda", poison: bool = False,
+                 num_layers: int = 1):
         if not torch.cuda.is_available():
             raise RuntimeError("the APAR library needs a CUDA device; there is no CPU path")
         self.shape, self.device = shape, torch.device(device)
         self.num_blocks = num_blocks
-        pool_shape = (num_blocks, shape.num_kv_heads, shape.block_size, shape.head_dim)
+        self.num_layers = num_layers
+        pool_shape = (num_layers * num_blocks, shape.num_kv_heads, shape.block_size,
+                      shape.head_dim)
         if poison:   # NaN bit patterns everywhere: any read of an unwritten row shows up
             self.k_pool = torch.full(pool_shape, float("nan"), dtype=torch.bfloat16, device=device)
             self.v_pool = torch.full(pool_shape, float("nan"), dtype=torch.bfloat16, device=device)
@@ -34,7 +37,7 @@ class PagedSession:
             self.k_pool = torch.zeros(pool_shape, dtype=torch.bfloat16, device=device)
             self.v_pool = torch.zeros(pool_shape, dtype=torch.bfloat16, device=device)
         cfg = B.make_config(num_blocks, shape.num_q_heads, shape.num_kv_heads, max_threads,
-                            max_blocks_per_thread)
+                            max_blocks_per_thread, num_layers=num_layers)
         ws_bytes = B.apar_workspace_bytes(cfg)
         self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
         cfg.k_pool, cfg.v_pool = self.k_pool.data_ptr(), self.v_pool.data_ptr()
@@ -85,6 +88,21 @@ class PagedSession:
         B.apar_tree_decode_attention(self.ctx, tids, q.data_ptr(), out.data_ptr(),
                                      self.sm_scale if sm_scale is None else sm_scale,
                                      self._stream())
+        return out
+
+    def append_layer(self, layer: int, k_rows: torch.Tensor, v_rows: torch.Tensor):
+        assert k_rows.is_cuda and k_rows.is_contiguous() and v_rows.is_contiguous()
+        B.apar_append_kv_layer(self.ctx, layer, k_rows.data_ptr(), v_rows.data_ptr(),
+                               self._stream())
+
+    def attention_layer(self, layer: int, q: torch.Tensor, out: torch.Tensor = None,
+                        sm_scale=None):
+        assert q.is_cuda and q.is_contiguous() and q.dtype == torch.bfloat16
+        if out is None:
+            out = torch.empty_like(q)
+        B.apar_tree_decode_attention_layer(self.ctx, layer, q.data_ptr(), out.data_ptr(),
+                                           self.sm_scale if sm_scale is None else sm_scale,
+                                           self._stream())
         return out
 
     def release(self, tids):
