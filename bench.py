@@ -175,10 +175,16 @@ def run_ours(args, cfg_id):
     n_live = len(spec.live_nodes())
     n_step_forks = sum(1 for n in spec.nodes if n.step_fork)
     grow_blocks = (n_live + n_step_forks) * (2 * steps_total // 16 + 2) + 2 * n_step_forks
+    L = max(1, args.layers)
     sess = PagedSession(shape, nb + grow_blocks, nt + n_step_forks, mb + 2 * steps_total // 16 + 2,
-                        device=dev)
+                        device=dev, num_layers=L)
     t_setup = time.perf_counter()
     step0 = synth.build_forest(spec, sess, device=dev)
+    if L > 1:      # give the other layers the same rows as layer 0 (setup, untimed)
+        for pool in (sess.k_pool, sess.v_pool):
+            per = pool.shape[0] // L
+            for l in range(1, L):
+                pool[l * per:(l + 1) * per].copy_(pool[:per])
     torch.cuda.synchronize()
     t_setup = time.perf_counter() - t_setup
 
@@ -210,6 +216,10 @@ def run_ours(args, cfg_id):
         if record:
             e1.record()
             attn_events.append((e0, e1))
+        for l in range(1, L):          # the other layers: scatter + attention launches only
+            B.apar_append_kv_layer(sess.ctx, l, k_new.data_ptr(), v_new.data_ptr(), stream)
+            B.apar_tree_decode_attention_layer(sess.ctx, l, q.data_ptr(), out.data_ptr(),
+                                               sess.sm_scale, stream)
         if kids:
             B.apar_release(sess.ctx, kids)
 
@@ -306,8 +316,8 @@ def run_ours(args, cfg_id):
 
     # ---------------- numbers
     total_T = sharding.reduce_timing(0.0, float(T), dist, dev)[1]
-    value = total_T * args.steps / (total_ms * 1e-3)
-    e2e_value = total_T * e2e_steps / (e2e_ms * 1e-3)
+    value = total_T * L * args.steps / (total_ms * 1e-3)
+    e2e_value = total_T * L * e2e_steps / (e2e_ms * 1e-3)
     bpt = shape.bytes_per_token
     # every persistent thread grows by one token per step: the counters of the last timed step
     # are brought back to their mean over the timed steps
@@ -334,7 +344,9 @@ def run_ours(args, cfg_id):
                 "workload": args.workload, "threads_per_gpu": T, "requests": args.requests or synth.DEFAULT_REQUESTS[cfg_id],
                 "num_q_heads": shape.num_q_heads, "num_kv_heads": shape.num_kv_heads,
                 "head_dim": shape.head_dim, "block_size": shape.block_size,
-                "step": ("fork+" if step0.fork_parents else "") + "append+attention, one layer",
+                "step": ("fork+" if step0.fork_parents else "") + "append+attention, " +
+                        ("one layer" if L == 1 else f"{L} layers (value counts thread-tokens "
+                                                    f"per layer)"),
                 "l2": "inputs larger than L2 (unique KV bytes per step >> 126 MB)"
                       if unique_bytes > 4 * 126e6 else "KV smaller than L2: not flushed",
                 "parallelism": f"{world} independent shard(s), no collective",
@@ -382,6 +394,8 @@ def main():
     ap.add_argument("--requests", type=int, default=None,
                     help="shrink the workload to this many requests (profiling captures)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=1,
+                    help="attention layers per step (layers > 0 replay the plan; default 1)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg_id = parse_workload(args.workload)
