@@ -156,6 +156,18 @@ apar_status apar_tree_decode_attention(apar_ctx* ctx, int32_t n, const int32_t* 
                                        const void* q /*[device]*/, void* out /*[device]*/,
                                        float sm_scale, void* cuda_stream);
 
+/* Tree-masked attention for queries at arbitrary positions (the training / prefill mask of
+ * Section 2.2: a token attends the tokens of its ancestors and, causally, those of its own
+ * node).  Query i sits on the chain of thread tid[i] and sees its first attend_len[i] tokens,
+ * 1 <= attend_len[i] <= len(tid[i]); a thread may be listed many times (all positions of a
+ * prompt, several candidate positions of one thread).  Blocks that several queries see in full
+ * are still read once for all of them.  Same shapes, arithmetic and errors as
+ * apar_tree_decode_attention, plus INVALID_ARG for a length out of range; n <= max_threads. */
+apar_status apar_tree_prefix_attention(apar_ctx* ctx, int32_t n, const int32_t* tid /*[host]*/,
+                                       const int32_t* attend_len /*[host]*/,
+                                       const void* q /*[device]*/, void* out /*[device]*/,
+                                       float sm_scale, void* cuda_stream);
+
 /* The same decode step for the other attention layers of a model (Algorithm 1's Sample runs
  * every layer over the same sequences; the paper states nothing per layer).  Both calls reuse
  * what the most recent apar_append_kv / apar_tree_decode_attention of this context prepared on

@@ -9,6 +9,8 @@ from __future__ import annotations
 import ctypes as C
 import os
 
+import numpy as np
+
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libapar.so")
 if not os.path.exists(_LIB_PATH):
     raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_2401_06761_b200.build`")
@@ -61,6 +63,8 @@ _SIGS = {
                                    C.c_void_p]),
     "apar_tree_decode_attention": (C.c_int32, [_ctx, C.c_int32, _i32p, C.c_void_p, C.c_void_p,
                                                C.c_float, C.c_void_p]),
+    "apar_tree_prefix_attention": (C.c_int32, [_ctx, C.c_int32, _i32p, _i32p, C.c_void_p,
+                                               C.c_void_p, C.c_float, C.c_void_p]),
     "apar_append_kv_layer": (C.c_int32, [_ctx, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "apar_tree_decode_attention_layer": (C.c_int32, [_ctx, C.c_int32, C.c_void_p, C.c_void_p,
                                                      C.c_float, C.c_void_p]),
@@ -89,8 +93,10 @@ EXPORTS = tuple(_SIGS)
 def _arr(xs):
     if isinstance(xs, tuple) and len(xs) == 2 and isinstance(xs[1], int):
         return xs          # already marshalled by int32_array()
-    xs = list(xs)
-    return (C.c_int32 * len(xs))(*xs), len(xs)
+    a = np.ascontiguousarray(np.fromiter(xs, dtype=np.int32) if not isinstance(xs, np.ndarray)
+                             else xs.astype(np.int32, copy=False))
+    buf = (C.c_int32 * max(a.size, 1)).from_buffer_copy(a.tobytes() if a.size else b"\0" * 4)
+    return buf, int(a.size)
 
 
 def _check(status: int):
@@ -142,6 +148,12 @@ def apar_append_kv(ctx, tid, n_tok, k_new: int, v_new: int, stream=0):
 def apar_tree_decode_attention(ctx, tid, q: int, out: int, sm_scale: float, stream=0):
     tids, n = _arr(tid)
     _check(lib.apar_tree_decode_attention(ctx, n, tids, q, out, sm_scale, stream))
+
+
+def apar_tree_prefix_attention(ctx, tid, attend_len, q: int, out: int, sm_scale: float, stream=0):
+    tids, n = _arr(tid)
+    lens, _ = _arr(attend_len)
+    _check(lib.apar_tree_prefix_attention(ctx, n, tids, lens, q, out, sm_scale, stream))
 
 
 def apar_append_kv_layer(ctx, layer: int, k_new: int, v_new: int, stream=0):

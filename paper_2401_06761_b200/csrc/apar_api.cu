@@ -304,14 +304,15 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
 }
 
 // The attention launch sequence for queries given as slots (already validated, len > 0).
+// qlens (optional): tokens query i attends, counted from the root; default the thread's length.
 apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32_t* tids,
                           bool has_dups, const void* q, void* out, float sm_scale,
-                          cudaStream_t st) {
+                          cudaStream_t st, const int32_t* qlens = nullptr) {
   c->last.attn_kernels = 0;
   int64_t attended = 0;
-  for (int i = 0; i < n; ++i) attended += c->slots[qslots[i]].len;
+  for (int i = 0; i < n; ++i) attended += qlens ? qlens[i] : c->slots[qslots[i]].len;
 
-  const bool cacheable = tids != nullptr && !has_dups;
+  const bool cacheable = tids != nullptr && !has_dups && !qlens;
   bool reuse = cacheable && c->plan_epoch == c->struct_epoch && c->plan_age < 64 &&
                (int)c->plan_tids.size() == n &&
                memcmp(c->plan_tids.data(), tids, (size_t)n * 4) == 0 &&
@@ -319,7 +320,8 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
   if (!reuse) {
     c->pq.resize(n);
     for (int i = 0; i < n; ++i)
-      c->pq[i] = PlanQuery{c->row(qslots[i]), qslots[i], c->slots[qslots[i]].len};
+      c->pq[i] = PlanQuery{c->row(qslots[i]), qslots[i],
+                           qlens ? qlens[i] : c->slots[qslots[i]].len};
     // finishing items land in the single-row vector kernel or the warp-stream kernel
     const bool fuse_final = c->use_ws && c->mma_min_rows <= 2;
     if (!c->planner.build(c->pq.data(), n, c->lay.slot_capacity, cacheable, c->mma_min_rows,
@@ -630,6 +632,26 @@ apar_status apar_tree_decode_attention(apar_ctx* c, int32_t n, const int32_t* ti
   }
   return run_attention(c, n, qslots.data(), tid, dups, q, out, sm_scale,
                        (cudaStream_t)cuda_stream);
+}
+
+apar_status apar_tree_prefix_attention(apar_ctx* c, int32_t n, const int32_t* tid,
+                                       const int32_t* attend_len, const void* q, void* out,
+                                       float sm_scale, void* cuda_stream) {
+  if (!c || n < 0 || n > c->cfg.max_threads || (n > 0 && (!tid || !attend_len || !q || !out)))
+    return APAR_ERR_INVALID_ARG;
+  if (n == 0) return APAR_OK;
+  std::vector<int32_t> qslots(n);
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, tid[i]);
+    if (s < 0) return APAR_ERR_BAD_THREAD;
+    qslots[i] = s;
+  }
+  for (int i = 0; i < n; ++i) {
+    if (attend_len[i] == 0) return APAR_ERR_EMPTY_CONTEXT;
+    if (attend_len[i] < 0 || attend_len[i] > c->slots[qslots[i]].len) return APAR_ERR_INVALID_ARG;
+  }
+  return run_attention(c, n, qslots.data(), tid, true, q, out, sm_scale,
+                       (cudaStream_t)cuda_stream, attend_len);
 }
 
 apar_status apar_append_kv_layer(apar_ctx* c, int32_t layer, const void* k_new, const void* v_new,
