@@ -53,7 +53,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+                 "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
             self.proc = None
@@ -169,6 +169,8 @@ def run_ours(args, cfg_id):
 
     # shard = the same workload with a rank-specific seed: independent requests, no exchange
     spec = sharding.shard_spec(cfg_id, rank, n_requests=args.requests)
+    if args.unshared:
+        spec = synth.unshared_spec(spec)
     shape = spec.shape
     steps_total = args.warmup + args.steps
     nb, nt, mb = pool_requirements(spec)
@@ -341,7 +343,8 @@ def run_ours(args, cfg_id):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
             "config": {
-                "workload": args.workload, "threads_per_gpu": T, "requests": args.requests or synth.DEFAULT_REQUESTS[cfg_id],
+                "workload": args.workload + ("-unshared" if args.unshared else ""),
+                "threads_per_gpu": T, "requests": args.requests or synth.DEFAULT_REQUESTS[cfg_id],
                 "num_q_heads": shape.num_q_heads, "num_kv_heads": shape.num_kv_heads,
                 "head_dim": shape.head_dim, "block_size": shape.block_size,
                 "step": ("fork+" if step0.fork_parents else "") + "append+attention, " +
@@ -387,13 +390,16 @@ def run_ours(args, cfg_id):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--requests", type=int, default=None,
                     help="shrink the workload to this many requests (profiling captures)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--unshared", action="store_true",
+                    help="same live threads, but every thread owns a private copy of its whole "
+                         "chain (the copy-the-prefix-on-fork policy); for comparison with the tree")
     ap.add_argument("--layers", type=int, default=1,
                     help="attention layers per step (layers > 0 replay the plan; default 1)")
     args = ap.parse_args()
