@@ -245,6 +245,21 @@ apar_status apar_tree_decode_attention_static(const void* k_pool /*[device]*/,
                                               void* out /*[device]*/, float sm_scale,
                                               void* cuda_stream);
 
+/* Paragraph tree of Algorithm 1 (host only): which slice of which sequence belongs where in the
+ * final text.  apar_paragraph_root makes thread tid (a prompt sequence, already holding its
+ * prompt) the root: its node starts at the thread's current length.  From then on every
+ * apar_fork of a tracked thread s at length L closes s's current node at L, opens the
+ * next-sibling node (s, start L) and the first-child node (child, start L + 1: the child's
+ * first appended row is taken to be the forced child token, which is not part of the text),
+ * as the algorithm does when the last token of s is the fork token.  apar_restore writes the
+ * slices (tid, start, end) in the order root, first child, next sibling; an open node ends at
+ * its thread's current length (or at its length when it was released).  n receives the
+ * number of slices; at most cap triples are written.
+ * Errors: BAD_THREAD (unknown thread / not a root), INVALID_ARG. */
+apar_status apar_paragraph_root(apar_ctx* ctx, int32_t tid);
+apar_status apar_restore(apar_ctx* ctx, int32_t root_tid, int32_t* slices /*[host] 3 x cap*/,
+                         int32_t cap, int32_t* n /*[host]*/);
+
 /* Introspection (host state only; used to compare bookkeeping entry by entry). */
 apar_status apar_get_thread(apar_ctx* ctx, int32_t tid, int32_t* len, int32_t* n_blocks,
                             int32_t* blocks /*[host] cap entries, may be NULL*/, int32_t cap);

@@ -9,6 +9,7 @@ with the CUDA path and never receives values computed by it.
 * `attention`   - fp64 dense softmax attention over a thread's path to the root.
 * `bookkeeping` - integer model of the paged pool: block tables, reference counts,
                   free list, copy-on-fork of the partial last block.
+* `paragraphs`  - Algorithm 1's paragraph tree and Restore on plain token lists.
 
 Parity status: every function here is pinned by tests under tests/ that do not go through
 the function itself (library routine on a reducing special case, an independent
@@ -18,6 +19,7 @@ unpinned".
 from .forest import Forest
 from .attention import softmax_weights, dense_attention, tree_decode_attention
 from .bookkeeping import BlockModel, BookkeepingError
+from .paragraphs import SequenceGroup, FORK, CHILD, EOS
 
 __all__ = ["Forest", "softmax_weights", "dense_attention", "tree_decode_attention",
-           "BlockModel", "BookkeepingError"]
+           "BlockModel", "BookkeepingError", "SequenceGroup", "FORK", "CHILD", "EOS"]

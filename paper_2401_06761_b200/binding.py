@@ -76,6 +76,8 @@ _SIGS = {
                                                       C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                                       C.c_int32, C.c_void_p, C.c_void_p, C.c_float,
                                                       C.c_void_p]),
+    "apar_paragraph_root": (C.c_int32, [_ctx, C.c_int32]),
+    "apar_restore": (C.c_int32, [_ctx, C.c_int32, _i32p, C.c_int32, _i32p]),
     "apar_get_thread": (C.c_int32, [_ctx, C.c_int32, _i32p, _i32p, _i32p, C.c_int32]),
     "apar_get_refcounts": (C.c_int32, [_ctx, _i32p]),
     "apar_get_free_list": (C.c_int32, [_ctx, _i32p, C.c_int32, _i32p]),
@@ -187,6 +189,19 @@ def apar_tree_decode_attention_static(k_pool: int, v_pool: int, num_q_heads: int
     _check(lib.apar_tree_decode_attention_static(k_pool, v_pool, num_q_heads, num_kv_heads,
                                                  n_threads, max_blocks_per_thread, block_tables,
                                                  ctx_lens, max_ctx_len, q, out, sm_scale, stream))
+
+
+def apar_paragraph_root(ctx, tid: int):
+    _check(lib.apar_paragraph_root(ctx, tid))
+
+
+def apar_restore(ctx, root_tid: int):
+    """Slices (tid, start, end) of the response in reading order."""
+    n = C.c_int32()
+    _check(lib.apar_restore(ctx, root_tid, None, 0, C.byref(n)))
+    buf = (C.c_int32 * max(3 * n.value, 1))()
+    _check(lib.apar_restore(ctx, root_tid, buf, n.value, C.byref(n)))
+    return [tuple(buf[3 * i:3 * i + 3]) for i in range(n.value)]
 
 
 def apar_get_thread(ctx, tid: int, cap: int = 0):

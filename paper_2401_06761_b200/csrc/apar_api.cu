@@ -112,6 +112,10 @@ struct apar_ctx {
   uint64_t book_seq = 1, attn_book_seq = 0;   // bookkeeping calls so far / at the last plan
   int64_t last_append_rows = -1;              // rows of the last append kept in the slot map
   int32_t last_cuda = 0;
+  // paragraph tree of Algorithm 1 (host only)
+  struct PNodeRec { int32_t tid, start, end, first_child, next_sibling; };
+  std::vector<PNodeRec> pnodes;
+  std::vector<int32_t> cur_node, root_node;   // by thread id; -1: not tracked / not a root
   bool external_tables = false;        // the table-driven entry point owns no pool state
 
   int32_t* row(int slot) { return tables.data() + (size_t)slot * cfg.max_blocks_per_thread; }
@@ -168,6 +172,8 @@ int32_t new_slot(apar_ctx* c) {
   t = ThreadRec();
   t.tid = c->next_tid++;
   c->tid_slot.push_back(s);
+  c->cur_node.push_back(-1);
+  c->root_node.push_back(-1);
   ++c->live;
   return s;
 }
@@ -520,6 +526,17 @@ apar_status apar_fork(apar_ctx* c, int32_t n, const int32_t* parent_tid, int32_t
     ch.len = L;
     child_tid_out[i] = ch.tid;
     ++c->forks;
+    const int32_t cur = c->cur_node[parent_tid[i]];
+    if (cur >= 0) {   // the parent is tracked: close its node, open sibling and child nodes
+      const int32_t sib = (int32_t)c->pnodes.size();
+      c->pnodes.push_back({parent_tid[i], L, -1, -1, -1});
+      c->pnodes.push_back({ch.tid, L + 1, -1, -1, -1});
+      c->pnodes[cur].end = L;
+      c->pnodes[cur].next_sibling = sib;
+      c->pnodes[cur].first_child = sib + 1;
+      c->cur_node[parent_tid[i]] = sib;
+      c->cur_node[ch.tid] = sib + 1;
+    }
   }
   if (n) ++c->struct_epoch;
   ++c->book_seq;
@@ -692,6 +709,7 @@ apar_status apar_release(apar_ctx* c, int32_t n, const int32_t* tid) {
     const int32_t* tab = c->row(s);
     for (int b = 0; b < t.n_blocks; ++b)
       if (--c->refcnt[tab[b]] == 0) c->free_stack.push_back(tab[b]);
+    if (c->cur_node[tid[i]] >= 0) c->pnodes[c->cur_node[tid[i]]].end = t.len;
     c->tid_slot[tid[i]] = -1;
     t = ThreadRec();
     c->free_slots.push_back(s);
@@ -740,6 +758,43 @@ apar_status apar_tree_decode_attention_tables(const apar_config* cfg, int32_t n,
     rc = APAR_ERR_CUDA;
   apar_destroy(c);
   return rc;
+}
+
+apar_status apar_paragraph_root(apar_ctx* c, int32_t tid) {
+  if (!c) return APAR_ERR_INVALID_ARG;
+  const int s = slot_of(c, tid);
+  if (s < 0) return APAR_ERR_BAD_THREAD;
+  if (c->cur_node[tid] >= 0) return APAR_ERR_INVALID_ARG;   // already part of a tree
+  c->root_node[tid] = c->cur_node[tid] = (int32_t)c->pnodes.size();
+  c->pnodes.push_back({tid, c->slots[s].len, -1, -1, -1});
+  return APAR_OK;
+}
+
+apar_status apar_restore(apar_ctx* c, int32_t root_tid, int32_t* slices, int32_t cap, int32_t* n) {
+  if (!c || !n || cap < 0 || (cap > 0 && !slices)) return APAR_ERR_INVALID_ARG;
+  if (root_tid < 0 || root_tid >= (int32_t)c->root_node.size() || c->root_node[root_tid] < 0)
+    return APAR_ERR_BAD_THREAD;
+  std::vector<int32_t> stack{c->root_node[root_tid]};
+  int32_t count = 0;
+  while (!stack.empty()) {
+    const apar_ctx::PNodeRec& nd = c->pnodes[stack.back()];
+    stack.pop_back();
+    int32_t end = nd.end;
+    if (end < 0) {                       // open: the thread is alive, the node runs to its end
+      const int s = slot_of(c, nd.tid);
+      end = s >= 0 ? c->slots[s].len : nd.start;
+    }
+    if (count < cap) {
+      slices[3 * count] = nd.tid;
+      slices[3 * count + 1] = nd.start;
+      slices[3 * count + 2] = end;
+    }
+    ++count;
+    if (nd.next_sibling >= 0) stack.push_back(nd.next_sibling);   // visited after the child
+    if (nd.first_child >= 0) stack.push_back(nd.first_child);
+  }
+  *n = count;
+  return APAR_OK;
 }
 
 apar_status apar_get_thread(apar_ctx* c, int32_t tid, int32_t* len, int32_t* n_blocks,
