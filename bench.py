@@ -332,6 +332,12 @@ def run_ours(args, cfg_id):
     algo_bytes = unique_bytes + qo_bytes
     peak, peak_kind = measured_peaks()
     achieved = algo_bytes / (attn_ms * 1e-3) / 1e9
+    # DRAM bytes (read + write) of the attention kernels of one call, from the ncu captures
+    # summarised under profiles/ (taken on a 64-request case of the same kernels and scaled by
+    # the requests processed; DRAM traffic is proportional to them).  Only for the full cfg4.
+    traffic = None
+    if cfg_id == 4 and args.requests is None and not args.unshared and L == 1:
+        traffic = ((546.5 + 29.3) + (735.1 + 12.8)) * 1e6 * (512 / 64)
 
     if rank == 0:
         cpu_rate, cpu_threads, cores = (oracle_sample(spec, 12.0)
@@ -360,7 +366,7 @@ def run_ours(args, cfg_id):
             "gpu_launches": launches,
             "roofline": {
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None,
+                "frac": achieved / peak, "traffic": traffic,
                 "peak_kind": f"of {peak_kind} copy bandwidth",
                 "kernel": "apar_tree_decode_attention call (table sync + attention + merge launches)",
                 "algorithmic_bytes": algo_bytes, "attention_ms": attn_ms,

@@ -319,7 +319,9 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
   for (int i = 0; i < n; ++i) attended += qlens ? qlens[i] : c->slots[qslots[i]].len;
 
   const bool cacheable = tids != nullptr && !has_dups && !qlens;
-  bool reuse = cacheable && c->plan_epoch == c->struct_epoch && c->plan_age < 64 &&
+  // a plan is kept while the tree is unchanged; it is rebuilt now and then only because the
+  // longest-first order of its items drifts as tails grow
+  bool reuse = cacheable && c->plan_epoch == c->struct_epoch && c->plan_age < 1024 &&
                (int)c->plan_tids.size() == n &&
                memcmp(c->plan_tids.data(), tids, (size_t)n * 4) == 0 &&
                attended - c->plan_attended < c->plan_attended / 4 + 64;
