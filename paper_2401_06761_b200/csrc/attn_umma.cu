@@ -173,10 +173,6 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(bp + kBarOff + 8 * NBARS + 8);
 
   const WorkItem it = a.d_items[item_begin + blockIdx.x];
-  // an earlier CTA gave up a wait: do not pile up (one reader, so the whole CTA agrees)
-  if (threadIdx.x == 0) *cta_abort = *(volatile int*)a.d_error;
-  __syncthreads();
-  if (*cta_abort) return;
   const int kvh = blockIdx.y;
   const int G = a.shape.group, HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;
   const int tok_end = it.tok_end < 0 ? a.d_lens[it.table_row] : it.tok_end;
@@ -188,8 +184,16 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int R = it.n_users * G;
   const int n_active = (R + 15) >> 4;              // softmax warps that own real rows
+  UserRef* s_users = (UserRef*)(bp + kUserOff);
 
+  // Everything that only needs the item is started before the one CTA-wide barrier of the
+  // prologue, so that these latencies overlap: descriptor prefetch, barrier init, TMEM
+  // allocation, the first block ids (producer), the item's users (softmax warps).
   if (threadIdx.x == 0) {
+    // an earlier CTA gave up a wait: do not pile up (one reader, so the whole CTA agrees)
+    *cta_abort = *(volatile int*)a.d_error;
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_k) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_v) : "memory");
     for (int s = 0; s < kKStages; ++s) {
       bar_init(bar(KFULL0 + s), 1);
       bar_init(bar(KEMPTY0 + s), 1);
@@ -207,23 +211,34 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     bar_init(bar(QFULL), 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  int ids0 = 0, ids1 = 0;                          // block ids 0-31 and 32-63 of the run
   if (warp == 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(s32((const void*)tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  } else if (warp == 4) {
+    ids0 = lane < n_blk ? table[lane] : 0;
+    ids1 = 32 + lane < n_blk ? table[32 + lane] : 0;
+  } else if (threadIdx.x < it.n_users) {
+    s_users[threadIdx.x] = a.d_users[it.user_begin + threadIdx.x];
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  if (*cta_abort) {
+    if (warp == 5)
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem),
+                   "r"(kTmemCols) : "memory");
+    return;
+  }
   const uint32_t tm_o = tmem + 128u;      // S buffer b sits at columns [64 b, 64 b + 64)
 
   if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
     // K and V tiles are two independent sequences; each is issued as soon as its ring slot has
     // been released.  Block ids are fetched 32 at a time (eight tiles), one batch ahead.
-    int kid_cur = lane < n_blk ? table[lane] : 0, vid_cur = kid_cur;
-    int kid_next = 32 + lane < n_blk ? table[32 + lane] : 0, vid_next = kid_next;
+    int kid_cur = ids0, vid_cur = ids0, kid_next = ids1, vid_next = ids1;
     int k_next = 0, v_next = 0;
     uint32_t idle = 0;
     while (k_next < n_tiles || v_next < n_tiles) {
@@ -348,9 +363,6 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   } else {
     // ---------------------------------------------------------------- softmax warps 0-3
     // the item's users once, then the query rows into the A-operand layout (rows past R zero)
-    UserRef* s_users = (UserRef*)(bp + kUserOff);
-    if (threadIdx.x < it.n_users) s_users[threadIdx.x] = a.d_users[it.user_begin + threadIdx.x];
-    asm volatile("bar.sync 1, 128;" ::: "memory");
     {
       // all eight loads of a thread are issued before the first store, so that their
       // latencies overlap

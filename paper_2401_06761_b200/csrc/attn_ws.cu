@@ -114,18 +114,6 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
   const WorkItem it = a.d_items[item_begin + blockIdx.x];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) {
-    *cta_abort = *(volatile int*)a.d_error;   // an earlier CTA gave up a wait: do not pile up
-    for (int i = 0; i < 4 * kSlots; ++i) {
-      wb_init(bars + 8u * i, 1);
-      wb_init(bars + 8u * (4 * kSlots + i), 1);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (threadIdx.x < it.n_users) s_users[threadIdx.x] = a.d_users[it.user_begin + threadIdx.x];
-  __syncthreads();
-  if (*cta_abort) return;
-
   const int G = a.shape.group, HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;
   const int tok_end = it.tok_end < 0 ? a.d_lens[it.table_row] : it.tok_end;
   const int n_tok = tok_end - it.tok_begin;
@@ -136,6 +124,23 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   // this CTA's kv heads: [h_begin, h_begin + n_heads); warp w takes h_begin + w, + w + 4, ...
   const int h_begin = blockIdx.y * heads_per_cta;
   const int n_heads = min(heads_per_cta, HKV - h_begin);
+  // started before the CTA's only barrier so that the latencies overlap: descriptor prefetch
+  // and barrier init (thread 0), the first block id (producer), the item's users
+  if (threadIdx.x == 0) {
+    *cta_abort = *(volatile int*)a.d_error;   // an earlier CTA gave up a wait: do not pile up
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_k) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_v) : "memory");
+    for (int i = 0; i < 4 * kSlots; ++i) {
+      wb_init(bars + 8u * i, 1);
+      wb_init(bars + 8u * (4 * kSlots + i), 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  int bid_first = 0;
+  if (warp == 4) bid_first = n_blk > 0 ? table[0] : 0;
+  else if (threadIdx.x < it.n_users) s_users[threadIdx.x] = a.d_users[it.user_begin + threadIdx.x];
+  __syncthreads();
+  if (*cta_abort) return;
 
   if (warp == 4) {
     // ------------------------------------------------------------------ producer warp
@@ -147,7 +152,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       const int heads_w = max(0, n_heads - w + 3) >> 2;
       const int total = heads_w * n_blk;
       const CUtensorMap* map = (op >> 1) ? &tm_v : &tm_k;
-      int bid_next = total > 0 ? table[0] : 0;
+      int bid_next = bid_first;
       for (int c = 0, hi = 0, b = 0; c < total; ++c) {
         const int bid = bid_next;
         const int b1 = b + 1 == n_blk ? 0 : b + 1;
