@@ -65,7 +65,7 @@ def _make(spec, path, monkeypatch, extra_blocks=0):
     return sess, orc, Both(sess, orc)
 
 
-@pytest.mark.parametrize("path", ["vec", "mma", "umma", "auto"])
+@pytest.mark.parametrize("path", ["vec", "mma", "umma", "ws", "auto"])
 @pytest.mark.parametrize("config,nreq", [(1, 1), (2, 3), (3, 6), (4, 2), (5, 24)])
 def test_config_step_parity(config, nreq, path, monkeypatch):
     spec = synth.forest_spec(config, n_requests=nreq)
