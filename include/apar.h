@@ -268,6 +268,12 @@ apar_status apar_get_refcounts(apar_ctx* ctx, int32_t* refcnt /*[host] [num_bloc
 apar_status apar_get_free_list(apar_ctx* ctx, int32_t* ids /*[host]*/, int32_t cap, int32_t* n);
 apar_status apar_get_stats(apar_ctx* ctx, apar_stats* out /*[host]*/);
 
+/* Debug aid: checks the host tables against each other - every table entry is a valid block,
+ * reference counts equal the number of table entries that name the block, free list and used
+ * blocks partition the pool without repeats, table lengths match thread lengths.
+ * Returns APAR_OK, or APAR_ERR_INVALID_ARG if an invariant is broken (a library bug). */
+apar_status apar_check_invariants(apar_ctx* ctx);
+
 /* cudaError_t value of the most recent failing CUDA call of this context (0 if none). */
 int32_t     apar_last_cuda_error(apar_ctx* ctx);
 const char* apar_status_string(apar_status s);

@@ -82,6 +82,7 @@ _SIGS = {
     "apar_get_refcounts": (C.c_int32, [_ctx, _i32p]),
     "apar_get_free_list": (C.c_int32, [_ctx, _i32p, C.c_int32, _i32p]),
     "apar_get_stats": (C.c_int32, [_ctx, C.POINTER(apar_stats)]),
+    "apar_check_invariants": (C.c_int32, [_ctx]),
     "apar_last_cuda_error": (C.c_int32, [_ctx]),
     "apar_status_string": (C.c_char_p, [C.c_int32]),
 }
@@ -230,6 +231,10 @@ def apar_get_stats(ctx) -> dict:
     s = apar_stats()
     _check(lib.apar_get_stats(ctx, C.byref(s)))
     return s.as_dict()
+
+
+def apar_check_invariants(ctx):
+    _check(lib.apar_check_invariants(ctx))
 
 
 def apar_last_cuda_error(ctx) -> int:

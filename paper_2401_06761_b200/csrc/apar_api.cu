@@ -116,7 +116,6 @@ struct apar_ctx {
   struct PNodeRec { int32_t tid, start, end, first_child, next_sibling; };
   std::vector<PNodeRec> pnodes;
   std::vector<int32_t> cur_node, root_node;   // by thread id; -1: not tracked / not a root
-  bool external_tables = false;        // the table-driven entry point owns no pool state
 
   int32_t* row(int slot) { return tables.data() + (size_t)slot * cfg.max_blocks_per_thread; }
   char* ws(size_t off) { return (char*)cfg.workspace + off; }
@@ -408,7 +407,6 @@ apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
   c->lay = lay;
   c->shape = Shape{cfg->num_q_heads, cfg->num_kv_heads, cfg->num_q_heads / cfg->num_kv_heads,
                    cfg->max_blocks_per_thread};
-  c->external_tables = external;
   c->refcnt.assign(cfg->num_blocks, 0);
   c->free_stack.resize(cfg->num_blocks);
   for (int i = 0; i < cfg->num_blocks; ++i) c->free_stack[i] = cfg->num_blocks - 1 - i;
@@ -842,6 +840,36 @@ apar_status apar_get_stats(apar_ctx* c, apar_stats* out) {
     return APAR_ERR_CUDA;
   }
   out->device_wait_timeouts = flag;
+  return APAR_OK;
+}
+
+apar_status apar_check_invariants(apar_ctx* c) {
+  if (!c) return APAR_ERR_INVALID_ARG;
+  const int32_t nb = c->cfg.num_blocks;
+  std::vector<int32_t> count(nb, 0);
+  int64_t live = 0;
+  for (size_t s = 0; s < c->slots.size(); ++s) {
+    const ThreadRec& t = c->slots[s];
+    if (t.tid < 0) continue;
+    ++live;
+    if (slot_of(c, t.tid) != (int)s) return APAR_ERR_INVALID_ARG;
+    if (t.n_blocks != (t.len + kBlock - 1) / kBlock) return APAR_ERR_INVALID_ARG;
+    if (t.synced > t.n_blocks) return APAR_ERR_INVALID_ARG;
+    for (int b = 0; b < t.n_blocks; ++b) {
+      const int32_t id = c->row((int)s)[b];
+      if (id < 0 || id >= nb) return APAR_ERR_INVALID_ARG;
+      ++count[id];
+    }
+  }
+  if (live != c->live) return APAR_ERR_INVALID_ARG;
+  for (int32_t id : c->free_stack) {
+    if (id < 0 || id >= nb || count[id] != 0) return APAR_ERR_INVALID_ARG;
+    count[id] = -1;                                   // seen in the free list
+  }
+  for (int32_t b = 0; b < nb; ++b) {
+    if (count[b] == -1) { if (c->refcnt[b] != 0) return APAR_ERR_INVALID_ARG; }
+    else if (count[b] == 0 || count[b] != c->refcnt[b]) return APAR_ERR_INVALID_ARG;
+  }
   return APAR_OK;
 }
 

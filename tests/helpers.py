@@ -61,6 +61,7 @@ def assert_close(got_bf16: torch.Tensor, ref: np.ndarray, what=""):
 def assert_same_bookkeeping(sess, model, tids):
     from paper_2401_06761_b200 import binding as B
     assert B.apar_get_stats(sess.ctx)["device_wait_timeouts"] == 0
+    B.apar_check_invariants(sess.ctx)
     for t in tids:
         ln, blocks = B.apar_get_thread(sess.ctx, t)
         assert ln == model.lens[t] and blocks == model.tables[t], f"thread {t}"
