@@ -274,6 +274,17 @@ apar_status apar_get_stats(apar_ctx* ctx, apar_stats* out /*[host]*/);
  * Returns APAR_OK, or APAR_ERR_INVALID_ARG if an invariant is broken (a library bug). */
 apar_status apar_check_invariants(apar_ctx* ctx);
 
+/* Measurement aid (the paper has no counterpart): enqueues one kernel that reads `bytes` bytes
+ * (rounded down to a multiple of 16) at `src` once, with the 16-byte streaming loads the
+ * attention kernels use, and xors them into the 8-byte word at `sink`.  Timing it over a buffer
+ * much larger than the L2 cache gives the read-only HBM rate, the ceiling for attention, which
+ * reads far more than it writes.
+ *   src   [device] 16-byte aligned, caller-owned, not modified
+ *   sink  [device] 8-byte aligned word, caller-owned; its old value is xor-ed into, not cleared
+ * Returns APAR_ERR_INVALID_ARG for NULL or misaligned pointers, APAR_ERR_CUDA if the launch
+ * failed (no context, so the CUDA error is read with cudaGetLastError by the caller). */
+apar_status apar_stream_read(const void* src, size_t bytes, void* sink, void* cuda_stream);
+
 /* cudaError_t value of the most recent failing CUDA call of this context (0 if none). */
 int32_t     apar_last_cuda_error(apar_ctx* ctx);
 const char* apar_status_string(apar_status s);

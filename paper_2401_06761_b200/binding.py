@@ -83,6 +83,7 @@ _SIGS = {
     "apar_get_free_list": (C.c_int32, [_ctx, _i32p, C.c_int32, _i32p]),
     "apar_get_stats": (C.c_int32, [_ctx, C.POINTER(apar_stats)]),
     "apar_check_invariants": (C.c_int32, [_ctx]),
+    "apar_stream_read": (C.c_int32, [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]),
     "apar_last_cuda_error": (C.c_int32, [_ctx]),
     "apar_status_string": (C.c_char_p, [C.c_int32]),
 }
@@ -235,6 +236,10 @@ def apar_get_stats(ctx) -> dict:
 
 def apar_check_invariants(ctx):
     _check(lib.apar_check_invariants(ctx))
+
+
+def apar_stream_read(src: int, nbytes: int, sink: int, stream=0):
+    _check(lib.apar_stream_read(src, nbytes, sink, stream))
 
 
 def apar_last_cuda_error(ctx) -> int:

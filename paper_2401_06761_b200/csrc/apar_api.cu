@@ -873,6 +873,18 @@ apar_status apar_check_invariants(apar_ctx* c) {
   return APAR_OK;
 }
 
+apar_status apar_stream_read(const void* src, size_t bytes, void* sink, void* stream) {
+  if (!src || !sink || (reinterpret_cast<uintptr_t>(src) & 15) ||
+      (reinterpret_cast<uintptr_t>(sink) & 7))
+    return APAR_ERR_INVALID_ARG;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return APAR_ERR_CUDA;
+  return launch_stream_read(src, bytes, sink, sms, (cudaStream_t)stream) == cudaSuccess
+             ? APAR_OK : APAR_ERR_CUDA;
+}
+
 int32_t apar_last_cuda_error(apar_ctx* c) { return c ? c->last_cuda : 0; }
 
 const char* apar_status_string(apar_status s) {

@@ -64,6 +64,9 @@ struct Shape {
 // ---- kernel launchers (kernels.cu); all enqueue on `st` and return cudaGetLastError() ----
 cudaError_t launch_cow_copy(void* k_pool, void* v_pool, const CowCopy* d_copies, int n,
                             int num_kv_heads, cudaStream_t st);
+// Reads `bytes` (rounded down to 16) once and xors them into *sink (8 bytes, device).
+cudaError_t launch_stream_read(const void* src, size_t bytes, void* sink, int num_sms,
+                               cudaStream_t st);
 // slots[r] = block * 16 + offset for new row r.
 cudaError_t launch_append(void* k_pool, void* v_pool, const void* k_new, const void* v_new,
                           const int32_t* d_slots, int64_t first_row, int n_rows,

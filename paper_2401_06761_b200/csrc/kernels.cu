@@ -408,6 +408,39 @@ cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items,
   return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------ read-only streaming probe
+// Reads a buffer once with the same 16-byte streaming loads as the attention kernels and folds
+// what it read into one word, so that the loads cannot be dropped.  Its rate is the ceiling for
+// a kernel that only reads HBM.
+__global__ void __launch_bounds__(256) stream_read_kernel(const uint4* __restrict__ src, size_t n16,
+                                                          unsigned long long* __restrict__ sink) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  uint32_t acc = 0;
+  for (; i + 7 * stride < n16; i += 8 * stride) {
+    uint4 v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v[k] = ld_stream(src + i + k * stride);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc ^= v[k].x ^ v[k].y ^ v[k].z ^ v[k].w;
+  }
+  for (; i < n16; i += stride) {
+    const uint4 v = ld_stream(src + i);
+    acc ^= v.x ^ v.y ^ v.z ^ v.w;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc ^= __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0 && acc != 0) atomicXor(sink, (unsigned long long)acc);
+}
+
+cudaError_t launch_stream_read(const void* src, size_t bytes, void* sink, int num_sms,
+                               cudaStream_t st) {
+  if (bytes < 16) return cudaSuccess;
+  stream_read_kernel<<<num_sms * 8, 256, 0, st>>>((const uint4*)src, bytes / 16,
+                                                  (unsigned long long*)sink);
+  return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ merge of partial results
 // One warp per (query, head): out = sum_j o_j 2^(m_j - M) / sum_j l_j 2^(m_j - M).
 __global__ void __launch_bounds__(128) merge_kernel(const AttnArgs a,
