@@ -335,6 +335,23 @@ def run_ours(args, cfg_id):
     h2d = sum(t[0].numel() * 2 for t in (dq, dk, dv))
     d2h = out.numel() * 2
 
+    # the same copies alone, both directions at once: the PCIe time a step cannot go below
+    def copies_only():
+        with torch.cuda.stream(s_in):
+            dq[0].copy_(hq[0], non_blocking=True)
+            dk[0].copy_(hk[0], non_blocking=True)
+            dv[0].copy_(hv[0], non_blocking=True)
+        with torch.cuda.stream(s_out):
+            hout.copy_(dout[0], non_blocking=True)
+    copies_only()
+    torch.cuda.synchronize()
+    reps = 10
+    t_c = time.perf_counter()
+    for _ in range(reps):
+        copies_only()
+    torch.cuda.synchronize()
+    copy_ms = 1e3 * (time.perf_counter() - t_c) / reps
+
     # ---------------- numbers
     total_T = sharding.reduce_timing(0.0, float(T), dist, dev)[1]
     value = total_T * L * args.steps / (total_ms * 1e-3)
@@ -383,7 +400,12 @@ def run_ours(args, cfg_id):
             },
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                    "ms_per_step": e2e_ms / e2e_steps,
+                    # host<->device copies of one step alone (up and down overlapped): the
+                    # end-to-end step is bound by them whenever they take longer than the compute
+                    "copies_only_ms": copy_ms,
+                    "copies_only_gbs": (h2d + d2h) / (copy_ms * 1e-3) / 1e9},
             "gpu_launches": launches,
             "roofline": {
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",

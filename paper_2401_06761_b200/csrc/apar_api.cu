@@ -68,6 +68,7 @@ struct ThreadRec {
 
 struct Staging {
   char* host = nullptr;
+  char* mapped = nullptr;   // the same buffer as the device sees it
   cudaEvent_t done = nullptr;
   bool in_flight = false;
 };
@@ -145,7 +146,16 @@ apar_status acquire(apar_ctx* c, Staging** out) {
 }
 
 apar_status send(apar_ctx* c, Staging* s, void* dst, size_t bytes, cudaStream_t st) {
-  if (bytes) APAR_CUDA(c, cudaMemcpyAsync(dst, s->host, bytes, cudaMemcpyHostToDevice, st));
+  // By a kernel, not a copy engine: these uploads gate the step's kernels and must not wait
+  // behind an application's large host-to-device copy on another stream.
+  if (bytes % 4 == 0 && s->mapped) {
+    if (bytes) {
+      APAR_CUDA(c, launch_stage_copy(dst, s->mapped, bytes, st));
+      ++c->kernels_total;
+    }
+  } else if (bytes) {
+    APAR_CUDA(c, cudaMemcpyAsync(dst, s->host, bytes, cudaMemcpyHostToDevice, st));
+  }
   APAR_CUDA(c, cudaEventRecord(s->done, st));
   s->in_flight = true;
   return APAR_OK;
@@ -439,7 +449,9 @@ apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
     return APAR_ERR_CUDA;
   }
   for (int i = 0; i < kRing; ++i) {
-    cudaError_t e = cudaMallocHost((void**)&c->ring[i].host, c->ring_bytes);
+    cudaError_t e = cudaHostAlloc((void**)&c->ring[i].host, c->ring_bytes, cudaHostAllocMapped);
+    if (e == cudaSuccess)
+      e = cudaHostGetDevicePointer((void**)&c->ring[i].mapped, c->ring[i].host, 0);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ring[i].done, cudaEventDisableTiming);
     if (e != cudaSuccess) {
       apar_destroy(c);

@@ -64,6 +64,9 @@ struct Shape {
 // ---- kernel launchers (kernels.cu); all enqueue on `st` and return cudaGetLastError() ----
 cudaError_t launch_cow_copy(void* k_pool, void* v_pool, const CowCopy* d_copies, int n,
                             int num_kv_heads, cudaStream_t st);
+// dst[0..bytes) = src_mapped[0..bytes) read by the SMs; src_mapped is the device alias of a
+// pinned, mapped host buffer; bytes is a multiple of 4.
+cudaError_t launch_stage_copy(void* dst, const void* src_mapped, size_t bytes, cudaStream_t st);
 // Reads `bytes` (rounded down to 16) once and xors them into *sink (8 bytes, device).
 cudaError_t launch_stream_read(const void* src, size_t bytes, void* sink, int num_sms,
                                cudaStream_t st);

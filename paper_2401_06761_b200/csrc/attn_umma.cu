@@ -2,11 +2,13 @@
 // a run of blocks shared by up to 64 (query, head) rows.
 //
 // One CTA owns one (work item, kv head).  Roles:
-//   warps 0-3  softmax: thread i < 16 of warp w owns query row 16w + i, which is TMEM lane
-//              32w + i of an M = 64 accumulator.  They read S from TMEM, keep the running
-//              reference maximum and the row sum, write P = exp2(S - ref) as bf16 into shared
-//              memory in the K-major 128-byte-swizzled operand layout, rescale O in TMEM in the
-//              rare case the reference has to move, and write the results at the end.
+//   warps 0-3  softmax: warp w owns query rows 16w .. 16w+15, which are TMEM lanes 32w .. 32w+15
+//              of an M = 64 accumulator.  S is read with the 16-lane x 256-bit TMEM load, which
+//              spreads a row over the four threads of a quad, so that all 32 lanes work; they
+//              keep the running reference maximum and the row sum, write P = exp2(S - ref) as
+//              bf16 into shared memory in the K-major 128-byte-swizzled operand layout, rescale
+//              O in TMEM in the rare case the reference has to move, and write the results at
+//              the end (O rows are read back one row per thread, lanes 0-15).
 //   warp 4     producer: walks the block table, TMA tensor copies of 16-token K/V tiles into
 //              two rings of 64-token stages - K (two deep, released as soon as Q K^T has
 //              read it) and V (three deep, released after P V) - same tile layout as the
@@ -127,6 +129,18 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
                  "=r"(r[o + 22]), "=r"(r[o + 23]), "=r"(r[o + 24]), "=r"(r[o + 25]),             \
                  "=r"(r[o + 26]), "=r"(r[o + 27]), "=r"(r[o + 28]), "=r"(r[o + 29]),             \
                  "=r"(r[o + 30]), "=r"(r[o + 31])                                                \
+               : "r"(taddr))
+
+#define TMEM_LD_16x256(taddr, r)                                                                 \
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x8.b32 "                                         \
+               "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"                          \
+               "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"         \
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]),         \
+                 "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]),       \
+                 "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]),   \
+                 "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),   \
+                 "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]),   \
+                 "=r"(r[30]), "=r"(r[31])                                                        \
                : "r"(taddr))
 
 #define TMEM_ST_32(taddr, r)                                                                     \
@@ -389,40 +403,64 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const int row = warp * 16 + (lane & 15);
     const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
     const float c = a.scale_log2e;
-    float ref = -INFINITY, l = 0.f;
+    // S is read with the 16-lane x 256-bit TMEM load, which deals a 16 x 64 tile over all 32
+    // threads like an MMA accumulator fragment: thread 4g + qd holds, for k = 0..7, columns
+    // 8k + 2qd and 8k + 2qd + 1 of row g (registers 4k, 4k + 1) and of row g + 8 (registers
+    // 4k + 2, 4k + 3).  A row is thus shared by the four threads of a quad: the maximum is
+    // reduced over the quad for every tile, the row sum only once at the end.
+    const int g8 = lane >> 2, qd = lane & 3;
+    float ref_lo = -INFINITY, ref_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+    float ref = -INFINITY, l = 0.f;        // of the row this thread writes out (lanes 0-15)
     bool alive = true;
     if (active) {
       for (int t = 0; t < n_tiles; ++t) {
         const int b = t & 1;
         if (!bar_wait(bar(SFULL0 + b), (t >> 1) & 1, cta_abort, a.d_error, 2000 + t)) { alive = false; break; }
         tc_fence_after();
-        uint32_t sr[64];
-        TMEM_LD_32((tmem + 64u * b) | lane_sel, sr, 0);
-        TMEM_LD_32((tmem + 64u * b + 32u) | lane_sel, sr, 32);
+        uint32_t sr[32];
+        TMEM_LD_16x256(( tmem + 64u * b) | lane_sel, sr);
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) bar_arrive(bar(SFREE0 + b));
         const int tile_tok = min(kTileTok, n_tok - t * kTileTok);
-        float mx = -INFINITY;
+        float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < 64; ++j) {
-          const float x = j < tile_tok ? __uint_as_float(sr[j]) * c : -INFINITY;
-          sr[j] = __float_as_uint(x);
-          mx = fmaxf(mx, x);
+        for (int k = 0; k < 8; ++k) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const bool in = 8 * k + 2 * qd + e < tile_tok;
+            const float x_lo = in ? __uint_as_float(sr[4 * k + e]) * c : -INFINITY;
+            const float x_hi = in ? __uint_as_float(sr[4 * k + 2 + e]) * c : -INFINITY;
+            sr[4 * k + e] = __float_as_uint(x_lo);
+            sr[4 * k + 2 + e] = __float_as_uint(x_hi);
+            mx_lo = fmaxf(mx_lo, x_lo);
+            mx_hi = fmaxf(mx_hi, x_hi);
+          }
         }
-        const bool move = mx > ref + kRefSlack || ref == -INFINITY;
-        const float new_ref = move ? mx : ref;
-        const bool rescale = t > 0 && __any_sync(0xffffffffu, move && lane < 16);
+        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+        const bool move_lo = mx_lo > ref_lo + kRefSlack || ref_lo == -INFINITY;
+        const bool move_hi = mx_hi > ref_hi + kRefSlack || ref_hi == -INFINITY;
+        const float new_lo = move_lo ? mx_lo : ref_lo, new_hi = move_hi ? mx_hi : ref_hi;
+        const bool rescale = t > 0 && __any_sync(0xffffffffu, move_lo || move_hi);
         if (rescale) {
-          // rare: the reference moves, so O (which P V(t-1) still accumulates into) is rescaled
+          // rare: a reference moves, so O (which P V(t-1) still accumulates into) is rescaled,
+          // by the thread that owns the whole row in the 32-lane layout (lanes 0-15)
           if (!bar_wait(bar(PFREE), (t - 1) & 1, cta_abort, a.d_error, 3000 + t)) {
             alive = false;
             break;
           }
           tc_fence_after();
-          const float f = move ? ex2(ref - new_ref) : 1.f;
-          l *= f;
+          const float f_lo = move_lo ? ex2(ref_lo - new_lo) : 1.f;
+          const float f_hi = move_hi ? ex2(ref_hi - new_hi) : 1.f;
+          l_lo *= f_lo;
+          l_hi *= f_hi;
+          const float fa = __shfl_sync(0xffffffffu, f_lo, 4 * (lane & 7));
+          const float fb = __shfl_sync(0xffffffffu, f_hi, 4 * (lane & 7));
+          const float f = (lane & 8) ? fb : fa;
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
             uint32_t orow[32];
@@ -435,28 +473,35 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           tmem_wait_st();
           tc_fence_before();
         }
-        ref = new_ref;
-        float ps = 0.f;
-        uint32_t pk[32];
+        ref_lo = new_lo;
+        ref_hi = new_hi;
+        uint32_t pk_lo[8], pk_hi[8];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float p0 = ex2(__uint_as_float(sr[2 * j]) - ref);
-          const float p1 = ex2(__uint_as_float(sr[2 * j + 1]) - ref);
-          ps += p0 + p1;
-          pk[j] = pack2(p0, p1);
+        for (int k = 0; k < 8; ++k) {
+          const float a0 = ex2(__uint_as_float(sr[4 * k]) - ref_lo);
+          const float a1 = ex2(__uint_as_float(sr[4 * k + 1]) - ref_lo);
+          const float b0 = ex2(__uint_as_float(sr[4 * k + 2]) - ref_hi);
+          const float b1 = ex2(__uint_as_float(sr[4 * k + 3]) - ref_hi);
+          l_lo += a0 + a1;
+          l_hi += b0 + b1;
+          pk_lo[k] = pack2(a0, a1);
+          pk_hi[k] = pack2(b0, b1);
         }
-        l += ps;
         // P(t) overwrites the buffer that P V(t-1) reads
         if (t > 0 && !rescale && !bar_wait(bar(PFREE), (t - 1) & 1, cta_abort, a.d_error, 3000 + t)) {
           alive = false;
           break;
         }
-        if (lane < 16) {
-          uint8_t* prow = bp + kPOff + row * 128;
+        {
+          // rows 16w + g and 16w + g + 8 have the same (row & 7), hence the same swizzle
+          const int r_lo = warp * 16 + g8;
+          uint8_t* p_lo = bp + kPOff + r_lo * 128 + 4 * qd;
 #pragma unroll
-          for (int ch = 0; ch < 8; ++ch)
-            *(uint4*)(prow + ((ch ^ (row & 7)) << 4)) =
-                make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+          for (int k = 0; k < 8; ++k) {
+            const int off = (k ^ (r_lo & 7)) << 4;
+            *(uint32_t*)(p_lo + off) = pk_lo[k];
+            *(uint32_t*)(p_lo + 8 * 128 + off) = pk_hi[k];
+          }
         }
         // rows of V past the valid length hold unspecified bits: zero them before P V
         if (tile_tok < kTileTok && warp == 0) {
@@ -477,6 +522,17 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       if (alive && n_tiles > 0)
         alive = bar_wait(bar(PFREE), (n_tiles - 1) & 1, cta_abort, a.d_error, 5000);
       tc_fence_after();
+      // row sums over the quad, then to the lane that writes the row out
+      l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+      l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+      l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+      l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+      const float la = __shfl_sync(0xffffffffu, l_lo, 4 * (lane & 7));
+      const float lb = __shfl_sync(0xffffffffu, l_hi, 4 * (lane & 7));
+      const float ra = __shfl_sync(0xffffffffu, ref_lo, 4 * (lane & 7));
+      const float rb = __shfl_sync(0xffffffffu, ref_hi, 4 * (lane & 7));
+      l = (lane & 8) ? lb : la;
+      ref = (lane & 8) ? rb : ra;
     }
     // ---- O rows out of TMEM: the thread that owns a row writes it, 32 columns at a time
     if (active && alive) {

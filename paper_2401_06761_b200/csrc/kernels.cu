@@ -1,6 +1,8 @@
 // CUDA kernels of the APAR decode hot path for sm_100a: copy-on-fork of a partial block,
 // KV append scatter, device-table sync, the vectorised CUDA-core attention path for
 // work items with few query rows (private tails under MHA), and the cross-item merge.
+#include <algorithm>
+
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -405,6 +407,27 @@ cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items,
   } else {
     attn_vec_kernel<4><<<dim3(n_items, a.shape.num_kv_heads), 128, 0, st>>>(a, item_begin);
   }
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ staging upload
+// Moves a staged host buffer (pinned, mapped) into device memory with SM loads over PCIe
+// instead of a copy engine.  The library's uploads are small (slot lists, table deltas, plan
+// pieces) but sit on the critical path of a step; on a copy engine they queue behind whatever
+// large host-to-device copy the application has in flight on another stream.
+__global__ void __launch_bounds__(256) stage_copy_kernel(uint32_t* __restrict__ dst,
+                                                         const uint32_t* __restrict__ src_mapped,
+                                                         size_t n_words) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += stride)
+    dst[i] = src_mapped[i];
+}
+
+cudaError_t launch_stage_copy(void* dst, const void* src_mapped, size_t bytes, cudaStream_t st) {
+  const size_t n = bytes / 4;
+  if (n == 0) return cudaSuccess;
+  const int blocks = (int)std::min<size_t>((n + 255) / 256, 1024);
+  stage_copy_kernel<<<blocks, 256, 0, st>>>((uint32_t*)dst, (const uint32_t*)src_mapped, n);
   return cudaGetLastError();
 }
 
