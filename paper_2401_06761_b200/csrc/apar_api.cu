@@ -15,7 +15,9 @@ using namespace apar;
 
 namespace {
 
-constexpr int kRing = 4;              // pinned staging buffers in flight
+constexpr int kRing = 12;             // pinned staging buffers in flight: enough for the uploads of
+                                      // two whole steps, so that the host can prepare a step
+                                      // while the GPU still runs the one before
 constexpr int kSlotsPerThread = 6;    // partial-result rows provisioned per live thread
 constexpr int kSlotMapRows = 262144;  // new-row slots of the last append kept for other layers
 
@@ -236,14 +238,19 @@ apar_status sync_device_tables(apar_ctx* c, const int32_t* slots, int n, cudaStr
       if (i < n) return APAR_ERR_WORKSPACE_TOO_SMALL;   // one row larger than the staging area
       break;
     }
-    const size_t bytes = ((char*)(data + used)) - s->host;
+    // close the gaps between the three arrays, so that only what was filled crosses PCIe
+    const size_t off_pairs = (size_t)nd * sizeof(TableDelta);
+    const size_t off_data = off_pairs + (size_t)np * 8;
+    memmove(s->host + off_pairs, pairs, (size_t)np * 8);
+    memmove(s->host + off_data, data, used * 4);
+    const size_t bytes = off_data + used * 4;
     char* d_stage = c->ws(c->lay.stage);
     rc = send(c, s, d_stage, bytes, st);
     if (rc) return rc;
     APAR_CUDA(c, launch_sync((int32_t*)c->ws(c->lay.tables), c->cfg.max_blocks_per_thread,
                              (int32_t*)c->ws(c->lay.lens), (const TableDelta*)d_stage,
-                             (const int32_t*)(d_stage + ((char*)data - s->host)), nd,
-                             (const int32_t*)(d_stage + ((char*)pairs - s->host)), np, st));
+                             (const int32_t*)(d_stage + off_data), nd,
+                             (const int32_t*)(d_stage + off_pairs), np, st));
     ++c->kernels_total;
     ++c->last.attn_kernels;
   }
