@@ -144,7 +144,9 @@ def run_reference(args, cfg_id):
     if rank != 0:
         return
     spec = synth.forest_spec(cfg_id)
-    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    # about a minute of timed oracle work over the whole run (input generation, untimed, takes
+    # about as long again)
+    per_step = max(0.5, min(20.0, 60.0 / max(1, args.steps + args.warmup)))
     for _ in range(args.warmup):
         oracle_sample(spec, per_step / 4)
     rates, threads = [], 0
@@ -197,22 +199,35 @@ def run_ours(args, cfg_id):
     n_step_forks = sum(1 for n in spec.nodes if n.step_fork)
     grow_blocks = (n_live + n_step_forks) * (2 * steps_total // 16 + 2) + 2 * n_step_forks
     L = max(1, args.layers)
-    sess = PagedSession(shape, nb + grow_blocks, nt + n_step_forks, mb + 2 * steps_total // 16 + 2,
-                        device=dev, num_layers=L)
-    t_setup = time.perf_counter()
-    step0 = synth.build_forest(spec, sess, device=dev)
-    if L > 1:      # give the other layers the same rows as layer 0 (setup, untimed)
-        for pool in (sess.k_pool, sess.v_pool):
-            per = pool.shape[0] // L
-            for l in range(1, L):
-                pool[l * per:(l + 1) * per].copy_(pool[:per])
-    torch.cuda.synchronize()
-    t_setup = time.perf_counter() - t_setup
-
     from paper_2401_06761_b200 import binding as B
+
+    class S:      # the session in use: the end-to-end arm rebuilds it, see below
+        sess = step0 = base_live = base_live_arr = None
+        setup_s = 0.0
+
+    def make_session():
+        if S.sess is not None:
+            S.sess.close()
+            S.sess = S.step0 = None
+            torch.cuda.empty_cache()
+        t0 = time.perf_counter()
+        S.sess = PagedSession(shape, nb + grow_blocks, nt + n_step_forks,
+                              mb + 2 * steps_total // 16 + 2, device=dev, num_layers=L)
+        S.step0 = synth.build_forest(spec, S.sess, device=dev)
+        if L > 1:      # give the other layers the same rows as layer 0 (setup, untimed)
+            for pool in (S.sess.k_pool, S.sess.v_pool):
+                per = pool.shape[0] // L
+                for l in range(1, L):
+                    pool[l * per:(l + 1) * per].copy_(pool[:per])
+        torch.cuda.synchronize()
+        S.setup_s = time.perf_counter() - t0
+        S.base_live = [h for h, n in zip(S.step0.live_handles, S.step0.live_nodes)
+                       if not n.step_fork]
+        S.base_live_arr = B.int32_array(S.base_live)
+
+    make_session()
+    t_setup = S.setup_s
     stream = torch.cuda.current_stream().cuda_stream
-    base_live = [h for h, n in zip(step0.live_handles, step0.live_nodes) if not n.step_fork]
-    base_live_arr = B.int32_array(base_live)
     T = n_live
     g = torch.Generator(device=dev).manual_seed(spec.seed + 99)
     row_shape = (T, shape.num_kv_heads, shape.head_dim)
@@ -226,8 +241,9 @@ def run_ours(args, cfg_id):
 
     def one_step(q, k_new, v_new, record, stream=stream, out=out):
         """fork (if the workload has one) + append + attention [+ release of the step's forks]."""
+        sess, step0 = S.sess, S.step0
         kids = B.apar_fork(sess.ctx, step0.fork_parents, stream) if step0.fork_parents else []
-        live = B.int32_array(base_live + kids) if kids else base_live_arr
+        live = B.int32_array(S.base_live + kids) if kids else S.base_live_arr
         B.apar_append_kv(sess.ctx, live, None, k_new.data_ptr(), v_new.data_ptr(), stream)
         if record:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -258,7 +274,7 @@ def run_ours(args, cfg_id):
     for i in range(args.warmup):
         one_step(*inputs[i % len(inputs)], record=False)
     barrier()
-    k0 = sess.stats()["kernels_total"]
+    k0 = S.sess.stats()["kernels_total"]
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -272,9 +288,10 @@ def run_ours(args, cfg_id):
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     total_ms = max_over_ranks(ev0.elapsed_time(ev1))
-    launches = sess.stats()["kernels_total"] - k0
+    launches = S.sess.stats()["kernels_total"] - k0
     attn_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_events)
-    st = sess.stats()
+    st = S.sess.stats()
+    n_base_live, has_fork = len(S.base_live), bool(S.step0.fork_parents)
     if st["device_wait_timeouts"]:
         raise SystemExit(f"a kernel gave up a bounded wait (code {st['device_wait_timeouts']}): "
                          "the timed results are invalid")
@@ -320,8 +337,13 @@ def run_ours(args, cfg_id):
             hout.copy_(dout[b], non_blocking=True)
             ev_out[b].record(s_out)
 
-    e2e_steps = max(1, min(args.steps, steps_total - 1))
-    e2e_step(0)
+    # The end-to-end arm starts from the same forest as the device arm did (every step makes
+    # each thread one token longer, so carrying on would time a larger problem): rebuild it,
+    # then the same number of warm-up steps, untimed.
+    make_session()
+    e2e_steps = args.steps
+    for i in range(args.warmup):
+        e2e_step(i)
     barrier()
     ev0.record()
     for i in range(e2e_steps):
@@ -359,7 +381,7 @@ def run_ours(args, cfg_id):
     bpt = shape.bytes_per_token
     # every persistent thread grows by one token per step: the counters of the last timed step
     # are brought back to their mean over the timed steps
-    grow = len(base_live) * (args.steps - 1) / 2.0
+    grow = n_base_live * (args.steps - 1) / 2.0
     unique_tokens = st["attn_unique_tokens"] - grow
     attended_tokens = st["attn_attended_tokens"] - grow
     unique_bytes = unique_tokens * bpt
@@ -391,7 +413,7 @@ def run_ours(args, cfg_id):
                 "threads_per_gpu": T, "requests": args.requests or synth.DEFAULT_REQUESTS[cfg_id],
                 "num_q_heads": shape.num_q_heads, "num_kv_heads": shape.num_kv_heads,
                 "head_dim": shape.head_dim, "block_size": shape.block_size,
-                "step": ("fork+" if step0.fork_parents else "") + "append+attention, " +
+                "step": ("fork+" if has_fork else "") + "append+attention, " +
                         ("one layer" if L == 1 else f"{L} layers (value counts thread-tokens "
                                                     f"per layer)"),
                 "l2": "inputs larger than L2 (unique KV bytes per step >> 126 MB)"
@@ -437,7 +459,7 @@ def run_ours(args, cfg_id):
                 "sample": f"{cpu_threads} live threads of {args.workload}, one at a time "
                           f"(fp64 chain materialisation + dense attention, all query heads)"}
         print(json.dumps(line))
-    sess.close()
+    S.sess.close()
     if dist is not None:
         dist.destroy_process_group()
 
