@@ -18,6 +18,8 @@
 //              signals completion with tcgen05.commit on mbarriers.  Owns the TMEM allocation.
 // All waits are bounded; a wait that gives up raises an error word and every role unwinds to
 // the common exit where TMEM is released.
+#include <cstdlib>
+
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -40,11 +42,12 @@ constexpr int kUserOff = kBarOff + 256;             // the item's UserRef entrie
 constexpr int kSmem = kUserOff + 64 * 8 + 1024;
 constexpr uint32_t kSpin = 1u << 20;
 constexpr int kTmemCols = 256;                     // S0 | S1 | O
+constexpr int kWavesMin = 6, kHeadsMax = 2;        // see launch_attention_umma
 constexpr float kRefSlack = 8.f;                   // P stays below 2^8 before the reference moves
 
 enum Bar { KFULL0 = 0, KEMPTY0 = KFULL0 + kKStages, VFULL0 = KEMPTY0 + kKStages,
            VEMPTY0 = VFULL0 + kVStages, SFULL0 = VEMPTY0 + kVStages, SFREE0 = SFULL0 + 2,
-           PFULL = SFREE0 + 2, PFREE, QFULL, NBARS };
+           PFULL = SFREE0 + 2, PFREE, QFULL, ODONE, NBARS };
 
 __device__ __forceinline__ uint32_t s32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -175,9 +178,16 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *(uint32_t*)&v;
 }
 
+// One CTA owns one work item and `heads_per_cta` consecutive kv heads of it, which it works
+// through one after the other.  All of them share the item's block table, token range and
+// users; only the Q rows and the output rows differ.  The mbarrier phases run on across the
+// heads (tile g = head ordinal x tiles per head + tile), so that the producer and the MMA
+// thread run ahead into the next head while the softmax warps write out the current one: the
+// start-up and write-out latencies, which dominate short items, are hidden for all heads of
+// a CTA but the first and the last.
 __global__ void __launch_bounds__(192, 2)
 attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                 const AttnArgs a, int item_begin) {
+                 const AttnArgs a, int item_begin, int heads_per_cta) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (s32(smem_raw) + 1023u) & ~1023u;
   uint8_t* bp = smem_raw + (base - s32(smem_raw));
@@ -187,12 +197,13 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(bp + kBarOff + 8 * NBARS + 8);
 
   const WorkItem it = a.d_items[item_begin + blockIdx.x];
-  const int kvh = blockIdx.y;
+  const int U = heads_per_cta, kvh0 = blockIdx.y * U;
   const int G = a.shape.group, HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;
   const int tok_end = it.tok_end < 0 ? a.d_lens[it.table_row] : it.tok_end;
   const int n_tok = tok_end - it.tok_begin;
   const int n_blk = (n_tok + kBlock - 1) / kBlock;
   const int n_tiles = (n_tok + kTileTok - 1) / kTileTok;
+  const int total = U * n_tiles;                   // tiles of the whole CTA
   const int32_t* table = a.d_tables + (size_t)it.table_row * a.shape.table_stride +
                          it.tok_begin / kBlock;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -222,7 +233,8 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     }
     bar_init(bar(PFULL), n_active);
     bar_init(bar(PFREE), 1);
-    bar_init(bar(QFULL), 4);
+    bar_init(bar(QFULL), n_active);
+    bar_init(bar(ODONE), n_active);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   int ids0 = 0, ids1 = 0;                          // block ids 0-31 and 32-63 of the run
@@ -233,8 +245,17 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   } else if (warp == 4) {
     ids0 = lane < n_blk ? table[lane] : 0;
     ids1 = 32 + lane < n_blk ? table[32 + lane] : 0;
-  } else if (threadIdx.x < it.n_users) {
-    s_users[threadIdx.x] = a.d_users[it.user_begin + threadIdx.x];
+  } else {
+    if (threadIdx.x < it.n_users) s_users[threadIdx.x] = a.d_users[it.user_begin + threadIdx.x];
+    // Q rows of warps without real rows stay zero for the whole CTA
+    if (warp >= n_active) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int i = lane + 32 * k;
+        *(uint4*)(bp + kQOff + swz_off(warp * 16 + (i >> 4), i & 15)) = make_uint4(0u, 0u, 0u, 0u);
+      }
+      fence_async_smem();
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -250,19 +271,24 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 
   if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
-    // K and V tiles are two independent sequences; each is issued as soon as its ring slot has
-    // been released.  Block ids are fetched 32 at a time (eight tiles), one batch ahead.
+    // K and V tiles are two independent sequences over all heads of the CTA; each tile is
+    // issued as soon as its ring slot has been released.  Block ids are fetched 32 at a time
+    // (eight tiles), one batch ahead; every head walks the same ids again.
     int kid_cur = ids0, vid_cur = ids0, kid_next = ids1, vid_next = ids1;
-    int k_next = 0, v_next = 0;
+    int k_next = 0, v_next = 0;             // tiles issued, all heads
+    int kt = 0, kh = 0, vt = 0, vh = 0;     // the same as (tile within the head, head ordinal)
     uint32_t idle = 0;
-    while (k_next < n_tiles || v_next < n_tiles) {
+    while (k_next < total || v_next < total) {
       bool did = false;
-      if (k_next < n_tiles) {
-        const int t = k_next, s = t % kKStages;
-        int ready = t < kKStages || bar_try(bar(KEMPTY0 + s), ((t / kKStages) - 1) & 1);
+      if (k_next < total) {
+        const int g = k_next, t = kt, s = g % kKStages;
+        int ready = g < kKStages || bar_try(bar(KEMPTY0 + s), ((g / kKStages) - 1) & 1);
         ready = __shfl_sync(0xffffffffu, ready, 0);
         if (ready) {
-          if (t > 0 && (t & 7) == 0) {
+          if (t == 0 && kh > 0) {
+            kid_cur = ids0;
+            kid_next = ids1;
+          } else if (t > 0 && (t & 7) == 0) {
             kid_cur = kid_next;
             const int nxt = (t + 8) * kTileBlocks + lane;
             kid_next = nxt < n_blk ? table[nxt] : 0;
@@ -275,17 +301,21 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           __syncwarp();
           if (lane < 2 * kTileBlocks && blk < n_blk)
             tma_2d(base + s * kKV + (lane & 1) * kHalf + (lane >> 1) * (kBlock * 128), &tm_k,
-                   (lane & 1) * 64, (bid * HKV + kvh) * kBlock, bar(KFULL0 + s));
+                   (lane & 1) * 64, (bid * HKV + kvh0 + kh) * kBlock, bar(KFULL0 + s));
           ++k_next;
+          if (++kt == n_tiles) { kt = 0; ++kh; }
           did = true;
         }
       }
-      if (v_next < n_tiles) {
-        const int t = v_next, s = t % kVStages;
-        int ready = t < kVStages || bar_try(bar(VEMPTY0 + s), ((t / kVStages) - 1) & 1);
+      if (v_next < total) {
+        const int g = v_next, t = vt, s = g % kVStages;
+        int ready = g < kVStages || bar_try(bar(VEMPTY0 + s), ((g / kVStages) - 1) & 1);
         ready = __shfl_sync(0xffffffffu, ready, 0);
         if (ready) {
-          if (t > 0 && (t & 7) == 0) {
+          if (t == 0 && vh > 0) {
+            vid_cur = ids0;
+            vid_next = ids1;
+          } else if (t > 0 && (t & 7) == 0) {
             vid_cur = vid_next;
             const int nxt = (t + 8) * kTileBlocks + lane;
             vid_next = nxt < n_blk ? table[nxt] : 0;
@@ -298,8 +328,9 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           __syncwarp();
           if (lane < 2 * kTileBlocks && blk < n_blk)
             tma_2d(base + kVOff + s * kKV + (lane & 1) * kHalf + (lane >> 1) * (kBlock * 128),
-                   &tm_v, (lane & 1) * 64, (bid * HKV + kvh) * kBlock, bar(VFULL0 + s));
+                   &tm_v, (lane & 1) * 64, (bid * HKV + kvh0 + vh) * kBlock, bar(VFULL0 + s));
           ++v_next;
+          if (++vt == n_tiles) { vt = 0; ++vh; }
           did = true;
         }
       }
@@ -309,7 +340,10 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         ++idle;
         int stop = idle > kSpin || ((idle & 255) == 0 && *cta_abort);
         if (__shfl_sync(0xffffffffu, stop, 0)) {
-          if (lane == 0 && idle > kSpin) { *cta_abort = 1; atomicCAS(a.d_error, 0, 6000 + k_next * 40 + v_next % 40); }
+          if (lane == 0 && idle > kSpin) {
+            *cta_abort = 1;
+            atomicCAS(a.d_error, 0, 6000 + (k_next % 25) * 40 + v_next % 40);
+          }
           break;
         }
       }
@@ -319,18 +353,21 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     constexpr uint32_t kIdescQK = instr_desc(kTileTok, false);
     constexpr uint32_t kIdescPV = instr_desc(kDim, true);
     // One thread issues everything.  It polls for whichever step can go next - Q K^T of the
-    // next tile as soon as its K has landed and an S buffer is free, P V of the oldest pending
-    // tile as soon as the softmax warps have published P - so that neither waits for the other.
-    if (lane == 0 && bar_wait(bar(QFULL), 0, cta_abort, a.d_error, 1000)) {
-      tc_fence_after();
-      int qk_next = 0, pv_next = 0;
+    // next tile as soon as its K has landed, an S buffer is free and (first tile of a head) the
+    // head's Q is staged; P V of the oldest pending tile as soon as the softmax warps have
+    // published P and (first tile of a head) drained the previous head's O - so that neither
+    // waits for the other.
+    if (lane == 0) {
+      int qk_next = 0, pv_next = 0;         // tiles issued, all heads
+      int qt = 0, qh = 0, pt = 0, ph = 0;   // the same as (tile within the head, head ordinal)
       uint32_t idle = 0;
-      while (pv_next < n_tiles) {
+      while (pv_next < total) {
         bool did = false;
-        if (qk_next < n_tiles) {
-          const int t = qk_next, s = t % kKStages, b = t & 1;
-          if (bar_try(bar(KFULL0 + s), (t / kKStages) & 1) &&
-              (t < 2 || bar_try(bar(SFREE0 + b), ((t >> 1) - 1) & 1))) {
+        if (qk_next < total) {
+          const int g = qk_next, s = g % kKStages, b = g & 1;
+          if (bar_try(bar(KFULL0 + s), (g / kKStages) & 1) &&
+              (g < 2 || bar_try(bar(SFREE0 + b), ((g >> 1) - 1) & 1)) &&
+              (qt > 0 || bar_try(bar(QFULL), qh & 1))) {
             tc_fence_after();
             const uint32_t kb = base + s * kKV, qb = base + kQOff;
 #pragma unroll
@@ -342,48 +379,52 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             umma_commit(bar(SFULL0 + b));
             umma_commit(bar(KEMPTY0 + s));
             ++qk_next;
+            if (++qt == n_tiles) { qt = 0; ++qh; }
             did = true;
           }
         }
         if (pv_next < qk_next) {
-          const int t = pv_next, s = t % kVStages;
-          if (bar_try(bar(PFULL), t & 1) && bar_try(bar(VFULL0 + s), (t / kVStages) & 1)) {
+          const int g = pv_next, s = g % kVStages;
+          if (bar_try(bar(PFULL), g & 1) && bar_try(bar(VFULL0 + s), (g / kVStages) & 1) &&
+              (pt > 0 || ph == 0 || bar_try(bar(ODONE), (ph - 1) & 1))) {
             tc_fence_after();
             const uint32_t vb = base + kVOff + s * kKV, pb = base + kPOff;
             // blocks past the end of the item were never loaded: leave their k-steps out
-            const int nk = min(kTileBlocks, (n_tok - t * kTileTok + kBlock - 1) / kBlock);
+            const int nk = min(kTileBlocks, (n_tok - pt * kTileTok + kBlock - 1) / kBlock);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
               if (kk < nk)
                 umma_bf16(tm_o, smem_desc(pb + kk * 32, 16, 1024),
                           smem_desc(vb + kk * (kBlock * 128), kHalf, 1024), kIdescPV,
-                          (t | kk) != 0);
+                          (pt | kk) != 0);
             umma_commit(bar(PFREE));
             umma_commit(bar(VEMPTY0 + s));
             ++pv_next;
+            if (++pt == n_tiles) { pt = 0; ++ph; }
             did = true;
           }
         }
         if (did) {
           idle = 0;
         } else if (++idle > kSpin || ((idle & 255) == 0 && *cta_abort)) {
-          if (idle > kSpin) atomicCAS(a.d_error, 0, 7000 + qk_next * 40 + pv_next % 40);
+          if (idle > kSpin) atomicCAS(a.d_error, 0, 7000 + (qk_next % 25) * 40 + pv_next % 40);
           *cta_abort = 1;
           break;
         }
       }
     }
     __syncwarp();
-  } else {
+  } else if (warp < n_active) {
     // ---------------------------------------------------------------- softmax warps 0-3
-    // the item's users once, then the query rows into the A-operand layout (rows past R zero)
-    {
+    // Warp w owns query rows 16w .. 16w+15 of every head: it stages them into the A-operand
+    // layout (rows past R as zeros), runs their softmax and writes their results.
+    auto stage_q = [&](int kvh) {
       // all eight loads of a thread are issued before the first store, so that their
       // latencies overlap
       uint4 qv[8];
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
-        const int i = threadIdx.x + 128 * k, row = i >> 4, c = i & 15;
+        const int i = lane + 32 * k, row = warp * 16 + (i >> 4), c = i & 15;
         qv[k] = make_uint4(0u, 0u, 0u, 0u);
         if (row < R)
           qv[k] = __ldg((const uint4*)a.q +
@@ -391,15 +432,15 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       }
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
-        const int i = threadIdx.x + 128 * k;
-        *(uint4*)(bp + kQOff + swz_off(i >> 4, i & 15)) = qv[k];
+        const int i = lane + 32 * k;
+        *(uint4*)(bp + kQOff + swz_off(warp * 16 + (i >> 4), i & 15)) = qv[k];
       }
-    }
-    fence_async_smem();
-    __syncwarp();
-    if (lane == 0) bar_arrive(bar(QFULL));
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) bar_arrive(bar(QFULL));
+    };
+    stage_q(kvh0);
 
-    const bool active = warp < n_active;
     const int row = warp * 16 + (lane & 15);
     const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
     const float c = a.scale_log2e;
@@ -409,16 +450,20 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     // 4k + 2, 4k + 3).  A row is thus shared by the four threads of a quad: the maximum is
     // reduced over the quad for every tile, the row sum only once at the end.
     const int g8 = lane >> 2, qd = lane & 3;
-    float ref_lo = -INFINITY, ref_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
-    float ref = -INFINITY, l = 0.f;        // of the row this thread writes out (lanes 0-15)
     bool alive = true;
-    if (active) {
+    for (int h = 0; h < U && alive; ++h) {
+      const int kvh = kvh0 + h;
+      const int g0 = h * n_tiles;            // tiles of earlier heads
+      float ref_lo = -INFINITY, ref_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
       for (int t = 0; t < n_tiles; ++t) {
-        const int b = t & 1;
-        if (!bar_wait(bar(SFULL0 + b), (t >> 1) & 1, cta_abort, a.d_error, 2000 + t)) { alive = false; break; }
+        const int g = g0 + t, b = g & 1;
+        if (!bar_wait(bar(SFULL0 + b), (g >> 1) & 1, cta_abort, a.d_error, 2000 + t % 1000)) {
+          alive = false;
+          break;
+        }
         tc_fence_after();
         uint32_t sr[32];
-        TMEM_LD_16x256(( tmem + 64u * b) | lane_sel, sr);
+        TMEM_LD_16x256((tmem + 64u * b) | lane_sel, sr);
         tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
@@ -449,7 +494,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         if (rescale) {
           // rare: a reference moves, so O (which P V(t-1) still accumulates into) is rescaled,
           // by the thread that owns the whole row in the 32-lane layout (lanes 0-15)
-          if (!bar_wait(bar(PFREE), (t - 1) & 1, cta_abort, a.d_error, 3000 + t)) {
+          if (!bar_wait(bar(PFREE), (g - 1) & 1, cta_abort, a.d_error, 3000 + t % 1000)) {
             alive = false;
             break;
           }
@@ -487,8 +532,9 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           pk_lo[k] = pack2(a0, a1);
           pk_hi[k] = pack2(b0, b1);
         }
-        // P(t) overwrites the buffer that P V(t-1) reads
-        if (t > 0 && !rescale && !bar_wait(bar(PFREE), (t - 1) & 1, cta_abort, a.d_error, 3000 + t)) {
+        // P(g) overwrites the buffer that the previous P V reads
+        if (g > 0 && !rescale &&
+            !bar_wait(bar(PFREE), (g - 1) & 1, cta_abort, a.d_error, 3000 + t % 1000)) {
           alive = false;
           break;
         }
@@ -505,8 +551,9 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
         // rows of V past the valid length hold unspecified bits: zero them before P V
         if (tile_tok < kTileTok && warp == 0) {
-          const int vs = t % kVStages;
-          if (!bar_wait(bar(VFULL0 + vs), (t / kVStages) & 1, cta_abort, a.d_error, 4000 + t)) {
+          const int vs = g % kVStages;
+          if (!bar_wait(bar(VFULL0 + vs), (g / kVStages) & 1, cta_abort, a.d_error,
+                        4000 + t % 1000)) {
             alive = false;
             break;
           }
@@ -519,8 +566,11 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         __syncwarp();
         if (lane == 0) bar_arrive(bar(PFULL));
       }
-      if (alive && n_tiles > 0)
-        alive = bar_wait(bar(PFREE), (n_tiles - 1) & 1, cta_abort, a.d_error, 5000);
+      if (!alive) break;
+      // every Q K^T of this head has completed (this warp has seen its last S tile): the next
+      // head's rows can take the Q buffer while the last P V is still running
+      if (h + 1 < U) stage_q(kvh + 1);
+      if (!bar_wait(bar(PFREE), (g0 + n_tiles - 1) & 1, cta_abort, a.d_error, 5000)) break;
       tc_fence_after();
       // row sums over the quad, then to the lane that writes the row out
       l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
@@ -531,43 +581,46 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       const float lb = __shfl_sync(0xffffffffu, l_hi, 4 * (lane & 7));
       const float ra = __shfl_sync(0xffffffffu, ref_lo, 4 * (lane & 7));
       const float rb = __shfl_sync(0xffffffffu, ref_hi, 4 * (lane & 7));
-      l = (lane & 8) ? lb : la;
-      ref = (lane & 8) ? rb : ra;
-    }
-    // ---- O rows out of TMEM: the thread that owns a row writes it, 32 columns at a time
-    if (active && alive) {
-      const bool mine = lane < 16 && row < R;
-      UserRef ur = UserRef{0, -1};
-      if (mine) ur = s_users[row / G];
-      const int head = kvh * G + row % G;
-      const float inv = 1.f / l;
-      uint4* dst_out = (uint4*)((__nv_bfloat16*)a.out + ((size_t)ur.query * HQ + head) * kDim);
-      const size_t prow = (size_t)(ur.slot + it.slot_add) * HQ + head;
-      float4* dst_part = (float4*)(a.part_o + prow * kDim);
+      const float l = (lane & 8) ? lb : la, ref = (lane & 8) ? rb : ra;
+      // ---- O rows out of TMEM: the thread that owns a row writes it, 32 columns at a time
+      {
+        const bool mine = lane < 16 && row < R;
+        UserRef ur = UserRef{0, -1};
+        if (mine) ur = s_users[row / G];
+        const int head = kvh * G + row % G;
+        const float inv = 1.f / l;
+        uint4* dst_out = (uint4*)((__nv_bfloat16*)a.out + ((size_t)ur.query * HQ + head) * kDim);
+        const size_t prow = (size_t)(ur.slot + it.slot_add) * HQ + head;
+        float4* dst_part = (float4*)(a.part_o + prow * kDim);
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        uint32_t orow[32];
-        TMEM_LD_32((tm_o + 32u * q4) | lane_sel, orow, 0);
-        tmem_wait_ld();
-        if (mine) {
-          if (ur.slot < 0) {
+        for (int q4 = 0; q4 < 4; ++q4) {
+          uint32_t orow[32];
+          TMEM_LD_32((tm_o + 32u * q4) | lane_sel, orow, 0);
+          tmem_wait_ld();
+          if (mine) {
+            if (ur.slot < 0) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 8)
-              dst_out[4 * q4 + (j >> 3)] = make_uint4(
-                  pack2(__uint_as_float(orow[j]) * inv, __uint_as_float(orow[j + 1]) * inv),
-                  pack2(__uint_as_float(orow[j + 2]) * inv, __uint_as_float(orow[j + 3]) * inv),
-                  pack2(__uint_as_float(orow[j + 4]) * inv, __uint_as_float(orow[j + 5]) * inv),
-                  pack2(__uint_as_float(orow[j + 6]) * inv, __uint_as_float(orow[j + 7]) * inv));
-          } else {
+              for (int j = 0; j < 32; j += 8)
+                dst_out[4 * q4 + (j >> 3)] = make_uint4(
+                    pack2(__uint_as_float(orow[j]) * inv, __uint_as_float(orow[j + 1]) * inv),
+                    pack2(__uint_as_float(orow[j + 2]) * inv, __uint_as_float(orow[j + 3]) * inv),
+                    pack2(__uint_as_float(orow[j + 4]) * inv, __uint_as_float(orow[j + 5]) * inv),
+                    pack2(__uint_as_float(orow[j + 6]) * inv, __uint_as_float(orow[j + 7]) * inv));
+            } else {
 #pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              dst_part[8 * q4 + (j >> 2)] =
-                  make_float4(__uint_as_float(orow[j]), __uint_as_float(orow[j + 1]),
-                              __uint_as_float(orow[j + 2]), __uint_as_float(orow[j + 3]));
+              for (int j = 0; j < 32; j += 4)
+                dst_part[8 * q4 + (j >> 2)] =
+                    make_float4(__uint_as_float(orow[j]), __uint_as_float(orow[j + 1]),
+                                __uint_as_float(orow[j + 2]), __uint_as_float(orow[j + 3]));
+            }
           }
         }
+        if (mine && ur.slot >= 0) a.part_ml[prow] = make_float2(ref, l);
       }
-      if (mine && ur.slot >= 0) a.part_ml[prow] = make_float2(ref, l);
+      // O has been read: the next head's first P V may overwrite it
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) bar_arrive(bar(ODONE));
     }
   }
   // ---- common exit: every role arrives here, then the allocating warp frees TMEM
@@ -586,16 +639,31 @@ cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items
                                   cudaStream_t st) {
   if (n_items <= 0) return cudaSuccess;
   static bool configured[64] = {};
+  static int sm_count[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
-  if (dev >= 0 && dev < 64 && !configured[dev]) {
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(attn_umma_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  attn_umma_kernel<<<dim3(n_items, a.shape.num_kv_heads), 192, kSmem, st>>>(*a.tm_k, *a.tm_v, a,
-                                                                            item_begin);
+  // Heads per CTA: up to kHeadsMax, if that leaves at least kWavesMin CTAs for each of the
+  // machine's CTA slots (two per SM), so that the hardware scheduler can still even out the
+  // load.  Measured: two heads per CTA take 2-3 % off the kernel, four or eight cost more in
+  // uneven last waves than the hidden start-up saves (the kernel is bound by HBM, not by the
+  // latencies that running on into the next head hides).
+  const int hkv = a.shape.num_kv_heads;
+  const char* force = getenv("APAR_UMMA_HEADS");      // testing
+  int u = 1;
+  for (int c = 2; c <= kHeadsMax && c <= hkv; c *= 2)
+    if (hkv % c == 0 && (long long)n_items * (hkv / c) >= (long long)kWavesMin * 2 * sm_count[dev])
+      u = c;
+  if (force && atoi(force) >= 1 && hkv % atoi(force) == 0) u = atoi(force);
+  attn_umma_kernel<<<dim3(n_items, hkv / u), 192, kSmem, st>>>(*a.tm_k, *a.tm_v, a, item_begin, u);
   return cudaGetLastError();
 }
 

@@ -324,3 +324,47 @@ def test_scores_that_keep_growing_move_the_softmax_reference(hq, hkv, kids, path
     assert np.isfinite(err).all() and err.max() <= 2e-2, (path, err.max())
     assert err.mean() <= 1e-3 + 2.0 ** -9 * np.abs(ref).mean(), (path, err.mean())
     sess.close()
+
+
+@pytest.mark.parametrize("heads", ["1", "2", "4", "8"])
+def test_tcgen05_kernel_with_several_kv_heads_per_cta(heads, monkeypatch):
+    """The tensor-core kernel lets a CTA walk several kv heads of its item, the barrier phases
+    running on from head to head; forced here to every group size, on items with one ragged
+    tile, with many tiles, and with scores that make the softmax reference move in each head."""
+    monkeypatch.setenv("APAR_UMMA_HEADS", heads)
+    for config, nreq in [(4, 2), (5, 24)]:
+        spec = synth.forest_spec(config, n_requests=nreq)
+        sess, orc, both = _make(spec, "umma", monkeypatch)
+        step = synth.build_forest(spec, both, device="cuda")
+        live = step.live_handles
+        both.append(live, None, step.k_new, step.v_new)
+        out = sess.attention(live, step.q)
+        assert_close(out, orc.attention(live, step.q, sess.sm_scale), f"cfg{config} heads {heads}")
+        assert sess.stats()["device_wait_timeouts"] == 0
+        sess.close()
+    # wide fork over 8 kv heads, prompt of 37 tokens (a single ragged tile) and of 700
+    shape = synth.LayerShape(16, 8)
+    for prompt in (37, 700):
+        sess = _session(shape, 400, 16, 64, poison=True)
+        orc = OracleBackend(shape, 400, 16, 64)
+        both = Both(sess, orc)
+        g = torch.Generator(device="cuda").manual_seed(prompt)
+        (p,) = both.new_threads(1)
+        ramp = torch.arange(prompt, device="cuda", dtype=torch.float32)[:, None, None] * 0.3
+        k = (ramp * torch.ones((1, 8, 128), device="cuda") / 11.3 +
+             torch.randn((prompt, 8, 128), generator=g, device="cuda")).to(torch.bfloat16)
+        v = torch.randn((prompt, 8, 128), generator=g, device="cuda").to(torch.bfloat16)
+        both.append([p], [prompt], k, v)
+        kids = both.fork([p] * 12)
+        both.append(kids, None,
+                    torch.randn((12, 8, 128), generator=g, device="cuda").to(torch.bfloat16),
+                    torch.randn((12, 8, 128), generator=g, device="cuda").to(torch.bfloat16))
+        q = (torch.ones((12, 16, 128), device="cuda") +
+             0.3 * torch.randn((12, 16, 128), generator=g, device="cuda")).to(torch.bfloat16)
+        out = sess.attention(kids, q, sm_scale=1.0)
+        ref = orc.attention(kids, q, 1.0)
+        err = np.abs(out.cpu().to(torch.float64).numpy() - ref)
+        assert np.isfinite(err).all() and err.max() <= 2e-2, (heads, prompt, err.max())
+        assert err.mean() <= 1e-3 + 2.0 ** -9 * np.abs(ref).mean(), (heads, prompt, err.mean())
+        assert sess.stats()["device_wait_timeouts"] == 0
+        sess.close()
