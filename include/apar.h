@@ -274,6 +274,31 @@ apar_status apar_get_stats(apar_ctx* ctx, apar_stats* out /*[host]*/);
  * Returns APAR_OK, or APAR_ERR_INVALID_ARG if an invariant is broken (a library bug). */
 apar_status apar_check_invariants(apar_ctx* ctx);
 
+/* Debug aid, host only (makes no CUDA call, needs no GPU): plans one attention call over
+ * explicit block tables exactly as apar_tree_decode_attention_tables would and returns the
+ * plan, so that the planner can be checked without a device.  The planner is the library's
+ * own part of the path (the paper reads shared blocks once per thread; Section 2.3 only says
+ * which blocks are shared).
+ *   block_tables [host] [n_threads][max_blocks] block ids, ctx_lens [host] [n_threads] > 0
+ *   mma_min_rows: items with at least this many query rows are classed for the tensor-core
+ *                 kernels; fuse_final != 0: the last item of a chain that ends in a private
+ *                 run finishes its query (folds the other partial results)
+ *   items_out [host] [cap_items][8] int32: table_row, tok_begin, tok_end, user_begin, n_users,
+ *             slot_add, fin_n, fin_begin (the fields of a work item; table_row = index of the
+ *             thread whose table the item walks)
+ *   users_out [host] [cap_users][2] int32: query (thread index), partial slot or -1
+ *   merges_out [host] [cap_merges][3] int32: query, first partial slot, number of slots
+ *   counts_out [host] [6] int64: items, users, merges, partial slots, unique tokens,
+ *              attended tokens
+ * Returns APAR_ERR_WORKSPACE_TOO_SMALL if a cap is too small (counts_out is still filled),
+ * APAR_ERR_INVALID_ARG for bad shapes, lengths or block ids. */
+apar_status apar_debug_plan(int32_t num_blocks, int32_t num_q_heads, int32_t num_kv_heads,
+                            int32_t n_threads, int32_t max_blocks, const int32_t* block_tables,
+                            const int32_t* ctx_lens, int32_t mma_min_rows, int32_t fuse_final,
+                            int32_t* items_out, int32_t cap_items, int32_t* users_out,
+                            int32_t cap_users, int32_t* merges_out, int32_t cap_merges,
+                            int64_t* counts_out);
+
 /* Measurement aid (the paper has no counterpart): enqueues one kernel that reads `bytes` bytes
  * (rounded down to a multiple of 16) at `src` once, with the 16-byte streaming loads the
  * attention kernels use, and xors them into the 8-byte word at `sink`.  Timing it over a buffer

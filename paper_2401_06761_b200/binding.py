@@ -83,6 +83,9 @@ _SIGS = {
     "apar_get_free_list": (C.c_int32, [_ctx, _i32p, C.c_int32, _i32p]),
     "apar_get_stats": (C.c_int32, [_ctx, C.POINTER(apar_stats)]),
     "apar_check_invariants": (C.c_int32, [_ctx]),
+    "apar_debug_plan": (C.c_int32, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _i32p,
+                                    _i32p, C.c_int32, C.c_int32, _i32p, C.c_int32, _i32p,
+                                    C.c_int32, _i32p, C.c_int32, C.POINTER(C.c_int64)]),
     "apar_stream_read": (C.c_int32, [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]),
     "apar_last_cuda_error": (C.c_int32, [_ctx]),
     "apar_status_string": (C.c_char_p, [C.c_int32]),
@@ -236,6 +239,28 @@ def apar_get_stats(ctx) -> dict:
 
 def apar_check_invariants(ctx):
     _check(lib.apar_check_invariants(ctx))
+
+
+def apar_debug_plan(num_blocks, num_q_heads, num_kv_heads, tables, lens, mma_min_rows=2,
+                    fuse_final=True):
+    """Host-only planning of one attention call; `tables` is an [n][max_blocks] int32 array.
+    Returns (items [k][8], users [m][2], merges [j][3], counts dict) as numpy arrays."""
+    tables = np.ascontiguousarray(tables, dtype=np.int32)
+    lens = np.ascontiguousarray(lens, dtype=np.int32)
+    n, mb = tables.shape
+    cap_users = int(sum((int(l) + 15) // 16 for l in lens)) + 1
+    cap_items = 4 * cap_users + 16
+    items = np.zeros((cap_items, 8), dtype=np.int32)
+    users = np.zeros((cap_users, 2), dtype=np.int32)
+    merges = np.zeros((n + 1, 3), dtype=np.int32)
+    counts = (C.c_int64 * 6)()
+    p = lambda a: a.ctypes.data_as(_i32p)
+    _check(lib.apar_debug_plan(num_blocks, num_q_heads, num_kv_heads, n, mb, p(tables), p(lens),
+                               mma_min_rows, int(bool(fuse_final)), p(items), cap_items,
+                               p(users), cap_users, p(merges), n + 1, counts))
+    names = ("items", "users", "merges", "partial_slots", "unique_tokens", "attended_tokens")
+    c = dict(zip(names, (int(x) for x in counts)))
+    return items[:c["items"]], users[:c["users"]], merges[:c["merges"]], c
 
 
 def apar_stream_read(src: int, nbytes: int, sink: int, stream=0):

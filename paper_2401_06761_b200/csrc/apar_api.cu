@@ -892,6 +892,52 @@ apar_status apar_check_invariants(apar_ctx* c) {
   return APAR_OK;
 }
 
+apar_status apar_debug_plan(int32_t num_blocks, int32_t num_q_heads, int32_t num_kv_heads,
+                            int32_t n_threads, int32_t max_blocks, const int32_t* block_tables,
+                            const int32_t* ctx_lens, int32_t mma_min_rows, int32_t fuse_final,
+                            int32_t* items_out, int32_t cap_items, int32_t* users_out,
+                            int32_t cap_users, int32_t* merges_out, int32_t cap_merges,
+                            int64_t* counts_out) {
+  if (num_blocks <= 0 || num_kv_heads <= 0 || num_q_heads <= 0 || num_q_heads % num_kv_heads ||
+      n_threads <= 0 || max_blocks <= 0 || !block_tables || !ctx_lens || !counts_out ||
+      cap_items < 0 || cap_users < 0 || cap_merges < 0 || (cap_items && !items_out) ||
+      (cap_users && !users_out) || (cap_merges && !merges_out))
+    return APAR_ERR_INVALID_ARG;
+  std::vector<PlanQuery> pq(n_threads);
+  for (int i = 0; i < n_threads; ++i) {
+    const int32_t len = ctx_lens[i];
+    if (len <= 0 || (len + kBlock - 1) / kBlock > max_blocks) return APAR_ERR_INVALID_ARG;
+    const int32_t* tab = block_tables + (size_t)i * max_blocks;
+    for (int b = 0; b < (len + kBlock - 1) / kBlock; ++b)
+      if (tab[b] < 0 || tab[b] >= num_blocks) return APAR_ERR_INVALID_ARG;
+    pq[i] = PlanQuery{tab, i, len};
+  }
+  Planner planner;
+  planner.init(num_blocks, num_q_heads / num_kv_heads, num_kv_heads);
+  Plan plan;
+  if (!planner.build(pq.data(), n_threads, (int64_t)kSlotsPerThread * n_threads, false,
+                     mma_min_rows, fuse_final != 0, &plan))
+    return APAR_ERR_WORKSPACE_TOO_SMALL;
+  counts_out[0] = (int64_t)plan.items.size();
+  counts_out[1] = (int64_t)plan.users.size();
+  counts_out[2] = (int64_t)plan.merges.size();
+  counts_out[3] = plan.total_slots;
+  counts_out[4] = plan.unique_tokens;
+  counts_out[5] = plan.attended_tokens;
+  if ((int64_t)cap_items < counts_out[0] || (int64_t)cap_users < counts_out[1] ||
+      (int64_t)cap_merges < counts_out[2])
+    return APAR_ERR_WORKSPACE_TOO_SMALL;
+  static_assert(sizeof(WorkItem) == 32 && sizeof(UserRef) == 8, "export layout");
+  if (!plan.items.empty()) memcpy(items_out, plan.items.data(), plan.items.size() * sizeof(WorkItem));
+  if (!plan.users.empty()) memcpy(users_out, plan.users.data(), plan.users.size() * sizeof(UserRef));
+  for (size_t i = 0; i < plan.merges.size(); ++i) {
+    merges_out[3 * i] = plan.merges[i].query;
+    merges_out[3 * i + 1] = plan.merges[i].slot_begin;
+    merges_out[3 * i + 2] = plan.merges[i].n;
+  }
+  return APAR_OK;
+}
+
 apar_status apar_stream_read(const void* src, size_t bytes, void* sink, void* stream) {
   if (!src || !sink || (reinterpret_cast<uintptr_t>(src) & 15) ||
       (reinterpret_cast<uintptr_t>(sink) & 7))
