@@ -280,14 +280,32 @@ def run_ours(args, cfg_id):
         sampler.start()
     host_t0 = time.perf_counter()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for i in range(args.steps):
-        one_step(*inputs[i % len(inputs)], record=True)
-    ev1.record()
-    host_issue_ms = 1e3 * (time.perf_counter() - host_t0)
-    barrier()
+    # A workload whose KV fits in the L2 cache would be timed on cache hits: for those, every
+    # step is timed on its own and a buffer larger than L2 is written between the steps.
+    small = spec.unique_tokens() * shape.bytes_per_token < 4 * 126e6
+    if small:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        step_events = []
+        for i in range(args.steps):
+            flush.fill_(i & 0xff)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            one_step(*inputs[i % len(inputs)], record=True)
+            b.record()
+            step_events.append((a, b))
+        host_issue_ms = 1e3 * (time.perf_counter() - host_t0)
+        barrier()
+        total_ms = max_over_ranks(sum(a.elapsed_time(b) for a, b in step_events))
+        del flush
+    else:
+        ev0.record()
+        for i in range(args.steps):
+            one_step(*inputs[i % len(inputs)], record=True)
+        ev1.record()
+        host_issue_ms = 1e3 * (time.perf_counter() - host_t0)
+        barrier()
+        total_ms = max_over_ranks(ev0.elapsed_time(ev1))
     clocks = sampler.stop() if rank == 0 else None
-    total_ms = max_over_ranks(ev0.elapsed_time(ev1))
     launches = S.sess.stats()["kernels_total"] - k0
     attn_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_events)
     st = S.sess.stats()
@@ -417,7 +435,8 @@ def run_ours(args, cfg_id):
                         ("one layer" if L == 1 else f"{L} layers (value counts thread-tokens "
                                                     f"per layer)"),
                 "l2": "inputs larger than L2 (unique KV bytes per step >> 126 MB)"
-                      if unique_bytes > 4 * 126e6 else "KV smaller than L2: not flushed",
+                      if not small else "KV fits in L2: 256 MB written between steps, each step "
+                                        "timed on its own (device arm)",
                 "parallelism": f"{world} independent shard(s), no collective",
             },
             "clocks": clocks,
