@@ -243,14 +243,22 @@ apar_status sync_device_tables(apar_ctx* c, const int32_t* slots, int n, cudaStr
     const size_t off_data = off_pairs + (size_t)np * 8;
     memmove(s->host + off_pairs, pairs, (size_t)np * 8);
     memmove(s->host + off_data, data, used * 4);
-    const size_t bytes = off_data + used * 4;
-    char* d_stage = c->ws(c->lay.stage);
-    rc = send(c, s, d_stage, bytes, st);
-    if (rc) return rc;
+    // Every entry is read exactly once, so the kernel takes them straight from the pinned
+    // buffer (mapped into the device's address space) instead of from a device copy.
+    const char* src = s->mapped;
+    if (!src) {
+      src = c->ws(c->lay.stage);
+      rc = send(c, s, c->ws(c->lay.stage), off_data + used * 4, st);
+      if (rc) return rc;
+    }
     APAR_CUDA(c, launch_sync((int32_t*)c->ws(c->lay.tables), c->cfg.max_blocks_per_thread,
-                             (int32_t*)c->ws(c->lay.lens), (const TableDelta*)d_stage,
-                             (const int32_t*)(d_stage + off_data), nd,
-                             (const int32_t*)(d_stage + off_pairs), np, st));
+                             (int32_t*)c->ws(c->lay.lens), (const TableDelta*)src,
+                             (const int32_t*)(src + off_data), nd,
+                             (const int32_t*)(src + off_pairs), np, st));
+    if (s->mapped) {
+      rc = send(c, s, nullptr, 0, st);      // nothing to copy: only marks the buffer in flight
+      if (rc) return rc;
+    }
     ++c->kernels_total;
     ++c->last.attn_kernels;
   }
