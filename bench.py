@@ -204,11 +204,12 @@ def run_ours(args, cfg_id):
     class S:      # the session in use: the end-to-end arm rebuilds it, see below
         sess = step0 = base_live = base_live_arr = None
         setup_s = 0.0
+        graph = graph_in = graph_ptrs = None
 
     def make_session():
         if S.sess is not None:
             S.sess.close()
-            S.sess = S.step0 = None
+            S.sess = S.step0 = S.graph = None
             torch.cuda.empty_cache()
         t0 = time.perf_counter()
         S.sess = PagedSession(shape, nb + grow_blocks, nt + n_step_forks,
@@ -253,10 +254,15 @@ def run_ours(args, cfg_id):
         if record:
             e1.record()
             attn_events.append((e0, e1))
-        for l in range(1, L):          # the other layers: scatter + attention launches only
-            B.apar_append_kv_layer(sess.ctx, l, k_new.data_ptr(), v_new.data_ptr(), stream)
-            B.apar_tree_decode_attention_layer(sess.ctx, l, q.data_ptr(), out.data_ptr(),
-                                               sess.sm_scale, stream)
+        if S.graph is not None:        # the other layers, replayed from the captured graph
+            if (q.data_ptr(), k_new.data_ptr(), out.data_ptr()) != S.graph_ptrs:
+                S.graph_in[0].copy_(q); S.graph_in[1].copy_(k_new); S.graph_in[2].copy_(v_new)
+            S.graph.replay()
+        else:
+            for l in range(1, L):      # the other layers: scatter + attention launches only
+                B.apar_append_kv_layer(sess.ctx, l, k_new.data_ptr(), v_new.data_ptr(), stream)
+                B.apar_tree_decode_attention_layer(sess.ctx, l, q.data_ptr(), out.data_ptr(),
+                                                   sess.sm_scale, stream)
         if kids:
             B.apar_release(sess.ctx, kids)
 
@@ -274,6 +280,31 @@ def run_ours(args, cfg_id):
     for i in range(args.warmup):
         one_step(*inputs[i % len(inputs)], record=False)
     barrier()
+
+    def capture_layer_loop(out_buf):
+        """Layers 1.. of a step only launch kernels whose sizes the cached plan fixes: capture
+        them once; valid while the plan is reused (threads only grow)."""
+        S.graph_in = [torch.empty_like(inputs[0][0]), torch.empty_like(inputs[0][1]),
+                      torch.empty_like(inputs[0][2])]
+        for dst, src in zip(S.graph_in, inputs[0]):
+            dst.copy_(src)
+        gq, gk, gv = S.graph_in
+        S.graph_ptrs = (gq.data_ptr(), gk.data_ptr(), out_buf.data_ptr())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            cs = torch.cuda.current_stream().cuda_stream
+            for l in range(1, L):
+                B.apar_append_kv_layer(S.sess.ctx, l, gk.data_ptr(), gv.data_ptr(), cs)
+                B.apar_tree_decode_attention_layer(S.sess.ctx, l, gq.data_ptr(), out_buf.data_ptr(),
+                                                   S.sess.sm_scale, cs)
+        S.graph = graph
+
+    if args.graph:
+        if L < 2 or S.step0.fork_parents:
+            raise SystemExit("--graph needs --layers >= 2 and a workload without forks in the step")
+        capture_layer_loop(out)
+        one_step(*inputs[0], record=False)
+        barrier()
     k0 = S.sess.stats()["kernels_total"]
     sampler = ClockSampler(local)
     if rank == 0:
@@ -433,7 +464,8 @@ def run_ours(args, cfg_id):
                 "head_dim": shape.head_dim, "block_size": shape.block_size,
                 "step": ("fork+" if has_fork else "") + "append+attention, " +
                         ("one layer" if L == 1 else f"{L} layers (value counts thread-tokens "
-                                                    f"per layer)"),
+                                                    f"per layer)") +
+                        (", layers 1.. replayed from a CUDA graph" if args.graph else ""),
                 "l2": "inputs larger than L2 (unique KV bytes per step >> 126 MB)"
                       if not small else "KV fits in L2: 256 MB written between steps, each step "
                                         "timed on its own (device arm)",
@@ -496,6 +528,9 @@ def main():
     ap.add_argument("--unshared", action="store_true",
                     help="same live threads, but every thread owns a private copy of its whole "
                          "chain (the copy-the-prefix-on-fork policy); for comparison with the tree")
+    ap.add_argument("--graph", action="store_true",
+                    help="with --layers >= 2: layers 1.. of a step are replayed from a CUDA graph "
+                         "(device arm only)")
     ap.add_argument("--layers", type=int, default=1,
                     help="attention layers per step (layers > 0 replay the plan; default 1)")
     args = ap.parse_args()

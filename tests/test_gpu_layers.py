@@ -72,3 +72,69 @@ def test_layers_share_tables_and_plan(config, nreq):
     sess.release(extra)
     assert sess.stats()["device_wait_timeouts"] == 0
     sess.close()
+
+
+def test_layer_loop_replayed_from_a_cuda_graph():
+    """The per-layer calls only launch kernels, with sizes fixed by the cached plan: the loop over
+    layers 1.. of a step is captured once in a CUDA graph and replayed, for this step and - the
+    plan being reused while threads only grow - for the next one."""
+    from paper_2401_06761_b200.session import PagedSession, pool_requirements
+    spec = synth.forest_spec(4, n_requests=3)
+    nb, nt, mb = pool_requirements(spec)
+    sess = PagedSession(spec.shape, nb + 64, nt, mb + 2, poison=True, num_layers=LAYERS)
+
+    class Layered:
+        new_threads, fork = sess.new_threads, sess.fork
+
+        @staticmethod
+        def append(tids, counts, k, v):
+            sess.append(tids, counts, k, v)
+            for l in range(1, LAYERS):
+                sess.append_layer(l, *_layer_rows(k, v, l))
+
+    step = synth.build_forest(spec, Layered, device="cuda")
+    live = step.live_handles
+    Layered.append(live, None, step.k_new, step.v_new)
+    sess.attention(live, step.q)                                   # plans; layer 0
+    q = [torch.roll(step.q, l, dims=-1).contiguous() for l in range(LAYERS)]
+    kv = [list(_layer_rows(step.k_new, step.v_new, l)) for l in range(LAYERS)]
+    eager = {l: sess.attention_layer(l, q[l]) for l in range(1, LAYERS)}
+    out_g = {l: torch.zeros_like(step.q) for l in range(1, LAYERS)}
+
+    def layer_loop():
+        for l in range(1, LAYERS):
+            sess.append_layer(l, kv[l][0], kv[l][1])
+            sess.attention_layer(l, q[l], out=out_g[l])
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        layer_loop()                                               # warm-up outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        layer_loop()
+    for o in out_g.values():
+        o.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    for l in range(1, LAYERS):
+        assert torch.equal(out_g[l], eager[l]), l
+    # next decode step: bookkeeping and layer 0 as usual, the other layers from the same graph
+    g = torch.Generator(device="cuda").manual_seed(5)
+    k2 = torch.randn(step.k_new.shape, generator=g, device="cuda").to(torch.bfloat16)
+    v2 = torch.randn(step.v_new.shape, generator=g, device="cuda").to(torch.bfloat16)
+    sess.append(live, None, k2, v2)
+    sess.attention(live, step.q)
+    assert sess.stats()["attn_plan_reused"] == 1
+    for l in range(1, LAYERS):
+        kl, vl = _layer_rows(k2, v2, l)
+        kv[l][0].copy_(kl)
+        kv[l][1].copy_(vl)
+        out_g[l].zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    for l in range(1, LAYERS):
+        assert torch.equal(out_g[l], sess.attention_layer(l, q[l])), l   # eager, same pools
+    assert sess.stats()["device_wait_timeouts"] == 0
+    sess.close()
