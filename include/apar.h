@@ -21,6 +21,9 @@
  *     as void*; NULL = the default stream).  Host bookkeeping is complete on return.  All
  *     calls on one context must use streams that are ordered with respect to each other
  *     (normally one stream); a context is not thread-safe.
+ *   - The library's own uploads (slot lists, table deltas, plans: KBs per step) are read from
+ *     its pinned, mapped staging buffers by kernels on `cuda_stream`, not by a copy engine,
+ *     so they never wait behind the caller's host-to-device copies on other streams.
  *   - Batched calls process their entries in index order and are all-or-nothing: on any
  *     error no host state changes and nothing is launched.
  *   - No exceptions, aborts or device traps cross this boundary; errors are status codes.
