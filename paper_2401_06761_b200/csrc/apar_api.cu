@@ -108,6 +108,8 @@ struct apar_ctx {
   int plan_age = 0;
   int mma_min_rows = INT_MAX;
   int umma_min_tiles = 2;               // items with at least this many 16-row tiles use tcgen05
+  int use_pdl = 1;                      // warp-stream launches may start before the kernel before
+                                        // them has finished (0: ordinary launches only)
   bool use_ws = true;                   // single-tile items use the warp-stream kernel
   std::vector<CUtensorMap> tm_k, tm_v;   // one pair per layer
   size_t layer_bytes = 0;                // bytes of one layer of a pool
@@ -285,6 +287,15 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
   a.tm_k = &c->tm_k[layer];
   a.tm_v = &c->tm_v[layer];
   a.d_error = (int*)c->ws(c->lay.err);
+  // The first attention kernel of the call is launched the ordinary way (it starts after the
+  // table sync and the append have completed).  A warp-stream launch that follows another
+  // attention kernel may start while that kernel is still in its last wave, and orders itself
+  // where it has to (pdl_wait).  Measured: worth 2 % where tensor-core and warp-stream
+  // kernels follow each other (config 5), nothing on config 4; the single-row kernel lost
+  // 10-25 % when its finishing items started early (configs 2 and 3), so it and the merge are
+  // launched the ordinary way, which also orders them after everything before them.
+  const int chain = c->use_pdl ? 1 : 0;
+  bool first = true;
   if (p.n_mma) {
     // items are ordered 4, 3, 2, 1 query tiles: the first umma_min_tiles.. classes go to tcgen05
     int32_t sync_counts[4], n_umma = 0;
@@ -294,33 +305,47 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
       if (umma) n_umma += p.n_mma_tiles[k];
     }
     if (n_umma) {
+      a.pdl = 0;
       APAR_CUDA(c, launch_attention_umma(a, p.n_vec, n_umma, st));
       ++*launches_out;
+      first = false;
     }
     if (c->use_ws && sync_counts[0] > 0) {
       // single-tile items are last in the list: whole items (all kv heads) per CTA; the
       // finishing ones wait until every other item has been launched
-      const int first = p.n_vec + p.n_mma - sync_counts[0];
+      const int first_item = p.n_vec + p.n_mma - sync_counts[0];
       const int n_plain = sync_counts[0] - p.n_mma1_final;
       if (n_plain > 0) {
-        APAR_CUDA(c, launch_attention_ws(a, first, n_plain, st));
+        a.pdl = first ? 0 : chain;
+        APAR_CUDA(c, launch_attention_ws(a, first_item, n_plain, st));
         ++*launches_out;
+        first = false;
       }
       sync_counts[0] = 0;
     }
+    a.pdl = 0;
     APAR_CUDA(c, launch_attention_mma(a, p.n_vec + n_umma, sync_counts, st));
-    for (int k = 0; k < 4; ++k) (*launches_out) += sync_counts[k] > 0;
+    for (int k = 0; k < 4; ++k)
+      if (sync_counts[k] > 0) {
+        ++*launches_out;
+        first = false;
+      }
   }
   const bool single_row = c->shape.group == 1 && c->mma_min_rows <= 2;
+  a.pdl = 0;
   if (p.n_vec - p.n_vec_final > 0) {
     APAR_CUDA(c, launch_attention_vec(a, 0, p.n_vec - p.n_vec_final, single_row, st));
     ++*launches_out;
+    first = false;
   }
   // finishing items: everything they fold has been enqueued before them on this stream
   if (p.n_mma1_final > 0) {
+    a.pdl = first ? 0 : chain;
     APAR_CUDA(c, launch_attention_ws(a, p.n_vec + p.n_mma - p.n_mma1_final, p.n_mma1_final, st));
     ++*launches_out;
+    first = false;
   }
+  a.pdl = 0;
   if (p.n_vec_final > 0) {
     APAR_CUDA(c, launch_attention_vec(a, p.n_vec - p.n_vec_final, p.n_vec_final, single_row, st));
     ++*launches_out;
@@ -447,6 +472,8 @@ apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
   const char* path = getenv("APAR_ATTN_PATH");
   c->mma_min_rows = (path && !strcmp(path, "vec")) ? INT_MAX : (path && !strcmp(path, "ws")) ? 1 : 2;
   c->umma_min_tiles = (path && !strcmp(path, "mma")) ? 5 : (path && !strcmp(path, "umma")) ? 1 : 2;
+  const char* pdl = getenv("APAR_PDL");                  // testing: 0 = ordinary launches only
+  c->use_pdl = pdl ? atoi(pdl) : 1;
   c->use_ws = !(path && (!strcmp(path, "mma") || !strcmp(path, "umma")));
   c->ring_bytes = lay.stage_cap;
   c->num_layers = std::max(1, cfg->num_layers);

@@ -61,6 +61,41 @@ struct Shape {
   int32_t table_stride;        // ints per device table row
 };
 
+// ---- programmatic dependent launch ------------------------------------------------------
+// A warp-stream attention launch that follows another attention kernel of the same call is
+// allowed to take the SM slots its predecessor's last wave leaves free.  Rules that keep this
+// correct:
+//   * the tensor-core and warp-stream kernels call pdl_launch_dependents() early, so that a
+//     successor may start as soon as all of their own CTAs have started;
+//   * a CTA calls pdl_wait() before it reads what an earlier kernel of the call wrote
+//     (partial results) - it returns once the predecessor grid has completed and flushed;
+//   * a CTA that reads nothing of the kind still calls pdl_wait() before it exits, so that
+//     "this grid has completed" implies "every earlier grid of the call has completed".
+// Both are no-ops in a kernel that was launched the ordinary way; all other kernels are
+// launched the ordinary way and start after everything before them on the stream.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t st, bool pdl, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // ---- kernel launchers (kernels.cu); all enqueue on `st` and return cudaGetLastError() ----
 cudaError_t launch_cow_copy(void* k_pool, void* v_pool, const CowCopy* d_copies, int n,
                             int num_kv_heads, cudaStream_t st);
@@ -90,6 +125,9 @@ struct AttnArgs {
   const CUtensorMap* tm_k = nullptr;  // [host] TMA descriptors of the pools (tensor-core path)
   const CUtensorMap* tm_v = nullptr;
   int* d_error = nullptr;             // [device] set to 1 when a bounded wait gave up
+  // 1: this launch is allowed to start before the launch before it on the stream has finished
+  // (programmatic dependent launch); its kernel then orders itself with pdl_wait()
+  int pdl = 0;
 };
 // single_row: every item carries exactly one query row.
 cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items, bool single_row,

@@ -268,6 +268,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     return;
   }
   const uint32_t tm_o = tmem + 128u;      // S buffer b sits at columns [64 b, 64 b + 64)
+  if (threadIdx.x == 0) pdl_launch_dependents();
 
   if (warp == 4) {
     // ---------------------------------------------------------------- TMA producer
@@ -624,6 +625,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     }
   }
   // ---- common exit: every role arrives here, then the allocating warp frees TMEM
+  if (a.pdl && threadIdx.x == 0) pdl_wait();      // this grid completes after its predecessor
   tc_fence_before();
   __syncthreads();
   if (warp == 5) {
@@ -663,8 +665,8 @@ cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items
     if (hkv % c == 0 && (long long)n_items * (hkv / c) >= (long long)kWavesMin * 2 * sm_count[dev])
       u = c;
   if (force && atoi(force) >= 1 && hkv % atoi(force) == 0) u = atoi(force);
-  attn_umma_kernel<<<dim3(n_items, hkv / u), 192, kSmem, st>>>(*a.tm_k, *a.tm_v, a, item_begin, u);
-  return cudaGetLastError();
+  return launch_kernel(attn_umma_kernel, dim3(n_items, hkv / u), dim3(192), kSmem, st, a.pdl != 0,
+                       *a.tm_k, *a.tm_v, a, item_begin, u);
 }
 
 }  // namespace apar

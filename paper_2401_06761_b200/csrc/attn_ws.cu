@@ -141,6 +141,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   else if (threadIdx.x < it.n_users) s_users[threadIdx.x] = a.d_users[it.user_begin + threadIdx.x];
   __syncthreads();
   if (*cta_abort) return;
+  if (threadIdx.x == 0) pdl_launch_dependents();
 
   if (warp == 4) {
     // ------------------------------------------------------------------ producer warp
@@ -169,6 +170,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         if (b == 0) ++hi;
       }
     }
+    if (a.pdl) pdl_wait();                         // this grid completes after its predecessor
     return;
   }
 
@@ -202,7 +204,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
   for (int ks = 0; ks < 8; ++ks) qn[ks][0] = qn[ks][1] = qn[ks][2] = qn[ks][3] = 0u;
   if (heads_w > 0) load_q(h_begin + w, qa);
   int c = 0;                                       // blocks consumed so far by this warp
-  bool alive = true;
+  bool alive = true, waited = false;
   for (int hi = 0; hi < heads_w && alive; ++hi) {
     const int h = h_begin + w + 4 * hi;
     if (hi + 1 < heads_w) load_q(h + 4, qn);       // lands while this head streams
@@ -295,6 +297,11 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    // the partial results a finishing item folds come from earlier kernels of the call
+    if (a.pdl && it.fin_n > 0 && !waited) {
+      pdl_wait();
+      waited = true;
+    }
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       const int r = g + 8 * half;
@@ -339,6 +346,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 #pragma unroll
       for (int e = 0; e < 4; ++e) qa[ks][e] = qn[ks][e];
   }
+  if (a.pdl) pdl_wait();                           // this grid completes after its predecessor
 }
 
 }  // namespace
@@ -362,9 +370,8 @@ cudaError_t launch_attention_ws(const AttnArgs& a, int item_begin, int n_items, 
   const int groups = want < 1 ? 1 : (want > max_groups ? max_groups : want);
   const int heads_per_cta = ((hkv + groups - 1) / groups + 3) / 4 * 4;
   const int grid_y = (hkv + heads_per_cta - 1) / heads_per_cta;
-  attn_ws_kernel<<<dim3(n_items, grid_y), 160, kSmemW, st>>>(*a.tm_k, *a.tm_v, a, item_begin,
-                                                             heads_per_cta);
-  return cudaGetLastError();
+  return launch_kernel(attn_ws_kernel, dim3(n_items, grid_y), dim3(160), kSmemW, st, a.pdl != 0,
+                       *a.tm_k, *a.tm_v, a, item_begin, heads_per_cta);
 }
 
 }  // namespace apar
