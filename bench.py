@@ -446,7 +446,7 @@ def run_ours(args, cfg_id):
     # the requests processed; DRAM traffic is proportional to them).  Only for the full cfg4.
     traffic = None
     if cfg_id == 4 and args.requests is None and not args.unshared and L == 1:
-        traffic = ((546.8 + 29.4) + (735.0 + 12.9)) * 1e6 * (512 / 64)
+        traffic = ((546.5 + 30.8) + (735.6 + 12.8)) * 1e6 * (512 / 64)
 
     if rank == 0:
         cpu_rate, cpu_threads, cores = (oracle_sample(spec, 12.0)
