@@ -41,7 +41,9 @@ bool supported(const apar_config* c) {
 Layout make_layout(const apar_config* c) {
   Layout L;
   const size_t table_bytes = (size_t)c->max_threads * c->max_blocks_per_thread * 4;
-  L.slot_capacity = (int64_t)c->max_threads * kSlotsPerThread;
+  // partial rows: several per live thread, and never fewer than one per (SM, resident CTA)
+  // so that a few very long threads can still be spread over the whole machine
+  L.slot_capacity = std::max<int64_t>((int64_t)c->max_threads * kSlotsPerThread, 148 * 8);
   L.entry_capacity = L.slot_capacity + c->max_threads;
   L.stage_cap = std::min<size_t>(std::max<size_t>(table_bytes / 4 + (64 << 10), 1 << 20), 64 << 20);
   size_t off = 0;
@@ -950,7 +952,8 @@ apar_status apar_debug_plan(int32_t num_blocks, int32_t num_q_heads, int32_t num
   Planner planner;
   planner.init(num_blocks, num_q_heads / num_kv_heads, num_kv_heads);
   Plan plan;
-  if (!planner.build(pq.data(), n_threads, (int64_t)kSlotsPerThread * n_threads, false,
+  if (!planner.build(pq.data(), n_threads,
+                     std::max<int64_t>((int64_t)kSlotsPerThread * n_threads, 148 * 8), false,
                      mma_min_rows, fuse_final != 0, &plan))
     return APAR_ERR_WORKSPACE_TOO_SMALL;
   counts_out[0] = (int64_t)plan.items.size();

@@ -368,3 +368,37 @@ def test_tcgen05_kernel_with_several_kv_heads_per_cta(heads, monkeypatch):
         assert err.mean() <= 1e-3 + 2.0 ** -9 * np.abs(ref).mean(), (heads, prompt, err.mean())
         assert sess.stats()["device_wait_timeouts"] == 0
         sess.close()
+
+
+@pytest.mark.parametrize("kids", [1, 3, 6])
+def test_long_context_shared_by_forks(kids, monkeypatch):
+    """A 131 077-token prompt (8193 blocks, ragged end) read by 1, 3 or 6 forked threads: the run
+    is cut into chunks over all SMs, shared chunks go to the warp-stream kernel (12 rows) or the
+    tensor-core kernel (24 rows), and every query merges dozens of partial results."""
+    shape = synth.LayerShape(8, 2)
+    monkeypatch.setenv("APAR_ATTN_PATH", "auto")
+    n = 131072 + 5
+    nb = 8193 + 8 * 3 + 4
+    sess = _session(shape, nb, 8, 8200, poison=True)
+    orc = OracleBackend(shape, nb, 8, 8200)
+    both = Both(sess, orc)
+    g = torch.Generator(device="cuda").manual_seed(77)
+    k = torch.randn((n, 2, 128), generator=g, device="cuda").to(torch.bfloat16)
+    v = torch.randn((n, 2, 128), generator=g, device="cuda").to(torch.bfloat16)
+    (p,) = both.new_threads(1)
+    both.append([p], [n], k, v)
+    tids = both.fork([p] * kids) if kids > 1 else [p]
+    if kids > 1:
+        cnt = [3 + 7 * i for i in range(kids)]
+        both.append(tids, cnt,
+                    torch.randn((sum(cnt), 2, 128), generator=g, device="cuda").to(torch.bfloat16),
+                    torch.randn((sum(cnt), 2, 128), generator=g, device="cuda").to(torch.bfloat16))
+    assert_same_bookkeeping(sess, orc.model, list(orc.model.tables))
+    q = torch.randn((len(tids), 8, 128), generator=g, device="cuda").to(torch.bfloat16)
+    out = sess.attention(tids, q)
+    assert_close(out, orc.attention(tids, q, sess.sm_scale), f"128k context, {kids} threads")
+    st = sess.stats()
+    assert st["device_wait_timeouts"] == 0
+    assert st["attn_unique_tokens"] == orc.model.unique_tokens(tids)
+    assert st["attn_work_items"] >= 100          # the prompt is spread over the machine
+    sess.close()
