@@ -473,18 +473,34 @@ __global__ void __launch_bounds__(128) merge_kernel(const AttnArgs a,
   const int lane = threadIdx.x & 31;
   const int HQ = a.shape.num_q_heads;
   if (head >= HQ) return;
+  // the reference maximum: the lanes share the partial results out among themselves
   float M = -INFINITY;
-  for (int j = 0; j < mr.n; ++j)
+  for (int j = lane; j < mr.n; j += 32)
     M = fmaxf(M, a.part_ml[(size_t)(mr.slot_begin + j) * HQ + head].x);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  // weighted sum in slot order, eight partial results in flight at a time
   float L = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int j = 0; j < mr.n; ++j) {
-    const size_t prow = (size_t)(mr.slot_begin + j) * HQ + head;
-    const float2 ml = a.part_ml[prow];
-    const float w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
-    const float4 o = ((const float4*)(a.part_o + prow * kDim))[lane];
-    L += ml.y * w;
-    acc.x += o.x * w; acc.y += o.y * w; acc.z += o.z * w; acc.w += o.w * w;
+  for (int j0 = 0; j0 < mr.n; j0 += 8) {
+    float2 ml[8];
+    float4 o[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      ml[k] = make_float2(-INFINITY, 0.f);
+      o[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (j0 + k < mr.n) {
+        const size_t prow = (size_t)(mr.slot_begin + j0 + k) * HQ + head;
+        ml[k] = a.part_ml[prow];
+        o[k] = ((const float4*)(a.part_o + prow * kDim))[lane];
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float w = ml[k].x == -INFINITY ? 0.f : exp2f(ml[k].x - M);
+      L += ml[k].y * w;
+      acc.x += o[k].x * w; acc.y += o[k].y * w; acc.z += o[k].z * w; acc.w += o[k].w * w;
+    }
   }
   const float inv = 1.f / L;
   __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);

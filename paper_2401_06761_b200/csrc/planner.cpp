@@ -28,6 +28,7 @@ void Planner::init(int num_blocks, int group, int num_kv_heads) {
 }
 
 static inline int64_t round_up16(int64_t x) { return (x + 15) / 16 * 16; }
+constexpr int kMaxFoldedParts = 8;   // partial results a finishing item may fold by itself
 
 bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_tails,
                     int mma_min_rows, bool fuse_final, Plan* out) {
@@ -105,6 +106,28 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
   // ---- chunk length: enough items to fill the machine, never below 128 tokens
   const int64_t kInf = (int64_t)1 << 40;
   int64_t chunk = std::max<int64_t>(128, round_up16(unique * hint_kv_heads_ / (148 * 8)));
+  // `chunk` is sized for the kernels that keep a CTA's loads in flight through TMA rings.  The
+  // single-row kernel has no such staging and needs several CTAs per SM to cover the latency:
+  // when its runs, dealt out four kv heads to a CTA, would give fewer than four CTAs per SM,
+  // they are cut finer (up to eight times).  This only happens with a few very long threads.
+  const int max_users = std::max(1, kMaxRowsPerItem / group_);
+  auto single_row = [&](const Seg& g) {
+    return std::min(g.n_users, max_users) * group_ < mma_min_rows;
+  };
+  int64_t vec_div = 1;
+  {
+    int64_t vec_chunks = 0;
+    for (const Seg& g : segs_)
+      if (single_row(g))
+        vec_chunks += (g.tok_end - g.tok_begin + chunk - 1) / chunk * ((g.n_users + max_users - 1) / max_users);
+    const int64_t head_groups = (hint_kv_heads_ + 3) / 4;
+    while (vec_chunks > 0 && vec_div < 8 && vec_chunks * vec_div * head_groups < 4 * 148) vec_div *= 2;
+  }
+  auto seg_chunk = [&](const Seg& g) -> int64_t {
+    if (chunk >= kInf) return kInf;
+    if (vec_div == 1 || !single_row(g)) return chunk;
+    return std::max<int64_t>(128, round_up16(chunk / vec_div));
+  };
   n_parts_.assign(n, 0);
   int64_t total_slots = 0;
   for (int attempt = 0;; ++attempt) {
@@ -113,8 +136,9 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
       int32_t ord = 0;
       for (int k = qbeg_[i]; k < qbeg_[i + 1]; ++k) {
         const Seg& g = segs_[seg_users_[k].seg];
+        const int64_t ck = seg_chunk(g);
         seg_users_[k].ord = ord;
-        ord += (int32_t)((g.tok_end - g.tok_begin + chunk - 1) / chunk);
+        ord += (int32_t)((g.tok_end - g.tok_begin + ck - 1) / ck);
       }
       n_parts_[i] = ord;
       if (ord >= 2) total_slots += ord;
@@ -134,7 +158,9 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
       part_off_[i] = off;
       // the chain ends in a private run: its last item can finish the query on its own
       const Seg& last = segs_[seg_users_[qbeg_[i + 1] - 1].seg];
-      if (fuse_final && last.priv && group_ <= 16) fused_[i] = 1;
+      // (folding is serial work of one CTA: chains cut into many pieces go to the merge kernel)
+      if (fuse_final && last.priv && group_ <= 16 && n_parts_[i] - 1 <= kMaxFoldedParts)
+        fused_[i] = 1;
       if (!fused_[i]) out->merges.push_back(MergeRef{i, off, n_parts_[i], 0});
       off += n_parts_[i];
     }
@@ -153,12 +179,12 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
         UserRef{su.query, part_off_[su.query] >= 0 ? part_off_[su.query] + su.ord : -1};
   }
   // ---- items
-  const int max_users = std::max(1, kMaxRowsPerItem / group_);
   vec_items_.clear();
   vec_final_.clear();
   mma1_final_.clear();
   for (auto& v : mma_items_) v.clear();
   for (const Seg& g : segs_) {
+    const int64_t chunk = seg_chunk(g);        // this run's own chunk length
     const int32_t n_chunks = (int32_t)((g.tok_end - g.tok_begin + chunk - 1) / chunk);
     for (int u0 = 0; u0 < g.n_users; u0 += max_users) {
       const int nu = std::min(max_users, g.n_users - u0);

@@ -158,3 +158,20 @@ def test_rejects_bad_input():
         B.apar_debug_plan(8, 4, 4, tab, [20])
     with pytest.raises(B.AparError):
         B.apar_debug_plan(8, 6, 4, tab[:, :1], [5])
+
+
+def test_few_long_threads_are_spread_over_the_machine():
+    m = BlockModel(9000, BS, 8, 8300)
+    (p,) = m.new_threads(1)
+    m.append([p], [131072 + 5])
+    # one thread, 8 kv heads, 8 query rows per kv head: the ring-fed kernels get about one
+    # (item, head) pair per CTA slot of the machine
+    c = check_plan(m, [p], 64, 8, 2, True)
+    assert 140 <= c["items"] <= 160 and c["merges"] == 1        # too many pieces to fold in one CTA
+    # single-row items (32 kv heads, no sharing): cut finer, several CTAs per SM
+    c1 = check_plan(m, [p], 32, 32, 2, True)
+    assert c1["items"] >= 2 * 37
+    # many threads: no cut at all
+    m2, live = random_forest(5, n_roots=3, steps=40)
+    c2 = check_plan(m2, live, 32, 32, 2, True)
+    assert c2["items"] <= 2 * c2["users"]
