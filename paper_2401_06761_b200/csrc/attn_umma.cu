@@ -1,7 +1,8 @@
 // Blackwell tensor-core attention path (tcgen05 + TMEM) for work items with many query rows:
 // a run of blocks shared by up to 64 (query, head) rows.
 //
-// One CTA owns one (work item, kv head).  Roles:
+// One CTA owns one work item and one kv head of it, or a few consecutive kv heads that it works
+// through back to back.  Roles:
 //   warps 0-3  softmax: warp w owns query rows 16w .. 16w+15, which are TMEM lanes 32w .. 32w+15
 //              of an M = 64 accumulator.  S is read with the 16-lane x 256-bit TMEM load, which
 //              spreads a row over the four threads of a quad, so that all 32 lanes work; they
