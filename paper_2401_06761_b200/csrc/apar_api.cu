@@ -18,6 +18,7 @@ namespace {
 constexpr int kRing = 12;             // pinned staging buffers in flight: enough for the uploads of
                                       // two whole steps, so that the host can prepare a step
                                       // while the GPU still runs the one before
+constexpr int kFewQueries = 768;      // up to here single-row items go to the warp-stream kernel
 constexpr int kSlotsPerThread = 6;    // partial-result rows provisioned per live thread
 constexpr int kSlotMapRows = 262144;  // new-row slots of the last append kept for other layers
 
@@ -109,6 +110,8 @@ struct apar_ctx {
   int64_t plan_attended = 0;
   int plan_age = 0;
   int mma_min_rows = INT_MAX;
+  int plan_min_rows = INT_MAX;          // the value the current plan was built with
+  bool auto_path = true;                // no kernel family forced
   int umma_min_tiles = 2;               // items with at least this many 16-row tiles use tcgen05
   int use_pdl = 1;                      // warp-stream launches may start before the kernel before
                                         // them has finished (0: ordinary launches only)
@@ -333,7 +336,7 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
         first = false;
       }
   }
-  const bool single_row = c->shape.group == 1 && c->mma_min_rows <= 2;
+  const bool single_row = c->shape.group == 1 && c->plan_min_rows <= 2;
   a.pdl = 0;
   if (p.n_vec - p.n_vec_final > 0) {
     APAR_CUDA(c, launch_attention_vec(a, 0, p.n_vec - p.n_vec_final, single_row, st));
@@ -381,9 +384,14 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
     for (int i = 0; i < n; ++i)
       c->pq[i] = PlanQuery{c->row(qslots[i]), qslots[i],
                            qlens ? qlens[i] : c->slots[qslots[i]].len};
+    // Single-row items (no GQA group, private tail): the vector kernel keeps up to 16 CTAs per
+    // SM in flight and wins when there are many of them; with few, the warp-stream kernel's
+    // deeper per-warp rings do better (measured crossover near 900 queries).
+    c->plan_min_rows = c->mma_min_rows;
+    if (c->auto_path && c->shape.group == 1 && n <= kFewQueries) c->plan_min_rows = 1;
     // finishing items land in the single-row vector kernel or the warp-stream kernel
-    const bool fuse_final = c->use_ws && c->mma_min_rows <= 2;
-    if (!c->planner.build(c->pq.data(), n, c->lay.slot_capacity, cacheable, c->mma_min_rows,
+    const bool fuse_final = c->use_ws && c->plan_min_rows <= 2;
+    if (!c->planner.build(c->pq.data(), n, c->lay.slot_capacity, cacheable, c->plan_min_rows,
                           fuse_final,
                           &c->plan))
       return APAR_ERR_WORKSPACE_TOO_SMALL;
@@ -477,6 +485,7 @@ apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
   const char* pdl = getenv("APAR_PDL");                  // testing: 0 = ordinary launches only
   c->use_pdl = pdl ? atoi(pdl) : 1;
   c->use_ws = !(path && (!strcmp(path, "mma") || !strcmp(path, "umma")));
+  c->auto_path = !path || !strcmp(path, "auto") || !*path;
   c->ring_bytes = lay.stage_cap;
   c->num_layers = std::max(1, cfg->num_layers);
   c->layer_bytes = (size_t)cfg->num_blocks * cfg->num_kv_heads * kTileBytes;
