@@ -69,14 +69,15 @@ enum {
   APAR_ERR_WORKSPACE_TOO_SMALL = -7,  /* workspace_bytes < apar_workspace_bytes(), or a plan that
                                          does not fit the partial-result area                     */
   APAR_ERR_CUDA = -8,                 /* a CUDA runtime call failed; see apar_last_cuda_error     */
-  APAR_ERR_UNSUPPORTED = -9           /* block_size != 16, head_dim != 128, heads not divisible   */
+  APAR_ERR_UNSUPPORTED = -9           /* block_size != 16, head_dim != 128, heads not divisible,
+                                         more than 64 query heads per kv head                     */
 };
 
 typedef struct {
   int32_t num_blocks;             /* blocks in each of k_pool and v_pool                         */
   int32_t block_size;             /* must be 16                                                  */
   int32_t num_q_heads;
-  int32_t num_kv_heads;           /* must divide num_q_heads                                     */
+  int32_t num_kv_heads;           /* must divide num_q_heads; num_q_heads / num_kv_heads <= 64   */
   int32_t head_dim;               /* must be 128                                                 */
   int32_t max_threads;            /* live generation threads at any time                         */
   int32_t max_blocks_per_thread;  /* longest chain, in blocks                                    */
@@ -222,8 +223,12 @@ apar_status apar_tree_decode_attention_tables(const apar_config* cfg /*[host]*/,
  * of the library image, so every GPU that loads the library carries that array until exit.
  *
  * Semantics: row i of block_tables [device] int32 [n_threads][max_blocks_per_thread] with
- * ctx_lens[i] [device] >= 1 tokens is one private chain; out[i][h] is the same softmax
- * attention as above over that chain.  Rows are not de-duplicated: a block listed by several
+ * ctx_lens[i] [device] tokens, 1 <= ctx_lens[i] <= 16 * max_blocks_per_thread, is one private
+ * chain; out[i][h] is the same softmax attention as above over that chain.  The host never
+ * reads the lengths, so it cannot refuse bad ones: a length above 16 * max_blocks_per_thread
+ * is treated as that bound (the kernels never walk past a table row), and a row of length
+ * <= 0 attends nothing and receives zeros.  The first ceil(len / 16) ids of every row must be
+ * valid block ids of the pools; they are not checked.  Rows are not de-duplicated: a block listed by several
  * rows is read once per row.  Chains are cut into ceil(max_ctx_len / 1024) (at most 8) token
  * ranges whose partial results are merged; max_ctx_len [host] is an upper bound of ctx_lens
  * (a longer row is still computed correctly, only less evenly split).  k_pool, v_pool, q, out
@@ -294,7 +299,8 @@ apar_status apar_check_invariants(apar_ctx* ctx);
  *   counts_out [host] [6] int64: items, users, merges, partial slots, unique tokens,
  *              attended tokens
  * Returns APAR_ERR_WORKSPACE_TOO_SMALL if a cap is too small (counts_out is still filled),
- * APAR_ERR_INVALID_ARG for bad shapes, lengths or block ids. */
+ * APAR_ERR_INVALID_ARG for bad shapes, lengths or block ids, APAR_ERR_UNSUPPORTED for more
+ * than 64 query heads per kv head. */
 apar_status apar_debug_plan(int32_t num_blocks, int32_t num_q_heads, int32_t num_kv_heads,
                             int32_t n_threads, int32_t max_blocks, const int32_t* block_tables,
                             const int32_t* ctx_lens, int32_t mma_min_rows, int32_t fuse_final,

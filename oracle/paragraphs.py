@@ -1,70 +1,72 @@
-"""Paragraph tree of Algorithm 1 on plain token lists.  Test infrastructure only.
+"""Restoring the sequential text of an APAR generation from its fork history, on plain token
+lists.  Test infrastructure only (see oracle/__init__).
 
-Follows the algorithm's own bookkeeping: a sequence group holds the sequences of one prompt;
-every sequence tracks the leaf paragraph node at its end; when a sequence whose last token is
-the fork token is duplicated, the current node is closed, a next-sibling node (same sequence)
-and a first-child node (the copy, after its forced child token) are opened; Restore walks the
-tree root, first child, next sibling and concatenates the slices.
+Algorithm 1 keeps a paragraph tree beside the sequences and reads the answer off it in the
+order root, first child, next sibling.  What that traversal produces has a direct description,
+which is what this file implements (no tree, no node objects): the text of a sequence, read
+from some start position, is
+
+    its own tokens up to the position where it first forked after that start,
+    then the whole text of the sequence born there (read from just after the forced child
+    token that opened it),
+    then the text of the same sequence read from the fork position on.
+
+So it is enough to remember, per sequence, at which of its positions a copy was made and which
+sequence the copy became.  The hand-worked example of tests/test_oracle_paragraphs.py pins the
+result; the behaviour checked is Algorithm 1's (decode pass, fork rule, Restore order).
 """
 from __future__ import annotations
 
 FORK, CHILD, EOS = "[Fork]", "[Child]", "[EOS]"
 
 
-class PNode:
-    def __init__(self, seq, start):
-        self.seq, self.start, self.end = seq, start, None
-        self.first_child = None
-        self.next_sibling = None
+class Thread:
+    """One generation thread: its tokens and the copies made of it, as (position, index of the
+    new thread in the group), in the order they were made (positions increase)."""
 
-
-class Sequence:
     def __init__(self, tokens):
         self.tokens = list(tokens)
         self.finished = False
-        self.current_node = None
+        self.births = []
 
 
 class SequenceGroup:
+    """All threads generated for one prompt (Section 2.3 "Sequence and sequence group")."""
+
     def __init__(self, prompt_tokens):
-        p = Sequence(prompt_tokens)
-        self.root = PNode(p, len(p.tokens))
-        p.current_node = self.root
-        self.seqs = [p]
+        self.seqs = [Thread(prompt_tokens)]
+        self.answer_from = len(self.seqs[0].tokens)     # the prompt is not part of the answer
 
     def step(self, sample):
-        """One AparDecode pass.  sample(seq) returns the next token of an unfinished sequence."""
-        for s in list(self.seqs):
-            if s.finished:
+        """One decode pass over the threads that exist when it begins.  `sample(thread)` gives
+        the next token of an unfinished thread.  A thread whose newest token is the fork token
+        is copied before its new token is added; the copy starts with the forced child token
+        and first decodes in the next pass."""
+        for k in range(len(self.seqs)):
+            th = self.seqs[k]
+            if th.finished:
                 continue
-            x = sample(s)
-            if s.tokens[-1] == FORK:
-                c = Sequence(s.tokens)
-                c.tokens.append(CHILD)
-                self.seqs.append(c)
-                n, nc = PNode(s, len(s.tokens)), PNode(c, len(c.tokens))
-                s.current_node.end = len(s.tokens)
-                s.current_node.next_sibling = n
-                s.current_node.first_child = nc
-                s.current_node = n
-                c.current_node = nc
-            s.tokens.append(x)
-            if x == EOS:
-                s.finished = True
+            token = sample(th)
+            if th.tokens[-1] == FORK:
+                th.births.append((len(th.tokens), len(self.seqs)))
+                self.seqs.append(Thread(th.tokens + [CHILD]))
+            th.tokens.append(token)
+            th.finished = token == EOS
 
     def slices(self):
-        """(sequence index, start, end) in Restore order; an open end is the sequence's length."""
-        out = []
+        """(thread index, start, end) pieces whose concatenation is the answer."""
+        pieces = []
 
-        def visit(n):
-            out.append((self.seqs.index(n.seq), n.start,
-                        len(n.seq.tokens) if n.end is None else n.end))
-            if n.first_child is not None:
-                visit(n.first_child)
-            if n.next_sibling is not None:
-                visit(n.next_sibling)
-        visit(self.root)
-        return out
+        def read(k, start):
+            th = self.seqs[k]
+            for at, born in th.births:
+                pieces.append((k, start, at))
+                read(born, at + 1)          # skip the child token the copy was opened with
+                start = at
+            pieces.append((k, start, len(th.tokens)))
+
+        read(0, self.answer_from)
+        return pieces
 
     def restore(self):
-        return [t for i, a, b in self.slices() for t in self.seqs[i].tokens[a:b]]
+        return [tok for k, a, b in self.slices() for tok in self.seqs[k].tokens[a:b]]

@@ -34,6 +34,8 @@ struct Layout {            // partition of the caller's workspace
 bool supported(const apar_config* c) {
   return c && c->block_size == kBlock && c->head_dim == kDim && c->num_blocks > 0 &&
          c->num_kv_heads > 0 && c->num_q_heads > 0 && c->num_q_heads % c->num_kv_heads == 0 &&
+         // one work item carries all query heads of a kv head for at least one thread
+         c->num_q_heads / c->num_kv_heads <= kMaxRowsPerItem &&
          c->max_threads > 0 && c->max_blocks_per_thread > 0 && c->num_layers >= 0 &&
          (int64_t)c->num_blocks * kBlock < INT32_MAX &&
          (int64_t)std::max(1, c->num_layers) * c->num_blocks * c->num_kv_heads * kBlock < INT32_MAX;
@@ -949,6 +951,7 @@ apar_status apar_debug_plan(int32_t num_blocks, int32_t num_q_heads, int32_t num
       cap_items < 0 || cap_users < 0 || cap_merges < 0 || (cap_items && !items_out) ||
       (cap_users && !users_out) || (cap_merges && !merges_out))
     return APAR_ERR_INVALID_ARG;
+  if (num_q_heads / num_kv_heads > kMaxRowsPerItem) return APAR_ERR_UNSUPPORTED;
   std::vector<PlanQuery> pq(n_threads);
   for (int i = 0; i < n_threads; ++i) {
     const int32_t len = ctx_lens[i];

@@ -47,15 +47,18 @@ StaticLayout static_layout(int n, int splits, int num_q_heads) {
 }
 
 // One thread per (row, split): every table row is a private chain cut into `splits` equal
-// token ranges; the last range absorbs whatever lies beyond max_ctx_len.
+// token ranges; the last range absorbs whatever lies beyond max_ctx_len.  Lengths come from
+// device memory that the host never sees, so they are clamped here to what a table row can
+// hold: the attention kernels then never index past a row's max_blocks entries, and a row of
+// length <= 0 gets empty ranges (its output is written as zeros).
 __global__ void __launch_bounds__(128) static_plan_kernel(WorkItem* items, UserRef* users,
                                                           MergeRef* merges,
                                                           const int32_t* __restrict__ lens, int n,
-                                                          int splits, int chunk) {
+                                                          int splits, int chunk, int max_blocks) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n * splits) return;
   const int i = idx / splits, s = idx % splits;
-  const int len = lens[i];
+  const int len = max(0, min(lens[i], max_blocks * kBlock));
   WorkItem it;
   it.table_row = i;
   it.tok_begin = s * chunk;
@@ -108,7 +111,7 @@ extern "C" apar_status apar_tree_decode_attention_static(
   const int n_items = n_threads * splits;
   static_plan_kernel<<<(n_items + 127) / 128, 128, 0, st>>>(
       (WorkItem*)(s + lay.items), (UserRef*)(s + lay.users), (MergeRef*)(s + lay.merges),
-      ctx_lens, n_threads, splits, chunk);
+      ctx_lens, n_threads, splits, chunk, max_blocks_per_thread);
   if (cudaGetLastError() != cudaSuccess) return APAR_ERR_CUDA;
 
   AttnArgs a;

@@ -247,8 +247,9 @@ __global__ void __launch_bounds__(128) attn_vec_kernel(const AttnArgs a, int ite
         const UserRef ur = a.d_users[it.user_begin + u];
         const int head = kvh * G + hg;
         if (ur.slot < 0) {
+          // an empty range (no tokens at all) has L = 0: its output is defined as zero
           ((__nv_bfloat16*)a.out)[((size_t)ur.query * HQ + head) * kDim + t] =
-              __float2bfloat16_rn(O / L);
+              __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
         } else {
           const size_t prow = (size_t)(ur.slot + it.slot_add) * HQ + head;
           a.part_o[prow * kDim + t] = O;
@@ -371,7 +372,7 @@ __global__ void __launch_bounds__(128) attn_vec_heads_kernel(const AttnArgs a, i
         m = mn;
       }
       if (ur.slot < 0 || it.fin_n > 0) {
-        const float inv = 1.f / l;
+        const float inv = l > 0.f ? 1.f / l : 0.f;      // no tokens at all: zeros
         __nv_bfloat162 p0 = __floats2bfloat162_rn(o[0] * inv, o[1] * inv);
         __nv_bfloat162 p1 = __floats2bfloat162_rn(o[2] * inv, o[3] * inv);
         __nv_bfloat162 p2 = __floats2bfloat162_rn(o[4] * inv, o[5] * inv);
@@ -502,7 +503,7 @@ __global__ void __launch_bounds__(128) merge_kernel(const AttnArgs a,
       acc.x += o[k].x * w; acc.y += o[k].y * w; acc.z += o[k].z * w; acc.w += o[k].w * w;
     }
   }
-  const float inv = 1.f / L;
+  const float inv = L > 0.f ? 1.f / L : 0.f;           // every part empty: zeros
   __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
   __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
   uint2 packed;

@@ -6,24 +6,53 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import MAX_ABS, MEAN_ABS
-from oracle import Forest, tree_decode_attention
+from helpers import MAX_ABS, MEAN_ABS, assert_same_bookkeeping
+from oracle import BlockModel, Forest, tree_decode_attention
 from paper_2401_06761_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
 
-# all threads of config 2, a fifth of config 3, a tenth of configs 4 and 5 (the checker does
-# 50-400 threads per second)
-@pytest.mark.parametrize("config,samples", [(2, 128), (3, 800), (4, 410), (5, 704)])
-def test_full_size_step_sampled(config, samples):
-    from paper_2401_06761_b200.session import PagedSession
+class WithModel:
+    """Replays every bookkeeping event on the integer pool model as well (ids must agree); the
+    rows themselves only go to the library - the attention checker regenerates them from seeds."""
+
+    def __init__(self, sess, model):
+        self.sess, self.model = sess, model
+
+    def new_threads(self, n):
+        a, b = self.sess.new_threads(n), self.model.new_threads(n)
+        assert a == b
+        return a
+
+    def fork(self, parents):
+        a, (b, _) = self.sess.fork(parents), self.model.fork(parents)
+        assert a == b
+        return a
+
+    def append(self, tids, counts, k, v):
+        self.sess.append(tids, counts, k, v)
+        self.model.append(tids, counts)
+
+
+# every thread of configs 1-3 (config 1 is covered in test_gpu_parity), a tenth of configs 4
+# and 5 (the checker does 50-400 threads per second)
+@pytest.mark.parametrize("config,samples", [(2, None), (3, None), (4, 410), (5, 704)])
+def test_full_size_step(config, samples):
+    from paper_2401_06761_b200.session import PagedSession, pool_requirements
     spec = synth.forest_spec(config)
     sess = PagedSession.for_spec(spec, extra_blocks=len(spec.nodes) + 64)
-    step = synth.build_forest(spec, sess, device="cuda")
-    synth.run_step_forks(step, sess)
+    _, nt, mb = pool_requirements(spec)
+    model = BlockModel(sess.num_blocks, 16, nt, mb)
+    both = WithModel(sess, model)
+    step = synth.build_forest(spec, both, device="cuda")
+    synth.run_step_forks(step, both)
     live = step.live_handles
-    sess.append(live, None, step.k_new, step.v_new)
+    both.append(live, None, step.k_new, step.v_new)
+    # tables, reference counts and free list of the whole pool, entry by entry
+    assert_same_bookkeeping(sess, model, list(model.tables))
+    assert sess.stats()["cow_blocks"] == model.cow_blocks
+    assert sess.stats()["peak_used_blocks"] == model.peak_used
     out = sess.attention(live, step.q)
     out2 = sess.attention(live, step.q)          # the cached plan gives the same answer
     torch.cuda.synchronize()
@@ -34,10 +63,14 @@ def test_full_size_step_sampled(config, samples):
     # every logical token once, plus the (at most 15) rows each fork copied for its child
     assert spec.unique_tokens() <= st["attn_unique_tokens"] <= spec.unique_tokens() + 15 * st["forks"]
     assert torch.isfinite(out.float()).all()
+    assert st["attn_unique_tokens"] == model.unique_tokens(live)
     nodes = step.live_nodes
     rng = np.random.default_rng(config)
-    idx = sorted(set(np.linspace(0, len(nodes) - 1, samples // 2).astype(int).tolist()) |
-                 set(rng.integers(0, len(nodes), samples // 2).tolist()))
+    if samples is None:
+        idx = list(range(len(nodes)))
+    else:
+        idx = sorted(set(np.linspace(0, len(nodes) - 1, samples // 2).astype(int).tolist()) |
+                     set(rng.integers(0, len(nodes), samples // 2).tolist()))
     errs = []
     for i in idx:
         k, v = synth.chain_kv(spec, nodes[i], "cuda")

@@ -32,6 +32,35 @@ def test_early_release_lowers_the_peak_in_the_pool_model():
 
 
 @pytest.mark.gpu
+def test_library_peak_counter_against_the_hand_worked_events():
+    """The library's max-cached counter against the values worked out by hand in
+    tests/golden/release_refork_peak.txt (not against the pool model)."""
+    from test_oracle_bookkeeping import load_golden, release_refork_events
+    from paper_2401_06761_b200.session import PagedSession
+    g = load_golden("release_refork_peak.txt")
+    sess = PagedSession(SHAPE, g["num_blocks"], 8, 16)
+    z = torch.zeros((64, 2, 128), dtype=torch.bfloat16, device="cuda")
+    in_use, peak = [], []
+    for ev in release_refork_events():
+        if ev[0] == "new+append":
+            (t,) = sess.new_threads(1)
+            sess.append([t], [ev[1]], z[:ev[1]], z[:ev[1]])
+        elif ev[0] == "fork":
+            sess.fork([ev[1]])
+        elif ev[0] == "append":
+            sess.append([ev[1]], [ev[2]], z[:ev[2]], z[:ev[2]])
+        else:
+            sess.release([ev[1]])
+        st = sess.stats()
+        in_use.append(st["used_blocks"])
+        peak.append(st["peak_used_blocks"])
+    assert in_use == g["in_use_after_event"] and peak == g["peak_after_event"]
+    for t, table in g["table"].items():
+        assert sess.thread(t) == (g["len"][t], table)
+    sess.close()
+
+
+@pytest.mark.gpu
 def test_lifecycle_replay_on_the_library_matches_the_model():
     from paper_2401_06761_b200.session import PagedSession
     steps, req = synth.lifecycle_schedule(seed=5, n_requests=24, n_steps=300)

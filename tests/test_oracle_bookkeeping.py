@@ -23,8 +23,8 @@ def load_golden(name):
             out[parts[0]][int(parts[1])] = vals if parts[0] == "table" else vals[0]
         elif parts[0] == "copies":
             out["copies"] = [tuple(int(x) for x in c.split()) for c in val.split(",") if c.strip()]
-        elif parts[0] == "refcount":
-            out["refcount"] = [int(x) for x in val.split()]
+        elif parts[0] in ("refcount", "in_use_after_event", "peak_after_event"):
+            out[parts[0]] = [int(x) for x in val.split()]
         else:
             out[parts[0]] = int(val)
     return out
@@ -55,6 +55,7 @@ def test_prompt64_hand_computed():
     slots = m.append(kids)
     assert slots == [[(5, 15)], [(10, 0)], [(9, 7)]]
     check_against_golden(m, g, copies)
+    assert m.peak_used == g["peak_used_blocks"] == 11
 
 
 def test_prompt70_hand_computed_copy_on_fork():
@@ -64,9 +65,38 @@ def test_prompt70_hand_computed_copy_on_fork():
     m.append([p], [70])
     kids, copies = m.fork([p, p, p])
     check_against_golden(m, g, copies)
+    assert m.peak_used == g["peak_used_blocks"] == 8
     assert m.cow_blocks == 3 and m.cow_rows == 18
     # parent keeps its own partial block and appends in place; children use their copies
     assert m.append([p] + kids) == [[(4, 6)], [(5, 6)], [(6, 6)], [(7, 6)]]
+
+
+def release_refork_events():
+    """The events of golden/release_refork_peak.txt as (method, arguments) on thread ids."""
+    return [("new+append", 40), ("fork", 0), ("append", 1, 30), ("release", 1), ("fork", 0),
+            ("append", 2, 9), ("append", 2, 17), ("append", 0, 1), ("append", 0, 24)]
+
+
+def test_peak_of_blocks_in_use_hand_computed():
+    g = load_golden("release_refork_peak.txt")
+    m = BlockModel(g["num_blocks"], g["block_size"], 8, 16)
+    in_use, peak = [], []
+    for ev in release_refork_events():
+        if ev[0] == "new+append":
+            (t,) = m.new_threads(1)
+            m.append([t], [ev[1]])
+        elif ev[0] == "fork":
+            m.fork([ev[1]])
+        elif ev[0] == "append":
+            m.append([ev[1]], [ev[2]])
+        else:
+            m.release([ev[1]])
+        in_use.append(m.used_blocks())
+        peak.append(m.peak_used)
+    assert in_use == g["in_use_after_event"]
+    assert peak == g["peak_after_event"]          # taking freed blocks again does not move it
+    for t, table in g["table"].items():
+        assert m.tables[t] == table and m.lens[t] == g["len"][t]
 
 
 def invariants(m):

@@ -27,3 +27,28 @@ def test_three_paragraph_response_restores_in_reading_order():
                            "r1a", FORK, "d1a", EOS, "r2a", "r2b", EOS]
     assert g.seqs[1].tokens[:6] == ["P0", "P1", "r0a", "r0b", FORK, CHILD]
     assert g.slices() == [(0, 2, 5), (1, 6, 10), (0, 5, 7), (2, 8, 10), (0, 7, 10)]
+
+
+def test_a_detail_thread_that_forks_again_is_read_depth_first():
+    # Worked by hand from Algorithm 1's traversal (root, first child, next sibling): the detail
+    # thread of the first paragraph forks itself, so its own detail comes before its remainder,
+    # and both come before the remainder of the root thread.
+    script = {0: ["a", FORK, "b", EOS], 1: ["c", FORK, "d", EOS], 2: ["e", EOS]}
+    g = SequenceGroup(["P"])
+    pos = {}
+
+    def sample(s):
+        i = g.seqs.index(s)
+        pos[i] = pos.get(i, 0) + 1
+        return script[i][pos[i] - 1]
+
+    passes = 0
+    while not all(s.finished for s in g.seqs):
+        g.step(sample)
+        passes += 1
+    assert passes == 8                      # a thread born in a pass first decodes in the next
+    assert g.seqs[0].tokens == ["P", "a", FORK, "b", EOS]
+    assert g.seqs[1].tokens == ["P", "a", FORK, CHILD, "c", FORK, "d", EOS]
+    assert g.seqs[2].tokens == ["P", "a", FORK, CHILD, "c", FORK, CHILD, "e", EOS]
+    assert g.slices() == [(0, 1, 3), (1, 4, 6), (2, 7, 9), (1, 6, 8), (0, 3, 5)]
+    assert g.restore() == ["a", FORK, "c", FORK, "e", EOS, "d", EOS, "b", EOS]

@@ -175,3 +175,18 @@ def test_few_long_threads_are_spread_over_the_machine():
     m2, live = random_forest(5, n_roots=3, steps=40)
     c2 = check_plan(m2, live, 32, 32, 2, True)
     assert c2["items"] <= 2 * c2["users"]
+
+
+@pytest.mark.parametrize("hq,hkv", [(65, 1), (71, 1), (128, 1), (256, 2)])
+def test_more_than_64_query_heads_per_kv_head_are_refused(hq, hkv):
+    """A work item carries every query head of a kv head for at least one thread, at most 64
+    rows: wider groups have no kernel and must be turned down before any planning."""
+    m = BlockModel(64, BS, 4, 16)
+    (t,) = m.new_threads(1)
+    m.append([t], [40])
+    tab, lens = tables_of(m, [t])
+    with pytest.raises(B.AparError) as e:
+        B.apar_debug_plan(m.num_blocks, hq, hkv, tab, lens, 2, True)
+    assert e.value.code == "UNSUPPORTED"
+    assert B.apar_workspace_bytes(B.make_config(64, hq, hkv, 4, 16)) == 0
+    B.apar_debug_plan(m.num_blocks, 64, 1, tab, lens, 2, True)        # the widest group allowed
