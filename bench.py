@@ -5,12 +5,21 @@ threads, for one attention layer.  Prints one JSON line.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl reference]
 
+The headline numbers (`value`, `roofline`, `e2e`) belong to `--workload` (default cfg4, the
+largest configuration by bytes).  With the default workload on one GPU the same line also
+carries, under `sweep`, the device-arm numbers of the other configurations (cfg1, cfg2, cfg3,
+cfg5 and cfg5 with every prefix copied instead of shared), the headline workload once more
+over a longer run (`sustained`: hundreds of steps, where the power cap sets the clock), and
+the early-release replay (`lifecycle`: most cached tokens at once when a finished thread
+gives its cache back at once, against at the end of its request).
+
 With N > 1 (under torchrun) every rank runs its own shard of requests (a different seed of the
 same workload) on its own GPU; there is no exchange between shards.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -28,6 +37,7 @@ from paper_2401_06761_b200 import sharding, synth  # noqa: E402
 
 METRIC = "tree decode-attention thread-tokens/s"
 UNIT = "thread-tokens/s"
+SWEEP = (("cfg1", False), ("cfg2", False), ("cfg3", False), ("cfg5", False), ("cfg5", True))
 
 
 def measured_peaks():
@@ -72,10 +82,12 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+                 "-lms", "20", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._read, daemon=True).start()
+            time.sleep(0.1)          # the first sample is on its way before the timed region
         except Exception:
             self.proc = None
+        return self
 
     def _read(self):
         for line in self.proc.stdout:
@@ -84,7 +96,7 @@ class ClockSampler:
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.1)
         self.proc.terminate()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
@@ -100,29 +112,65 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_mhz_min": min(sm) if sm else None,
                 "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
                 "samples": len(sm)}
 
 
 def parse_workload(name: str) -> int:
     if not (name.startswith("cfg") and name[3:].isdigit() and int(name[3:]) in synth.LAYER_SHAPES):
-        raise SystemExit(f"unknown workload {name}; use cfg1..cfg5")
+        raise SystemExit(f"unknown workload {name}; use cfg1..cfg5 or lifecycle")
     return int(name[3:])
 
 
+def workload_config(name, spec, unshared, layers=1, graph=False, world=1):
+    """The `config` object of the JSON line; both arms print the same one."""
+    shape = spec.shape
+    small = spec.unique_tokens() * shape.bytes_per_token < 4 * 126e6
+    has_fork = any(n.step_fork for n in spec.nodes)
+    return {
+        "workload": name + ("-unshared" if unshared else ""),
+        "threads_per_gpu": len(spec.live_nodes()),
+        "requests": len({n.request for n in spec.nodes}),
+        "num_q_heads": shape.num_q_heads, "num_kv_heads": shape.num_kv_heads,
+        "head_dim": shape.head_dim, "block_size": shape.block_size,
+        "step": ("fork+" if has_fork else "") + "append+attention, " +
+                ("one layer" if layers == 1 else f"{layers} layers (value counts thread-tokens "
+                                                 f"per layer)") +
+                (", layers 1.. replayed from a CUDA graph" if graph else ""),
+        "l2": "inputs larger than L2 (unique KV bytes per step >> 126 MB)" if not small else
+              "KV fits in L2: 256 MB written between steps, each step timed on its own "
+              "(device arm)",
+        "parallelism": f"{world} independent shard(s), no collective",
+    }
+
+
 # ------------------------------------------------------------------------------ CPU baseline
-def oracle_sample(spec, budget_s: float, min_threads: int = 2):
-    """Times the fp64 checker, as it stands, on live threads of `spec` until the budget is used.
-    Returns (thread-tokens per second, threads done, cores used)."""
+def _oracle_worker(job):
+    """One host core: times the fp64 checker, as it stands, on live threads of the workload
+    until the budget is used.  Runs in a process of its own; one BLAS thread."""
+    cfg_id, seed, n_requests, unshared, offset, stride, budget_s = job
     import numpy as np
-    from oracle import Forest, tree_decode_attention
+    try:
+        from threadpoolctl import threadpool_limits
+        threadpool_limits(1)
+    except Exception:
+        pass
     torch.set_num_threads(1)
+    from oracle import Forest, tree_decode_attention
+    spec = synth.forest_spec(cfg_id, seed=seed, n_requests=n_requests)
+    if unshared:
+        spec = synth.unshared_spec(spec)
     live = spec.live_nodes()
-    order = list(range(0, len(live), max(1, len(live) // 64))) + list(range(len(live)))
     scale = spec.shape.head_dim ** -0.5
     q_all = synth.queries(spec, len(live), "cpu").to(torch.float64).numpy()
     done, spent = 0, 0.0
-    for i in order:
+    # this worker's share: threads offset, offset + stride, ... of a walk that visits every
+    # region of the request range first
+    coarse = list(range(0, len(live), max(1, len(live) // 64)))
+    first = set(coarse)
+    order = coarse + [i for i in range(len(live)) if i not in first]
+    for i in order[offset::stride]:
         node = live[i]
         k, v = synth.chain_kv(spec, node, "cpu")          # input generation: not timed
         k, v = k.to(torch.float64).numpy(), v.to(torch.float64).numpy()
@@ -134,47 +182,327 @@ def oracle_sample(spec, budget_s: float, min_threads: int = 2):
         spent += time.perf_counter() - t0
         assert np.isfinite(out).all()
         done += 1
-        if spent >= budget_s and done >= min_threads:
+        if spent >= budget_s:
             break
-    return done / spent, done, 1
+    return done, spent
+
+
+class OraclePool:
+    """The checker on all host cores: one single-threaded process per core, each timing its own
+    share of the workload's live threads.  Rate = sum of the per-core rates, every core's rate
+    taken while all the others were busy as well."""
+
+    def __init__(self, max_cores=None):
+        import multiprocessing as mp
+        try:
+            avail = len(os.sched_getaffinity(0))
+        except AttributeError:
+            avail = os.cpu_count() or 1
+        self.cores = max(1, min(avail, max_cores or 32))
+        os.environ.setdefault("OMP_NUM_THREADS", "1")
+        os.environ.setdefault("MKL_NUM_THREADS", "1")
+        os.environ.setdefault("OPENBLAS_NUM_THREADS", "1")
+        self.pool = mp.get_context("spawn").Pool(self.cores)
+
+    def sample(self, cfg_id, seed, n_requests, unshared, budget_s):
+        """(thread-tokens per second over all cores, threads done, cores that did work)."""
+        jobs = [(cfg_id, seed, n_requests, unshared, w, self.cores, budget_s)
+                for w in range(self.cores)]
+        res = [r for r in self.pool.map(_oracle_worker, jobs) if r[0] > 0]
+        return sum(d / s for d, s in res), sum(d for d, _ in res), len(res)
+
+    def close(self):
+        self.pool.close()
+        self.pool.join()
 
 
 def run_reference(args, cfg_id):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    spec = synth.forest_spec(cfg_id)
-    # about a minute of timed oracle work over the whole run (input generation, untimed, takes
-    # about as long again)
+    spec = synth.forest_spec(cfg_id, n_requests=args.requests)
+    if args.unshared:
+        spec = synth.unshared_spec(spec)
+    # about a minute of timed checker work per core over the whole run (input generation,
+    # untimed, takes about as long again)
     per_step = max(0.5, min(20.0, 60.0 / max(1, args.steps + args.warmup)))
+    pool = OraclePool()
     for _ in range(args.warmup):
-        oracle_sample(spec, per_step / 4)
-    rates, threads = [], 0
+        pool.sample(cfg_id, spec.seed, args.requests, args.unshared, per_step / 4)
+    rates, threads, cores = [], 0, 0
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        r, n, cores = oracle_sample(spec, per_step)
+        r, n, cores = pool.sample(cfg_id, spec.seed, args.requests, args.unshared, per_step)
         rates.append(r); threads += n
     wall = time.perf_counter() - t0
+    pool.close()
     value = statistics.mean(rates)
-    sample = (f"{threads} live threads of {args.workload} over {args.steps} steps, one thread "
-              f"at a time: chain materialised in fp64 + dense softmax attention, all "
-              f"{spec.shape.num_q_heads} query heads")
+    sample = (f"{threads} live threads of {args.workload} over {args.steps} steps on {cores} host "
+              f"cores (one single-threaded process per core), one thread at a time: chain "
+              f"materialised in fp64 + dense softmax attention, all {spec.shape.num_q_heads} "
+              f"query heads")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wall / max(1, args.steps),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": args.workload},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+        "data": "synthetic",
+        "config": workload_config(args.workload, spec, args.unshared, max(1, args.layers),
+                                  args.graph, 1),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
+# ------------------------------------------------------------------------------ DRAM traffic
+def profiled_traffic(workload_key, requests_run):
+    """DRAM bytes (read + write) of the attention kernels of one call, from the ncu captures
+    summarised in profiles/dram_traffic.txt: taken on a small case of the same kernels and
+    scaled by the requests processed (DRAM traffic is proportional to them).  None when there
+    is no capture for the workload, or when a kernel source has changed since its capture
+    (the file records a digest of every source file)."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None, "no capture"
+    total, found = 0.0, False
+    for line in open(path):
+        f = line.split()
+        if len(f) < 7 or f[0].startswith("#") or f[0] != workload_key:
+            continue
+        _, kernel, source, digest, req, rd_mb, wr_mb = f[:7]
+        src = os.path.join(ROOT, "paper_2401_06761_b200", "csrc", source)
+        if not os.path.exists(src) or hashlib.sha256(open(src, "rb").read()).hexdigest()[:16] != digest:
+            return None, f"{source} changed since the capture"
+        total += (float(rd_mb) + float(wr_mb)) * 1e6 * requests_run / float(req)
+        found = True
+    return (total, "profiles/dram_traffic.txt, scaled by requests") if found else (None, "no capture")
+
+
 # ------------------------------------------------------------------------------ GPU arm
-def run_ours(args, cfg_id):
+class DeviceRun:
+    """One workload on this rank's GPU: builds the forest through the library, runs steps."""
+
+    def __init__(self, name, cfg_id, unshared, args, dev, rank, steps_total, layers=1):
+        from paper_2401_06761_b200 import binding as B
+        from paper_2401_06761_b200.session import pool_requirements
+        self.B, self.name, self.cfg_id, self.unshared, self.dev = B, name, cfg_id, unshared, dev
+        spec = sharding.shard_spec(cfg_id, rank, n_requests=args.requests)
+        if unshared:
+            spec = synth.unshared_spec(spec)
+        self.spec, self.shape, self.L = spec, spec.shape, layers
+        nb, nt, mb = pool_requirements(spec)
+        self.T = len(spec.live_nodes())
+        self.n_step_forks = sum(1 for n in spec.nodes if n.step_fork)
+        grow = (self.T + self.n_step_forks) * (2 * steps_total // 16 + 2) + 2 * self.n_step_forks
+        self.dims = (nb + grow, nt + self.n_step_forks, mb + 2 * steps_total // 16 + 2)
+        self.sess = self.step0 = self.graph = None
+        self.setup_s = 0.0
+        self.attn_events = []
+        g = torch.Generator(device=dev).manual_seed(spec.seed + 99)
+        self.row_shape = (self.T, self.shape.num_kv_heads, self.shape.head_dim)
+        self.q_shape = (self.T, self.shape.num_q_heads, self.shape.head_dim)
+        self.inputs = [tuple(torch.randn(s, generator=g, device=dev).to(torch.bfloat16)
+                             for s in (self.q_shape, self.row_shape, self.row_shape))
+                       for _ in range(min(4, steps_total))]
+        self.out = torch.empty(self.q_shape, dtype=torch.bfloat16, device=dev)
+        self.stream = torch.cuda.current_stream().cuda_stream
+        self.small = spec.unique_tokens() * self.shape.bytes_per_token < 4 * 126e6
+
+    def make_session(self):
+        from paper_2401_06761_b200.session import PagedSession
+        self.close()
+        t0 = time.perf_counter()
+        self.sess = PagedSession(self.shape, *self.dims, device=self.dev, num_layers=self.L)
+        self.step0 = synth.build_forest(self.spec, self.sess, device=self.dev)
+        if self.L > 1:      # give the other layers the same rows as layer 0 (setup, untimed)
+            for pool in (self.sess.k_pool, self.sess.v_pool):
+                per = pool.shape[0] // self.L
+                for l in range(1, self.L):
+                    pool[l * per:(l + 1) * per].copy_(pool[:per])
+        torch.cuda.synchronize()
+        self.setup_s = time.perf_counter() - t0
+        self.base_live = [h for h, n in zip(self.step0.live_handles, self.step0.live_nodes)
+                          if not n.step_fork]
+        self.base_live_arr = self.B.int32_array(self.base_live)
+        self.attn_events = []
+
+    def close(self):
+        if self.sess is not None:
+            self.sess.close()
+            self.sess = self.step0 = self.graph = None
+            torch.cuda.empty_cache()
+
+    def one_step(self, q, k_new, v_new, record, stream=None, out=None):
+        """fork (if the workload has one) + append + attention [+ release of the step's forks]."""
+        B, sess, step0 = self.B, self.sess, self.step0
+        stream = self.stream if stream is None else stream
+        out = self.out if out is None else out
+        kids = B.apar_fork(sess.ctx, step0.fork_parents, stream) if step0.fork_parents else []
+        live = B.int32_array(self.base_live + kids) if kids else self.base_live_arr
+        B.apar_append_kv(sess.ctx, live, None, k_new.data_ptr(), v_new.data_ptr(), stream)
+        if record:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        B.apar_tree_decode_attention(sess.ctx, live, q.data_ptr(), out.data_ptr(), sess.sm_scale,
+                                     stream)
+        if record:
+            e1.record()
+            self.attn_events.append((e0, e1))
+        if self.graph is not None:        # the other layers, replayed from the captured graph
+            if (q.data_ptr(), k_new.data_ptr(), out.data_ptr()) != self.graph_ptrs:
+                for dst, src in zip(self.graph_in, (q, k_new, v_new)):
+                    dst.copy_(src)
+            self.graph.replay()
+        else:
+            for l in range(1, self.L):      # the other layers: scatter + attention launches only
+                B.apar_append_kv_layer(sess.ctx, l, k_new.data_ptr(), v_new.data_ptr(), stream)
+                B.apar_tree_decode_attention_layer(sess.ctx, l, q.data_ptr(), out.data_ptr(),
+                                                   sess.sm_scale, stream)
+        if kids:
+            B.apar_release(sess.ctx, kids)
+
+    def capture_layer_loop(self):
+        """Layers 1.. of a step only launch kernels whose sizes the cached plan fixes: capture
+        them once; valid while the plan is reused (threads only grow)."""
+        B = self.B
+        self.graph_in = [torch.empty_like(t) for t in self.inputs[0]]
+        for dst, src in zip(self.graph_in, self.inputs[0]):
+            dst.copy_(src)
+        gq, gk, gv = self.graph_in
+        self.graph_ptrs = (gq.data_ptr(), gk.data_ptr(), self.out.data_ptr())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            cs = torch.cuda.current_stream().cuda_stream
+            for l in range(1, self.L):
+                B.apar_append_kv_layer(self.sess.ctx, l, gk.data_ptr(), gv.data_ptr(), cs)
+                B.apar_tree_decode_attention_layer(self.sess.ctx, l, gq.data_ptr(),
+                                                   self.out.data_ptr(), self.sess.sm_scale, cs)
+        self.graph = graph
+
+    def timed_device_arm(self, steps, warmup, sync, reduce_ms, clock_index=None, graph=False):
+        """`warmup` untimed steps, then exactly `steps` timed ones.  Returns a dict of raw
+        results of this rank (times already reduced over ranks by `reduce_ms`)."""
+        inputs = self.inputs
+        for i in range(warmup):
+            self.one_step(*inputs[i % len(inputs)], record=False)
+        sync()
+        if graph:
+            self.capture_layer_loop()
+            self.one_step(*inputs[0], record=False)
+            sync()
+        k0 = self.sess.stats()["kernels_total"]
+        sampler = ClockSampler(clock_index).start() if clock_index is not None else None
+        self.attn_events = []
+        host_t0 = time.perf_counter()
+        # A workload whose KV fits in the L2 cache would be timed on cache hits: for those,
+        # every step is timed on its own and a buffer larger than L2 is written between steps.
+        if self.small:
+            flush = torch.empty(256 << 20, dtype=torch.uint8, device=self.dev)
+            step_events = []
+            for i in range(steps):
+                flush.fill_(i & 0xff)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                self.one_step(*inputs[i % len(inputs)], record=True)
+                b.record()
+                step_events.append((a, b))
+            host_ms = 1e3 * (time.perf_counter() - host_t0)
+            sync()
+            total_ms = reduce_ms(sum(a.elapsed_time(b) for a, b in step_events))
+            del flush
+        else:
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            for i in range(steps):
+                self.one_step(*inputs[i % len(inputs)], record=True)
+            ev1.record()
+            host_ms = 1e3 * (time.perf_counter() - host_t0)
+            sync()
+            total_ms = reduce_ms(ev0.elapsed_time(ev1))
+        clocks = sampler.stop() if sampler is not None else None
+        st = self.sess.stats()
+        if st["device_wait_timeouts"]:
+            raise SystemExit(f"a kernel gave up a bounded wait (code {st['device_wait_timeouts']}): "
+                             "the timed results are invalid")
+        attn = sorted(a.elapsed_time(b) for a, b in self.attn_events)
+        return {"total_ms": total_ms, "host_issue_ms": host_ms, "clocks": clocks, "stats": st,
+                "launches": st["kernels_total"] - k0, "attn_ms": statistics.mean(attn),
+                "attn_ms_median": attn[len(attn) // 2], "attn_ms_min": attn[0], "steps": steps}
+
+    def summary(self, r, peak):
+        """Throughput, byte counts and roofline figures of one timed device arm."""
+        st, steps, shape = r["stats"], r["steps"], self.shape
+        bpt = shape.bytes_per_token
+        # every persistent thread grows by one token per step: the counters of the last timed
+        # step are brought back to their mean over the timed steps
+        grow = len(self.base_live) * (steps - 1) / 2.0
+        unique_tokens = st["attn_unique_tokens"] - grow
+        attended_tokens = st["attn_attended_tokens"] - grow
+        unique_bytes, unshared_bytes = unique_tokens * bpt, attended_tokens * bpt
+        qo_bytes = 2 * self.T * shape.num_q_heads * shape.head_dim * 2
+        algo_bytes = unique_bytes + qo_bytes
+        achieved = algo_bytes / (r["attn_ms"] * 1e-3) / 1e9
+        return {
+            "threads": self.T, "steps": steps, "ms_per_step": r["total_ms"] / steps,
+            "thread_tokens_per_s": self.T * self.L * steps / (r["total_ms"] * 1e-3),
+            "attention_ms": r["attn_ms"], "attention_ms_median": r["attn_ms_median"],
+            "attention_ms_min": r["attn_ms_min"],
+            "unique_kv_bytes_per_step": unique_bytes, "unshared_kv_bytes_per_step": unshared_bytes,
+            "sharing_ratio": unshared_bytes / max(1.0, unique_bytes),
+            "unique_tokens": unique_tokens, "attended_tokens": attended_tokens,
+            "algorithmic_bytes": algo_bytes, "achieved_gbs": achieved,
+            "frac_of_measured_peak": achieved / peak,
+            "unique_kv_frac_of_nominal": unique_bytes / (r["attn_ms"] * 1e-3) / 1e9 / 8000.0,
+            "host_issue_ms_per_step": r["host_issue_ms"] / steps,
+            "gpu_launches": r["launches"], "clocks": r["clocks"],
+            "l2": "flushed between steps" if self.small else "inputs larger than L2",
+        }
+
+
+def lifecycle_report(dev, n_requests=96, n_steps=1500, max_live=96):
+    """Early release as a measurement (Section 2.4 feature 2; "max cached tokens", Section 3.4):
+    a seeded stream of requests whose threads fork and finish at different steps is replayed
+    through the library twice, once giving a finished thread's cache back at once and once only
+    when its whole request has finished.  Both peaks are the library's own counter."""
+    from paper_2401_06761_b200.session import PagedSession
+    shape = synth.LAYER_SHAPES[1]
+    steps, req = synth.lifecycle_schedule(seed=7, n_requests=n_requests, n_steps=n_steps,
+                                          max_live=max_live)
+    z = torch.zeros((4096, shape.num_kv_heads, shape.head_dim), dtype=torch.bfloat16, device=dev)
+    q = torch.zeros((max_live + 8, shape.num_q_heads, shape.head_dim), dtype=torch.bfloat16,
+                    device=dev)
+    rep = {"requests": n_requests, "steps": n_steps, "max_live_threads": max_live,
+           "threads": len(req), "forks": sum(len(s.fork) for s in steps)}
+    for early in (True, False):
+        sess = PagedSession(shape, 16384, len(req) + 8, 64, device=dev)
+        tokens = [0]
+
+        def rows(n):
+            return z[:n], z[:n]
+
+        def on_step(i, live):
+            tokens[0] += len(live)
+            sess.attention(live, q[:len(live)])
+
+        t0 = time.perf_counter()
+        synth.run_lifecycle(steps, req, sess, rows, early_release=early, on_step=on_step)
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - t0
+        st = sess.stats()
+        assert st["free_blocks"] == 16384 and st["device_wait_timeouts"] == 0
+        key = "early_release" if early else "release_at_request_end"
+        rep[key] = {"peak_cached_tokens": 16 * st["peak_used_blocks"],
+                    "peak_used_blocks": st["peak_used_blocks"],
+                    "thread_tokens": tokens[0], "wall_s": wall}
+        sess.close()
+    rep["peak_saving"] = 1.0 - (rep["early_release"]["peak_cached_tokens"] /
+                                rep["release_at_request_end"]["peak_cached_tokens"])
+    return rep
+
+
+def run_ours(args):
     from paper_2401_06761_b200 import build
     build.build()
-    from paper_2401_06761_b200.session import PagedSession, pool_requirements
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -188,162 +516,43 @@ def run_ours(args, cfg_id):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    # shard = the same workload with a rank-specific seed: independent requests, no exchange
-    spec = sharding.shard_spec(cfg_id, rank, n_requests=args.requests)
-    if args.unshared:
-        spec = synth.unshared_spec(spec)
-    shape = spec.shape
-    steps_total = args.warmup + args.steps
-    nb, nt, mb = pool_requirements(spec)
-    n_live = len(spec.live_nodes())
-    n_step_forks = sum(1 for n in spec.nodes if n.step_fork)
-    grow_blocks = (n_live + n_step_forks) * (2 * steps_total // 16 + 2) + 2 * n_step_forks
-    L = max(1, args.layers)
-    from paper_2401_06761_b200 import binding as B
-
-    class S:      # the session in use: the end-to-end arm rebuilds it, see below
-        sess = step0 = base_live = base_live_arr = None
-        setup_s = 0.0
-        graph = graph_in = graph_ptrs = None
-
-    def make_session():
-        if S.sess is not None:
-            S.sess.close()
-            S.sess = S.step0 = S.graph = None
-            torch.cuda.empty_cache()
-        t0 = time.perf_counter()
-        S.sess = PagedSession(shape, nb + grow_blocks, nt + n_step_forks,
-                              mb + 2 * steps_total // 16 + 2, device=dev, num_layers=L)
-        S.step0 = synth.build_forest(spec, S.sess, device=dev)
-        if L > 1:      # give the other layers the same rows as layer 0 (setup, untimed)
-            for pool in (S.sess.k_pool, S.sess.v_pool):
-                per = pool.shape[0] // L
-                for l in range(1, L):
-                    pool[l * per:(l + 1) * per].copy_(pool[:per])
-        torch.cuda.synchronize()
-        S.setup_s = time.perf_counter() - t0
-        S.base_live = [h for h, n in zip(S.step0.live_handles, S.step0.live_nodes)
-                       if not n.step_fork]
-        S.base_live_arr = B.int32_array(S.base_live)
-
-    make_session()
-    t_setup = S.setup_s
-    stream = torch.cuda.current_stream().cuda_stream
-    T = n_live
-    g = torch.Generator(device=dev).manual_seed(spec.seed + 99)
-    row_shape = (T, shape.num_kv_heads, shape.head_dim)
-    q_shape = (T, shape.num_q_heads, shape.head_dim)
-
-    def fresh(shp):
-        return torch.randn(shp, generator=g, device=dev).to(torch.bfloat16)
-
-    out = torch.empty(q_shape, dtype=torch.bfloat16, device=dev)
-    attn_events = []
-
-    def one_step(q, k_new, v_new, record, stream=stream, out=out):
-        """fork (if the workload has one) + append + attention [+ release of the step's forks]."""
-        sess, step0 = S.sess, S.step0
-        kids = B.apar_fork(sess.ctx, step0.fork_parents, stream) if step0.fork_parents else []
-        live = B.int32_array(S.base_live + kids) if kids else S.base_live_arr
-        B.apar_append_kv(sess.ctx, live, None, k_new.data_ptr(), v_new.data_ptr(), stream)
-        if record:
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-        B.apar_tree_decode_attention(sess.ctx, live, q.data_ptr(), out.data_ptr(), sess.sm_scale,
-                                     stream)
-        if record:
-            e1.record()
-            attn_events.append((e0, e1))
-        if S.graph is not None:        # the other layers, replayed from the captured graph
-            if (q.data_ptr(), k_new.data_ptr(), out.data_ptr()) != S.graph_ptrs:
-                S.graph_in[0].copy_(q); S.graph_in[1].copy_(k_new); S.graph_in[2].copy_(v_new)
-            S.graph.replay()
-        else:
-            for l in range(1, L):      # the other layers: scatter + attention launches only
-                B.apar_append_kv_layer(sess.ctx, l, k_new.data_ptr(), v_new.data_ptr(), stream)
-                B.apar_tree_decode_attention_layer(sess.ctx, l, q.data_ptr(), out.data_ptr(),
-                                                   sess.sm_scale, stream)
-        if kids:
-            B.apar_release(sess.ctx, kids)
-
-    def barrier():
+    def sync():
         torch.cuda.synchronize()
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(ms):
+    def reduce_ms(ms):
         return sharding.reduce_timing(ms, 0.0, dist, dev)[0]
 
+    peak, peak_kind = measured_peaks()
+    if args.workload == "lifecycle":
+        if rank == 0:
+            rep = lifecycle_report(dev)
+            e = rep["early_release"]
+            print(json.dumps({
+                "metric": METRIC, "value": e["thread_tokens"] / e["wall_s"], "unit": UNIT,
+                "n_gpus": 1, "steps": rep["steps"], "warmup": 0,
+                "ms_per_step": 1e3 * e["wall_s"] / rep["steps"], "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "lifecycle"}, "lifecycle": rep}))
+        return
+    cfg_id = parse_workload(args.workload)
+    L = max(1, args.layers)
+    steps_total = args.warmup + args.steps
+    run = DeviceRun(args.workload, cfg_id, args.unshared, args, dev, rank, steps_total, L)
+    if args.graph and (L < 2 or any(n.step_fork for n in run.spec.nodes)):
+        raise SystemExit("--graph needs --layers >= 2 and a workload without forks in the step")
+
     # ---------------- device-resident arm
-    inputs = [(fresh(q_shape), fresh(row_shape), fresh(row_shape)) for _ in range(min(4, steps_total))]
-    for i in range(args.warmup):
-        one_step(*inputs[i % len(inputs)], record=False)
-    barrier()
-
-    def capture_layer_loop(out_buf):
-        """Layers 1.. of a step only launch kernels whose sizes the cached plan fixes: capture
-        them once; valid while the plan is reused (threads only grow)."""
-        S.graph_in = [torch.empty_like(inputs[0][0]), torch.empty_like(inputs[0][1]),
-                      torch.empty_like(inputs[0][2])]
-        for dst, src in zip(S.graph_in, inputs[0]):
-            dst.copy_(src)
-        gq, gk, gv = S.graph_in
-        S.graph_ptrs = (gq.data_ptr(), gk.data_ptr(), out_buf.data_ptr())
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            cs = torch.cuda.current_stream().cuda_stream
-            for l in range(1, L):
-                B.apar_append_kv_layer(S.sess.ctx, l, gk.data_ptr(), gv.data_ptr(), cs)
-                B.apar_tree_decode_attention_layer(S.sess.ctx, l, gq.data_ptr(), out_buf.data_ptr(),
-                                                   S.sess.sm_scale, cs)
-        S.graph = graph
-
-    if args.graph:
-        if L < 2 or S.step0.fork_parents:
-            raise SystemExit("--graph needs --layers >= 2 and a workload without forks in the step")
-        capture_layer_loop(out)
-        one_step(*inputs[0], record=False)
-        barrier()
-    k0 = S.sess.stats()["kernels_total"]
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    host_t0 = time.perf_counter()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    # A workload whose KV fits in the L2 cache would be timed on cache hits: for those, every
-    # step is timed on its own and a buffer larger than L2 is written between the steps.
-    small = spec.unique_tokens() * shape.bytes_per_token < 4 * 126e6
-    if small:
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-        step_events = []
-        for i in range(args.steps):
-            flush.fill_(i & 0xff)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            one_step(*inputs[i % len(inputs)], record=True)
-            b.record()
-            step_events.append((a, b))
-        host_issue_ms = 1e3 * (time.perf_counter() - host_t0)
-        barrier()
-        total_ms = max_over_ranks(sum(a.elapsed_time(b) for a, b in step_events))
-        del flush
-    else:
-        ev0.record()
-        for i in range(args.steps):
-            one_step(*inputs[i % len(inputs)], record=True)
-        ev1.record()
-        host_issue_ms = 1e3 * (time.perf_counter() - host_t0)
-        barrier()
-        total_ms = max_over_ranks(ev0.elapsed_time(ev1))
-    clocks = sampler.stop() if rank == 0 else None
-    launches = S.sess.stats()["kernels_total"] - k0
-    attn_ms = statistics.mean(a.elapsed_time(b) for a, b in attn_events)
-    st = S.sess.stats()
-    n_base_live, has_fork = len(S.base_live), bool(S.step0.fork_parents)
-    if st["device_wait_timeouts"]:
-        raise SystemExit(f"a kernel gave up a bounded wait (code {st['device_wait_timeouts']}): "
-                         "the timed results are invalid")
+    run.make_session()
+    t_setup = run.setup_s
+    r = run.timed_device_arm(args.steps, args.warmup, sync, reduce_ms,
+                             clock_index=local if rank == 0 else None, graph=args.graph)
+    head = run.summary(r, peak)
+    T, shape = run.T, run.shape
+    q_shape, row_shape = run.q_shape, run.row_shape
+    out, inputs = run.out, run.inputs
 
     # ---------------- end-to-end arm: host buffers in, host buffer out, copies inside the timing
     hq = [torch.empty(q_shape, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
@@ -379,7 +588,7 @@ def run_ours(args, cfg_id):
         s_cmp.wait_event(ev_in[b])
         if i >= 2:
             s_cmp.wait_event(ev_out[b])             # the result of step i-2 has left dout[b]
-        one_step(dq[b], dk[b], dv[b], record=False, out=dout[b])
+        run.one_step(dq[b], dk[b], dv[b], record=False, out=dout[b])
         ev_cmp[b].record(s_cmp)
         with torch.cuda.stream(s_out):
             s_out.wait_event(ev_cmp[b])
@@ -389,11 +598,12 @@ def run_ours(args, cfg_id):
     # The end-to-end arm starts from the same forest as the device arm did (every step makes
     # each thread one token longer, so carrying on would time a larger problem): rebuild it,
     # then the same number of warm-up steps, untimed.
-    make_session()
+    run.make_session()
     e2e_steps = args.steps
     for i in range(args.warmup):
         e2e_step(i)
-    barrier()
+    sync()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     for i in range(e2e_steps):
         e2e_step(i)
@@ -401,8 +611,8 @@ def run_ours(args, cfg_id):
     if e2e_steps >= 2:
         s_cmp.wait_event(ev_out[e2e_steps % 2])
     ev1.record()
-    barrier()
-    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1))
+    sync()
+    e2e_ms = reduce_ms(ev0.elapsed_time(ev1))
     h2d = sum(t[0].numel() * 2 for t in (dq, dk, dv))
     d2h = out.numel() * 2
 
@@ -422,56 +632,53 @@ def run_ours(args, cfg_id):
         copies_only()
     torch.cuda.synchronize()
     copy_ms = 1e3 * (time.perf_counter() - t_c) / reps
+    run.close()
+    del hq, hk, hv, hout, dq, dk, dv, dout
+
+    # ---------------- the rest of the contract: longer run, other workloads, early release
+    extras = {}
+    default_line = (world == 1 and not args.no_sweep and args.workload == "cfg4" and
+                    not args.unshared and args.requests is None and L == 1)
+    if default_line:
+        n_sus = args.sustained_steps
+        sus = DeviceRun(args.workload, cfg_id, False, args, dev, rank, n_sus + args.warmup, 1)
+        sus.make_session()
+        extras["sustained"] = sus.summary(
+            sus.timed_device_arm(n_sus, args.warmup, sync, reduce_ms, clock_index=local), peak)
+        sus.close()
+        del sus
+        sweep = {}
+        for name, unshared in SWEEP:
+            n_sw = max(30, args.sweep_steps)
+            w = DeviceRun(name, parse_workload(name), unshared, args, dev, rank,
+                          n_sw + args.warmup, 1)
+            w.make_session()
+            sweep[name + ("-unshared" if unshared else "")] = w.summary(
+                w.timed_device_arm(n_sw, args.warmup, sync, reduce_ms, clock_index=local), peak)
+            w.close()
+            del w
+        extras["sweep"] = sweep
+        extras["lifecycle"] = lifecycle_report(dev)
 
     # ---------------- numbers
     total_T = sharding.reduce_timing(0.0, float(T), dist, dev)[1]
-    value = total_T * L * args.steps / (total_ms * 1e-3)
+    value = total_T * L * args.steps / (r["total_ms"] * 1e-3)
     e2e_value = total_T * L * e2e_steps / (e2e_ms * 1e-3)
-    bpt = shape.bytes_per_token
-    # every persistent thread grows by one token per step: the counters of the last timed step
-    # are brought back to their mean over the timed steps
-    grow = n_base_live * (args.steps - 1) / 2.0
-    unique_tokens = st["attn_unique_tokens"] - grow
-    attended_tokens = st["attn_attended_tokens"] - grow
-    unique_bytes = unique_tokens * bpt
-    unshared_bytes = attended_tokens * bpt
-    qo_bytes = 2 * T * shape.num_q_heads * shape.head_dim * 2
-    algo_bytes = unique_bytes + qo_bytes
-    peak, peak_kind = measured_peaks()
-    achieved = algo_bytes / (attn_ms * 1e-3) / 1e9
-    attn_all = sorted(a.elapsed_time(b) for a, b in attn_events)
     read_peak = read_only_rate(dev) if rank == 0 else None
-    # DRAM bytes (read + write) of the attention kernels of one call, from the ncu captures
-    # summarised under profiles/ (taken on a 64-request case of the same kernels and scaled by
-    # the requests processed; DRAM traffic is proportional to them).  Only for the full cfg4.
-    traffic = None
-    if cfg_id == 4 and args.requests is None and not args.unshared and L == 1:
-        traffic = ((546.5 + 30.8) + (735.6 + 12.8)) * 1e6 * (512 / 64)
+    traffic, traffic_src = (None, "not the profiled workload")
+    if L == 1 and world == 1:
+        traffic, traffic_src = profiled_traffic(
+            args.workload + ("-unshared" if args.unshared else ""),
+            len({n.request for n in run.spec.nodes}))
 
     if rank == 0:
-        cpu_rate, cpu_threads, cores = (oracle_sample(spec, 12.0)
-                                        if world == 1 and not args.skip_cpu_baseline
-                                        else (None, 0, 0))
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+            "warmup": args.warmup, "ms_per_step": r["total_ms"] / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": {
-                "workload": args.workload + ("-unshared" if args.unshared else ""),
-                "threads_per_gpu": T, "requests": args.requests or synth.DEFAULT_REQUESTS[cfg_id],
-                "num_q_heads": shape.num_q_heads, "num_kv_heads": shape.num_kv_heads,
-                "head_dim": shape.head_dim, "block_size": shape.block_size,
-                "step": ("fork+" if has_fork else "") + "append+attention, " +
-                        ("one layer" if L == 1 else f"{L} layers (value counts thread-tokens "
-                                                    f"per layer)") +
-                        (", layers 1.. replayed from a CUDA graph" if args.graph else ""),
-                "l2": "inputs larger than L2 (unique KV bytes per step >> 126 MB)"
-                      if not small else "KV fits in L2: 256 MB written between steps, each step "
-                                        "timed on its own (device arm)",
-                "parallelism": f"{world} independent shard(s), no collective",
-            },
-            "clocks": clocks,
+            "config": workload_config(args.workload, run.spec, args.unshared, L, args.graph, world),
+            "clocks": r["clocks"],
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                     "ms_per_step": e2e_ms / e2e_steps,
@@ -479,38 +686,50 @@ def run_ours(args, cfg_id):
                     # end-to-end step is bound by them whenever they take longer than the compute
                     "copies_only_ms": copy_ms,
                     "copies_only_gbs": (h2d + d2h) / (copy_ms * 1e-3) / 1e9},
-            "gpu_launches": launches,
+            "gpu_launches": r["launches"],
             "roofline": {
-                "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": traffic,
+                "bound": "hbm", "achieved": head["achieved_gbs"], "peak": peak, "unit": "GB/s",
+                "frac": head["achieved_gbs"] / peak, "traffic": traffic,
+                "traffic_source": traffic_src,
                 "peak_kind": f"of {peak_kind} copy bandwidth",
                 # the same achieved rate against two other ceilings: this library's read-only
                 # streaming probe, run just now on this GPU, and the nominal HBM3e figure
-                "peak_read_only": read_peak, "frac_of_read_only": achieved / read_peak,
-                "peak_nominal": 8000.0, "frac_of_nominal": achieved / 8000.0,
-                "attention_ms_median": attn_all[len(attn_all) // 2],
-                "attention_ms_min": attn_all[0],
+                "peak_read_only": read_peak,
+                "frac_of_read_only": head["achieved_gbs"] / read_peak,
+                "peak_nominal": 8000.0, "frac_of_nominal": head["achieved_gbs"] / 8000.0,
+                "unique_kv_frac_of_nominal": head["unique_kv_frac_of_nominal"],
+                "attention_ms_median": head["attention_ms_median"],
+                "attention_ms_min": head["attention_ms_min"],
                 "kernel": "apar_tree_decode_attention call (table sync + attention + merge launches)",
-                "algorithmic_bytes": algo_bytes, "attention_ms": attn_ms,
+                "algorithmic_bytes": head["algorithmic_bytes"], "attention_ms": head["attention_ms"],
             },
-            "kv_bytes": {"unique_per_step": unique_bytes, "unshared_per_step": unshared_bytes,
-                         "sharing_ratio": unshared_bytes / max(1, unique_bytes),
-                         "attended_tokens_per_thread": attended_tokens / T,
-                         "unique_tokens": unique_tokens,
+            "kv_bytes": {"unique_per_step": head["unique_kv_bytes_per_step"],
+                         "unshared_per_step": head["unshared_kv_bytes_per_step"],
+                         "sharing_ratio": head["sharing_ratio"],
+                         "attended_tokens_per_thread": head["attended_tokens"] / T,
+                         "unique_tokens": head["unique_tokens"],
                          "note": "means over the timed steps (threads grow one token per step)"},
-            "plan": {"work_items": st["attn_work_items"], "vec_items": st["attn_vec_items"],
-                     "mma_items": st["attn_mma_items"], "partials": st["attn_partials"],
-                     "reused_last_step": st["attn_plan_reused"],
-                     "host_issue_ms_per_step": host_issue_ms / args.steps},
+            "plan": {"work_items": r["stats"]["attn_work_items"],
+                     "vec_items": r["stats"]["attn_vec_items"],
+                     "mma_items": r["stats"]["attn_mma_items"],
+                     "partials": r["stats"]["attn_partials"],
+                     "reused_last_step": r["stats"]["attn_plan_reused"],
+                     "host_issue_ms_per_step": head["host_issue_ms_per_step"]},
             "setup_s": t_setup,
         }
-        if cpu_rate is not None:
+        line.update(extras)
+        if world == 1 and not args.skip_cpu_baseline:
+            pool = OraclePool()
+            cpu_rate, cpu_threads, cores = pool.sample(cfg_id, run.spec.seed, args.requests,
+                                                       args.unshared, 10.0)
+            pool.close()
             line["cpu_baseline"] = {
                 "value": cpu_rate, "unit": UNIT, "cores": cores, "kind": "oracle",
-                "sample": f"{cpu_threads} live threads of {args.workload}, one at a time "
-                          f"(fp64 chain materialisation + dense attention, all query heads)"}
+                "sample": f"{cpu_threads} live threads of {args.workload} on {cores} host cores "
+                          f"(one single-threaded process per core, about 10 s of checker time "
+                          f"each), one thread at a time: fp64 chain materialisation + dense "
+                          f"attention, all query heads"}
         print(json.dumps(line))
-    S.sess.close()
     if dist is not None:
         dist.destroy_process_group()
 
@@ -518,13 +737,19 @@ def run_ours(args, cfg_id):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--requests", type=int, default=None,
                     help="shrink the workload to this many requests (profiling captures)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="only the headline workload: no sustained run, no other configurations")
+    ap.add_argument("--sustained-steps", type=int, default=300,
+                    help="steps of the longer run of the headline workload (default line only)")
+    ap.add_argument("--sweep-steps", type=int, default=50,
+                    help="timed steps of each of the other configurations (at least 30)")
     ap.add_argument("--unshared", action="store_true",
                     help="same live threads, but every thread owns a private copy of its whole "
                          "chain (the copy-the-prefix-on-fork policy); for comparison with the tree")
@@ -535,11 +760,10 @@ def main():
                     help="attention layers per step (layers > 0 replay the plan; default 1)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    cfg_id = parse_workload(args.workload)
     if args.impl == "reference":
-        run_reference(args, cfg_id)
+        run_reference(args, parse_workload(args.workload))
     else:
-        run_ours(args, cfg_id)
+        run_ours(args)
 
 
 if __name__ == "__main__":

@@ -25,7 +25,11 @@
  *     its pinned, mapped staging buffers by kernels on `cuda_stream`, not by a copy engine,
  *     so they never wait behind the caller's host-to-device copies on other streams.
  *   - Batched calls process their entries in index order and are all-or-nothing: on any
- *     error no host state changes and nothing is launched.
+ *     error other than APAR_ERR_CUDA no host state changes and nothing is launched.
+ *     APAR_ERR_CUDA means a CUDA runtime call (an event wait, a launch) failed part-way
+ *     through a call: the host tables may then already describe rows or forks whose kernels
+ *     were never enqueued.  Such errors are sticky in the CUDA runtime; the context must not
+ *     be used further except for apar_last_cuda_error and apar_destroy.
  *   - No exceptions, aborts or device traps cross this boundary; errors are status codes.
  *     There is no CPU fallback: without a usable CUDA device calls fail with APAR_ERR_CUDA.
  *
@@ -131,7 +135,8 @@ apar_status apar_new_threads(apar_ctx* ctx, int32_t n, int32_t* tid_out /*[host]
  * block is taken from the free list and the r valid rows of the parent's last block (K and V,
  * all KV heads) are copied into it by a kernel enqueued on the stream.  Child length = len.
  * The same parent may appear several times.  child_tid_out [host] receives n ids.
- * Errors: BAD_THREAD, NO_THREADS, NO_BLOCKS (needs one block per parent with r != 0). */
+ * Errors: BAD_THREAD, NO_THREADS, NO_BLOCKS (needs one block per parent with r != 0),
+ * WORKSPACE_TOO_SMALL (more copies in one call than the staging area holds), CUDA. */
 apar_status apar_fork(apar_ctx* ctx, int32_t n, const int32_t* parent_tid /*[host]*/,
                       int32_t* child_tid_out /*[host]*/, void* cuda_stream);
 

@@ -682,7 +682,7 @@ apar_status apar_append_kv(apar_ctx* c, int32_t n, const int32_t* tid, const int
       }
       if (!stg) {
         apar_status rc = acquire(c, &stg);
-        if (rc) return rc;   // bookkeeping of earlier rows stands; the CUDA error is sticky
+        if (rc) return rc;   // APAR_ERR_CUDA: the context is unusable from here on (apar.h)
         slots = (int32_t*)stg->host;
       }
       slots[filled++] = tab[pos / kBlock] * kBlock + pos % kBlock;
