@@ -84,7 +84,9 @@ class ClockSampler:
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
                  "-lms", "20", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._read, daemon=True).start()
-            time.sleep(0.1)          # the first sample is on its way before the timed region
+            t0 = time.time()         # the first sample has arrived before the timed region starts
+            while not self.lines and time.time() - t0 < 3.0:
+                time.sleep(0.01)
         except Exception:
             self.proc = None
         return self
@@ -292,6 +294,7 @@ class DeviceRun:
         self.spec, self.shape, self.L = spec, spec.shape, layers
         nb, nt, mb = pool_requirements(spec)
         self.T = len(spec.live_nodes())
+        steps_total += 12          # the host-cost pass after the timed steps
         self.n_step_forks = sum(1 for n in spec.nodes if n.step_fork)
         grow = (self.T + self.n_step_forks) * (2 * steps_total // 16 + 2) + 2 * self.n_step_forks
         self.dims = (nb + grow, nt + self.n_step_forks, mb + 2 * steps_total // 16 + 2)
@@ -332,22 +335,27 @@ class DeviceRun:
             self.sess = self.step0 = self.graph = None
             torch.cuda.empty_cache()
 
-    def one_step(self, q, k_new, v_new, record, stream=None, out=None):
-        """fork (if the workload has one) + append + attention [+ release of the step's forks]."""
+    def one_step(self, q, k_new, v_new, record, stream=None, out=None, host=None):
+        """fork (if the workload has one) + one decode step (apar_decode_step: append of one row
+        per live thread + attention) [+ release of the step's forks].  record: the library
+        records a pair of CUDA events around the attention kernels of the step.  host: a dict
+        that receives the wall time of each library call."""
         B, sess, step0 = self.B, self.sess, self.step0
         stream = self.stream if stream is None else stream
         out = self.out if out is None else out
+        t0 = time.perf_counter()
         kids = B.apar_fork(sess.ctx, step0.fork_parents, stream) if step0.fork_parents else []
         live = B.int32_array(self.base_live + kids) if kids else self.base_live_arr
-        B.apar_append_kv(sess.ctx, live, None, k_new.data_ptr(), v_new.data_ptr(), stream)
+        t1 = time.perf_counter()
         if record:
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-        B.apar_tree_decode_attention(sess.ctx, live, q.data_ptr(), out.data_ptr(), sess.sm_scale,
-                                     stream)
+            pair = self.event_pool[len(self.attn_events)]
+            B.apar_set_timing_events(sess.ctx, pair[0].cuda_event, pair[1].cuda_event)
+            self.attn_events.append(pair)
+        B.apar_decode_step(sess.ctx, live, k_new.data_ptr(), v_new.data_ptr(), q.data_ptr(),
+                           out.data_ptr(), sess.sm_scale, stream)
         if record:
-            e1.record()
-            self.attn_events.append((e0, e1))
+            B.apar_set_timing_events(sess.ctx, 0, 0)
+        t2 = time.perf_counter()
         if self.graph is not None:        # the other layers, replayed from the captured graph
             if (q.data_ptr(), k_new.data_ptr(), out.data_ptr()) != self.graph_ptrs:
                 for dst, src in zip(self.graph_in, (q, k_new, v_new)):
@@ -358,8 +366,14 @@ class DeviceRun:
                 B.apar_append_kv_layer(sess.ctx, l, k_new.data_ptr(), v_new.data_ptr(), stream)
                 B.apar_tree_decode_attention_layer(sess.ctx, l, q.data_ptr(), out.data_ptr(),
                                                    sess.sm_scale, stream)
+        t3 = time.perf_counter()
         if kids:
             B.apar_release(sess.ctx, kids)
+        if host is not None:
+            t4 = time.perf_counter()
+            for key, dt in (("fork", t1 - t0), ("decode_step", t2 - t1), ("other_layers", t3 - t2),
+                            ("release", t4 - t3), ("total", t4 - t0)):
+                host.setdefault(key, []).append(dt)
 
     def capture_layer_loop(self):
         """Layers 1.. of a step only launch kernels whose sizes the cached plan fixes: capture
@@ -391,8 +405,14 @@ class DeviceRun:
             self.one_step(*inputs[0], record=False)
             sync()
         k0 = self.sess.stats()["kernels_total"]
-        sampler = ClockSampler(clock_index).start() if clock_index is not None else None
+        # events the library records around the attention kernels of every timed step
+        self.event_pool = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                           for _ in range(steps)]
+        for a, b in self.event_pool:
+            a.record(); b.record()            # creates the handles
+        sync()
         self.attn_events = []
+        sampler = ClockSampler(clock_index).start() if clock_index is not None else None
         host_t0 = time.perf_counter()
         # A workload whose KV fits in the L2 cache would be timed on cache hits: for those,
         # every step is timed on its own and a buffer larger than L2 is written between steps.
@@ -425,9 +445,21 @@ class DeviceRun:
             raise SystemExit(f"a kernel gave up a bounded wait (code {st['device_wait_timeouts']}): "
                              "the timed results are invalid")
         attn = sorted(a.elapsed_time(b) for a, b in self.attn_events)
+        # What the calls of a step cost the host thread: further steps, each started on an idle
+        # GPU (so that no call waits for a staging buffer the GPU still holds), calls timed alone.
+        host = {}
+        plan_us = []
+        for i in range(min(steps, 10)):
+            sync()
+            self.one_step(*inputs[i % len(inputs)], record=False, host=host)
+            plan_us.append(self.B.apar_get_stats(self.sess.ctx)["attn_plan_host_us"])
+        sync()
+        host_calls = {k: 1e3 * statistics.median(v) for k, v in host.items()}
+        host_calls["planner"] = 1e-3 * statistics.median(plan_us)
         return {"total_ms": total_ms, "host_issue_ms": host_ms, "clocks": clocks, "stats": st,
                 "launches": st["kernels_total"] - k0, "attn_ms": statistics.mean(attn),
-                "attn_ms_median": attn[len(attn) // 2], "attn_ms_min": attn[0], "steps": steps}
+                "attn_ms_median": attn[len(attn) // 2], "attn_ms_min": attn[0], "steps": steps,
+                "host_calls_ms": host_calls}
 
     def summary(self, r, peak):
         """Throughput, byte counts and roofline figures of one timed device arm."""
@@ -453,7 +485,11 @@ class DeviceRun:
             "algorithmic_bytes": algo_bytes, "achieved_gbs": achieved,
             "frac_of_measured_peak": achieved / peak,
             "unique_kv_frac_of_nominal": unique_bytes / (r["attn_ms"] * 1e-3) / 1e9 / 8000.0,
+            # wall time of the issuing loop per step (the host runs ahead of the GPU until the
+            # staging ring is full, then at the GPU's pace) and the calls' own cost on an idle GPU
             "host_issue_ms_per_step": r["host_issue_ms"] / steps,
+            "host_calls_ms_per_step": r["host_calls_ms"]["total"],
+            "host_calls_ms": r["host_calls_ms"],
             "gpu_launches": r["launches"], "clocks": r["clocks"],
             "l2": "flushed between steps" if self.small else "inputs larger than L2",
         }
@@ -473,8 +509,9 @@ def lifecycle_report(dev, n_requests=96, n_steps=1500, max_live=96):
                     device=dev)
     rep = {"requests": n_requests, "steps": n_steps, "max_live_threads": max_live,
            "threads": len(req), "forks": sum(len(s.fork) for s in steps)}
+    table_blocks = synth.lifecycle_longest_thread(steps) // shape.block_size + 2
     for early in (True, False):
-        sess = PagedSession(shape, 16384, len(req) + 8, 64, device=dev)
+        sess = PagedSession(shape, 16384, len(req) + 8, table_blocks, device=dev)
         tokens = [0]
 
         def rows(n):
@@ -700,7 +737,7 @@ def run_ours(args):
                 "unique_kv_frac_of_nominal": head["unique_kv_frac_of_nominal"],
                 "attention_ms_median": head["attention_ms_median"],
                 "attention_ms_min": head["attention_ms_min"],
-                "kernel": "apar_tree_decode_attention call (table sync + attention + merge launches)",
+                "kernel": "the attention kernels of apar_decode_step (tcgen05 + warp-stream + single-row + merge launches), between events the library records on the stream",
                 "algorithmic_bytes": head["algorithmic_bytes"], "attention_ms": head["attention_ms"],
             },
             "kv_bytes": {"unique_per_step": head["unique_kv_bytes_per_step"],
@@ -714,7 +751,9 @@ def run_ours(args):
                      "mma_items": r["stats"]["attn_mma_items"],
                      "partials": r["stats"]["attn_partials"],
                      "reused_last_step": r["stats"]["attn_plan_reused"],
-                     "host_issue_ms_per_step": head["host_issue_ms_per_step"]},
+                     "host_issue_ms_per_step": head["host_issue_ms_per_step"],
+                     "host_calls_ms_per_step": head["host_calls_ms_per_step"],
+                     "host_calls_ms": head["host_calls_ms"]},
             "setup_s": t_setup,
         }
         line.update(extras)

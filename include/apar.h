@@ -114,6 +114,9 @@ typedef struct {
                                      Section 3.4, in block granularity)                           */
   int64_t device_wait_timeouts;   /* non-zero once a kernel gave up a bounded wait (results of
                                      that call are invalid); reading it synchronises the device   */
+  int64_t attn_plan_host_us;      /* host time the most recent attention call spent planning
+                                     (0 when it reused the cached plan), microseconds            */
+  int64_t attn_upload_bytes;      /* bytes that call staged for the device (plan, table deltas)  */
 } apar_stats;
 
 /* Bytes of device scratch a context with this configuration needs (pool pointers and the
@@ -123,6 +126,14 @@ size_t apar_workspace_bytes(const apar_config* cfg /*[host]*/);
 /* Creates a context over an empty pool.  Allocates host memory and pinned staging only.
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL, CUDA. */
 apar_status apar_create(const apar_config* cfg /*[host]*/, apar_ctx** out /*[host]*/);
+/* The same bookkeeping without a device (the paper has no counterpart): k_pool, v_pool and
+ * workspace are ignored, no CUDA call is made, nothing is ever launched.  apar_new_threads,
+ * apar_fork, apar_append_kv (row pointers may be NULL), apar_release, the paragraph calls and
+ * all introspection work as documented and hand out the same ids as a device context would;
+ * every attention call and apar_decode_step return APAR_ERR_UNSUPPORTED.  For schedulers that
+ * want to try an admission decision (will this fork or append fit?) on a copy of the state,
+ * and for checking the bookkeeping on a machine without a GPU. */
+apar_status apar_create_host_only(const apar_config* cfg /*[host]*/, apar_ctx** out /*[host]*/);
 apar_status apar_destroy(apar_ctx* ctx);
 
 /* n new prompt sequences (roots of paragraph trees; the initial sequence group of Algorithm 1): empty block
@@ -196,6 +207,43 @@ apar_status apar_append_kv_layer(apar_ctx* ctx, int32_t layer, const void* k_new
 apar_status apar_tree_decode_attention_layer(apar_ctx* ctx, int32_t layer,
                                              const void* q /*[device]*/, void* out /*[device]*/,
                                              float sm_scale, void* cuda_stream);
+
+/* One decode step of Algorithm 1 for the threads tid[0..n) in a single call: every thread gains
+ * one token (the Sample / append pair of the algorithm's loop; Section 2.3 "Decoding"), then
+ * attends over its chain, the new token included.  Equivalent to apar_append_kv (one row each)
+ * followed by apar_tree_decode_attention on the same list, with the same block ids, and built
+ * so that a steady step costs the host almost nothing: while the list stays the same from one
+ * step to the next (no release, no apar_append_kv in between), the device keeps the list, the
+ * tables and the lengths; one small kernel bumps the lengths and derives the pool slot of every
+ * new row from the device tables, and the host only handles the threads that start a new block
+ * in this step (one in sixteen) plus a counter per thread.  The work plan is reused as in
+ * apar_tree_decode_attention.  Layer 0 of the pools is written and read; other layers follow
+ * with apar_append_kv_layer / apar_tree_decode_attention_layer.
+ *   tid [host] distinct ids; k_new, v_new [device] bf16 [n][num_kv_heads][128], row i for tid[i];
+ *   q, out [device] bf16 [n][num_q_heads][128].
+ * CUDA graphs: a step whose list is unchanged and in which no thread starts a new block
+ * (apar_steps_before_new_block() > 0) launches kernels only and uses no staging buffer, so it
+ * can be captured (together with the layer calls that follow it) and replayed.  The capturing
+ * call does the host bookkeeping of the first replay; before every further replay call
+ * apar_note_step_replay.  While a stream is capturing, a step that would need staging is refused
+ * with APAR_ERR_INVALID_ARG and changes nothing.
+ * Errors: INVALID_ARG (also duplicate ids), BAD_THREAD, TABLE_FULL, NO_BLOCKS,
+ * WORKSPACE_TOO_SMALL, CUDA. */
+apar_status apar_decode_step(apar_ctx* ctx, int32_t n, const int32_t* tid /*[host]*/,
+                             const void* k_new /*[device]*/, const void* v_new /*[device]*/,
+                             const void* q /*[device]*/, void* out /*[device]*/, float sm_scale,
+                             void* cuda_stream);
+/* How many more steps the thread list of the most recent apar_decode_step can take before one
+ * of its threads starts a new block (0: the next step allocates).  Errors: INVALID_ARG if there
+ * is no such list or a release / apar_append_kv came after it. */
+apar_status apar_steps_before_new_block(apar_ctx* ctx, int32_t* steps_out /*[host]*/);
+/* Host side of one replay of a captured apar_decode_step: every thread of the list is one token
+ * longer, exactly what the replayed kernels do on the device.  Launches nothing.
+ * Errors: INVALID_ARG if the step list or the plan is no longer the captured one (any
+ * bookkeeping call since), or if a thread of the list would start a new block - make an
+ * ordinary apar_decode_step then, and capture again afterwards if block ids matter to the
+ * graph (they do not: the captured kernels read tables and lengths from the device). */
+apar_status apar_note_step_replay(apar_ctx* ctx);
 
 /* ReleaseCache (Algorithm 1; Section 2.3: a finished sequence gives back the cache that no
  * other sequence holds):
@@ -313,6 +361,20 @@ apar_status apar_debug_plan(int32_t num_blocks, int32_t num_q_heads, int32_t num
                             int32_t cap_users, int32_t* merges_out, int32_t cap_merges,
                             int64_t* counts_out);
 
+/* Debug aid, host only: the plan apar_tree_decode_attention would make for the threads
+ * tid[0..n) of this context (closed tails: token ranges are written out in full), in the same
+ * output arrays as apar_debug_plan; table_row of an item is the library's internal row of the
+ * thread.  by_groups != 0: the planner counts per group of blocks that the same threads hold
+ * (what the library does when no thread is listed twice), which needs distinct ids;
+ * by_groups == 0: it counts per block id, as apar_debug_plan does.  Both must give the same
+ * plan.  Drops the context's cached plan.
+ * Errors: INVALID_ARG, BAD_THREAD, EMPTY_CONTEXT, WORKSPACE_TOO_SMALL (counts_out filled). */
+apar_status apar_debug_plan_threads(apar_ctx* ctx, int32_t n, const int32_t* tid /*[host]*/,
+                                    int32_t by_groups, int32_t mma_min_rows, int32_t fuse_final,
+                                    int32_t* items_out, int32_t cap_items, int32_t* users_out,
+                                    int32_t cap_users, int32_t* merges_out, int32_t cap_merges,
+                                    int64_t* counts_out);
+
 /* Measurement aid (the paper has no counterpart): enqueues one kernel that reads `bytes` bytes
  * (rounded down to a multiple of 16) at `src` once, with the 16-byte streaming loads the
  * attention kernels use, and xors them into the 8-byte word at `sink`.  Timing it over a buffer
@@ -323,6 +385,14 @@ apar_status apar_debug_plan(int32_t num_blocks, int32_t num_q_heads, int32_t num
  * Returns APAR_ERR_INVALID_ARG for NULL or misaligned pointers, APAR_ERR_CUDA if the launch
  * failed (no context, so the CUDA error is read with cudaGetLastError by the caller). */
 apar_status apar_stream_read(const void* src, size_t bytes, void* sink, void* cuda_stream);
+
+/* Measurement aid (the paper has no counterpart): from now on every attention call of this
+ * context (apar_tree_decode_attention, apar_decode_step, the prefix and layer forms) records
+ * `start` on its stream just before its attention kernels and `stop` just after them, so that
+ * the caller can time those kernels alone inside a larger call.  Both are cudaEvent_t handles
+ * created by the caller with timing enabled; the library does not own them.  NULL, NULL turns
+ * it off.  Errors: INVALID_ARG if only one of the two is NULL. */
+apar_status apar_set_timing_events(apar_ctx* ctx, void* start, void* stop);
 
 /* cudaError_t value of the most recent failing CUDA call of this context (0 if none). */
 int32_t     apar_last_cuda_error(apar_ctx* ctx);

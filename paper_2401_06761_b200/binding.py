@@ -43,7 +43,8 @@ class apar_stats(C.Structure):
         "live_threads", "free_blocks", "used_blocks", "forks", "cow_blocks", "cow_rows",
         "attn_threads", "attn_attended_tokens", "attn_unique_tokens", "attn_work_items",
         "attn_partials", "attn_kernels", "attn_plan_reused", "attn_vec_items",
-        "attn_mma_items", "kernels_total", "peak_used_blocks", "device_wait_timeouts")]
+        "attn_mma_items", "kernels_total", "peak_used_blocks", "device_wait_timeouts",
+        "attn_plan_host_us", "attn_upload_bytes")]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -56,6 +57,7 @@ _cfgp = C.POINTER(apar_config)
 _SIGS = {
     "apar_workspace_bytes": (C.c_size_t, [_cfgp]),
     "apar_create": (C.c_int32, [_cfgp, C.POINTER(_ctx)]),
+    "apar_create_host_only": (C.c_int32, [_cfgp, C.POINTER(_ctx)]),
     "apar_destroy": (C.c_int32, [_ctx]),
     "apar_new_threads": (C.c_int32, [_ctx, C.c_int32, _i32p]),
     "apar_fork": (C.c_int32, [_ctx, C.c_int32, _i32p, _i32p, C.c_void_p]),
@@ -68,6 +70,10 @@ _SIGS = {
     "apar_append_kv_layer": (C.c_int32, [_ctx, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "apar_tree_decode_attention_layer": (C.c_int32, [_ctx, C.c_int32, C.c_void_p, C.c_void_p,
                                                      C.c_float, C.c_void_p]),
+    "apar_decode_step": (C.c_int32, [_ctx, C.c_int32, _i32p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                     C.c_void_p, C.c_float, C.c_void_p]),
+    "apar_steps_before_new_block": (C.c_int32, [_ctx, _i32p]),
+    "apar_note_step_replay": (C.c_int32, [_ctx]),
     "apar_release": (C.c_int32, [_ctx, C.c_int32, _i32p]),
     "apar_tree_decode_attention_tables": (C.c_int32, [_cfgp, C.c_int32, _i32p, _i32p,
                                                       C.c_void_p, C.c_void_p, C.c_float,
@@ -86,7 +92,11 @@ _SIGS = {
     "apar_debug_plan": (C.c_int32, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, _i32p,
                                     _i32p, C.c_int32, C.c_int32, _i32p, C.c_int32, _i32p,
                                     C.c_int32, _i32p, C.c_int32, C.POINTER(C.c_int64)]),
+    "apar_debug_plan_threads": (C.c_int32, [_ctx, C.c_int32, _i32p, C.c_int32, C.c_int32,
+                                            C.c_int32, _i32p, C.c_int32, _i32p, C.c_int32, _i32p,
+                                            C.c_int32, C.POINTER(C.c_int64)]),
     "apar_stream_read": (C.c_int32, [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]),
+    "apar_set_timing_events": (C.c_int32, [_ctx, C.c_void_p, C.c_void_p]),
     "apar_last_cuda_error": (C.c_int32, [_ctx]),
     "apar_status_string": (C.c_char_p, [C.c_int32]),
 }
@@ -126,6 +136,12 @@ def apar_workspace_bytes(cfg: apar_config) -> int:
 def apar_create(cfg: apar_config):
     ctx = _ctx()
     _check(lib.apar_create(C.byref(cfg), C.byref(ctx)))
+    return ctx
+
+
+def apar_create_host_only(cfg: apar_config):
+    ctx = _ctx()
+    _check(lib.apar_create_host_only(C.byref(cfg), C.byref(ctx)))
     return ctx
 
 
@@ -169,6 +185,22 @@ def apar_append_kv_layer(ctx, layer: int, k_new: int, v_new: int, stream=0):
 
 def apar_tree_decode_attention_layer(ctx, layer: int, q: int, out: int, sm_scale: float, stream=0):
     _check(lib.apar_tree_decode_attention_layer(ctx, layer, q, out, sm_scale, stream))
+
+
+def apar_decode_step(ctx, tid, k_new: int, v_new: int, q: int, out: int, sm_scale: float,
+                     stream=0):
+    tids, n = _arr(tid)
+    _check(lib.apar_decode_step(ctx, n, tids, k_new, v_new, q, out, sm_scale, stream))
+
+
+def apar_steps_before_new_block(ctx) -> int:
+    steps = C.c_int32()
+    _check(lib.apar_steps_before_new_block(ctx, C.byref(steps)))
+    return steps.value
+
+
+def apar_note_step_replay(ctx):
+    _check(lib.apar_note_step_replay(ctx))
 
 
 def apar_release(ctx, tid):
@@ -263,8 +295,32 @@ def apar_debug_plan(num_blocks, num_q_heads, num_kv_heads, tables, lens, mma_min
     return items[:c["items"]], users[:c["users"]], merges[:c["merges"]], c
 
 
+def apar_debug_plan_threads(ctx, tid, by_groups: bool, mma_min_rows=2, fuse_final=True):
+    """Host-only planning for threads of a context; same return value as apar_debug_plan."""
+    tids, n = _arr(tid)
+    lens = [apar_get_thread(ctx, t)[0] for t in tid]
+    cap_users = int(sum((int(l) + 15) // 16 for l in lens)) + 1
+    cap_items = 4 * cap_users + 16
+    items = np.zeros((cap_items, 8), dtype=np.int32)
+    users = np.zeros((cap_users, 2), dtype=np.int32)
+    merges = np.zeros((n + 1, 3), dtype=np.int32)
+    counts = (C.c_int64 * 6)()
+    p = lambda a: a.ctypes.data_as(_i32p)
+    _check(lib.apar_debug_plan_threads(ctx, n, tids, int(bool(by_groups)), mma_min_rows,
+                                       int(bool(fuse_final)), p(items), cap_items, p(users),
+                                       cap_users, p(merges), n + 1, counts))
+    names = ("items", "users", "merges", "partial_slots", "unique_tokens", "attended_tokens")
+    c = dict(zip(names, (int(x) for x in counts)))
+    return items[:c["items"]], users[:c["users"]], merges[:c["merges"]], c
+
+
 def apar_stream_read(src: int, nbytes: int, sink: int, stream=0):
     _check(lib.apar_stream_read(src, nbytes, sink, stream))
+
+
+def apar_set_timing_events(ctx, start: int, stop: int):
+    """cudaEvent_t handles (integers), or 0, 0 to turn the recording off."""
+    _check(lib.apar_set_timing_events(ctx, start or None, stop or None))
 
 
 def apar_last_cuda_error(ctx) -> int:

@@ -1,6 +1,7 @@
 // C-ABI entry points (include/apar.h): host bookkeeping of the paged pool, staging of
 // per-call metadata, and the launch sequence of each call.
 #include <algorithm>
+#include <chrono>
 #include <climits>
 #include <cmath>
 #include <cstdlib>
@@ -25,7 +26,7 @@ constexpr int kSlotMapRows = 262144;  // new-row slots of the last append kept f
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {            // partition of the caller's workspace
-  size_t err, tables, lens, stage, slot_map, plan_items, plan_users, plan_merges, part_ml, part_o, total;
+  size_t err, tables, lens, stage, slot_map, step_rows, plan_items, plan_users, plan_merges, part_ml, part_o, total;
   size_t stage_cap;        // bytes of the transient staging area
   int64_t slot_capacity;   // partial rows (before the head dimension)
   int64_t entry_capacity;  // (item, user) pairs a plan may hold
@@ -55,7 +56,8 @@ Layout make_layout(const apar_config* c) {
   L.tables = take(table_bytes);
   L.lens = take((size_t)c->max_threads * 4);
   L.stage = take(L.stage_cap);
-  L.slot_map = take((size_t)kSlotMapRows * 4);
+  L.slot_map = take((size_t)std::max(kSlotMapRows, c->max_threads) * 4);
+  L.step_rows = take((size_t)c->max_threads * 4);
   L.plan_items = take((size_t)L.entry_capacity * sizeof(WorkItem));
   L.plan_users = take((size_t)L.entry_capacity * sizeof(UserRef));
   L.plan_merges = take((size_t)c->max_threads * sizeof(MergeRef));
@@ -124,6 +126,21 @@ struct apar_ctx {
   uint64_t book_seq = 1, attn_book_seq = 0;   // bookkeeping calls so far / at the last plan
   int64_t last_append_rows = -1;              // rows of the last append kept in the slot map
   int32_t last_cuda = 0;
+  bool host_only = false;                     // bookkeeping only: no device, nothing is launched
+  // Every thread's table as runs of groups (blocks held by the same set of threads).  A
+  // thread's blocks since it was last forked form its own, open group; a fork closes the full
+  // blocks of that group (the child lists them from then on) and opens a new one.
+  std::vector<std::vector<BlockRun>> runs;    // by slot
+  std::vector<uint8_t> own_open;              // by slot: the last run is the open group
+  std::vector<int32_t> gid_ref, gid_free;     // threads listing each group; ids to reuse
+  bool track_runs = true;                     // false: tables were filled in directly
+  bool plan_by_runs = true;                   // APAR_PLANNER=tables (testing): walk block ids
+  cudaEvent_t time_start = nullptr, time_stop = nullptr;   // caller's events around the kernels
+  // thread list of the most recent apar_decode_step; its table rows are resident on the device
+  std::vector<int32_t> step_tids, step_slots, tmp_slots;
+  bool step_valid = false;
+  uint64_t life_seq = 1, mod_seq = 1;         // releases so far / appends outside apar_decode_step
+  uint64_t step_life = 0, step_mod = 0;       // their values when the list was last brought in sync
   // paragraph tree of Algorithm 1 (host only)
   struct PNodeRec { int32_t tid, start, end, first_child, next_sibling; };
   std::vector<PNodeRec> pnodes;
@@ -206,6 +223,64 @@ int32_t alloc_block(apar_ctx* c) {
   return b;
 }
 
+int32_t new_gid(apar_ctx* c) {
+  int32_t g;
+  if (!c->gid_free.empty()) {
+    g = c->gid_free.back();
+    c->gid_free.pop_back();
+  } else {
+    g = (int32_t)c->gid_ref.size();
+    c->gid_ref.push_back(0);
+  }
+  c->gid_ref[g] = 1;
+  return g;
+}
+
+// The thread in `slot` gained a block at table position `pos` (its new last block).
+void run_add_block(apar_ctx* c, int slot, int32_t pos) {
+  std::vector<BlockRun>& r = c->runs[slot];
+  if (c->own_open[slot]) {
+    ++r.back().n;
+  } else {
+    r.push_back(BlockRun{new_gid(c), pos, 1});
+    c->own_open[slot] = 1;
+  }
+}
+
+// Fork of the thread in slot `ps`, which holds `full` full blocks, into the fresh slot `cs`:
+// the full blocks of the parent's open group become a group of their own, shared from now
+// on, and the child lists every run below `full`.
+void run_fork(apar_ctx* c, int ps, int cs, int32_t full) {
+  std::vector<BlockRun>& pr = c->runs[ps];
+  if (c->own_open[ps]) {
+    BlockRun& last = pr.back();
+    if (full > last.pos) {
+      if (last.pos + last.n > full) {           // the partial block stays the parent's own
+        const int32_t rest = last.pos + last.n - full;
+        last.n = full - last.pos;
+        pr.push_back(BlockRun{new_gid(c), full, rest});
+      } else {
+        c->own_open[ps] = 0;                    // all of it full: the next block opens a group
+      }
+    }
+  }
+  std::vector<BlockRun>& cr = c->runs[cs];
+  cr.clear();
+  for (const BlockRun& r : pr) {
+    if (r.pos + r.n > full) break;
+    cr.push_back(r);
+    ++c->gid_ref[r.gid];
+  }
+  c->own_open[cs] = 0;
+}
+
+void run_release(apar_ctx* c, int slot) {
+  for (const BlockRun& r : c->runs[slot])
+    if (--c->gid_ref[r.gid] == 0) c->gid_free.push_back(r.gid);
+  c->runs[slot].clear();
+  c->own_open[slot] = 0;
+}
+
 // Brings the device copies of block tables and lengths up to date for the given slots.
 apar_status sync_device_tables(apar_ctx* c, const int32_t* slots, int n, cudaStream_t st) {
   int i = 0;
@@ -250,6 +325,7 @@ apar_status sync_device_tables(apar_ctx* c, const int32_t* slots, int n, cudaStr
     // close the gaps between the three arrays, so that only what was filled crosses PCIe
     const size_t off_pairs = (size_t)nd * sizeof(TableDelta);
     const size_t off_data = off_pairs + (size_t)np * 8;
+    c->last.attn_upload_bytes += (int64_t)(off_data + used * 4);
     memmove(s->host + off_pairs, pairs, (size_t)np * 8);
     memmove(s->host + off_data, data, used * 4);
     // Every entry is read exactly once, so the kernel takes them straight from the pinned
@@ -365,27 +441,43 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
   return APAR_OK;
 }
 
+// A plan is kept while the tree is unchanged and the same threads are queried; it is rebuilt
+// now and then only because the longest-first order of its items drifts as tails grow.
+bool plan_reusable(const apar_ctx* c, int n, const int32_t* tids, int64_t attended) {
+  return c->plan_epoch == c->struct_epoch && c->plan_age < 1024 &&
+         (int)c->plan_tids.size() == n &&
+         memcmp(c->plan_tids.data(), tids, (size_t)n * 4) == 0 &&
+         attended - c->plan_attended < c->plan_attended / 4 + 64;
+}
+
 // The attention launch sequence for queries given as slots (already validated, len > 0).
 // qlens (optional): tokens query i attends, counted from the root; default the thread's length.
 apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32_t* tids,
                           bool has_dups, const void* q, void* out, float sm_scale,
-                          cudaStream_t st, const int32_t* qlens = nullptr) {
+                          cudaStream_t st, const int32_t* qlens = nullptr,
+                          bool tables_in_sync = false) {
   c->last.attn_kernels = 0;
   int64_t attended = 0;
   for (int i = 0; i < n; ++i) attended += qlens ? qlens[i] : c->slots[qslots[i]].len;
 
   const bool cacheable = tids != nullptr && !has_dups && !qlens;
-  // a plan is kept while the tree is unchanged; it is rebuilt now and then only because the
-  // longest-first order of its items drifts as tails grow
-  bool reuse = cacheable && c->plan_epoch == c->struct_epoch && c->plan_age < 1024 &&
-               (int)c->plan_tids.size() == n &&
-               memcmp(c->plan_tids.data(), tids, (size_t)n * 4) == 0 &&
-               attended - c->plan_attended < c->plan_attended / 4 + 64;
+  bool reuse = cacheable && plan_reusable(c, n, tids, attended);
+  c->last.attn_plan_host_us = 0;
+  if (!tables_in_sync) c->last.attn_upload_bytes = 0;   // (else the caller's uploads count too)
   if (!reuse) {
+    const auto t_plan = std::chrono::steady_clock::now();
     c->pq.resize(n);
-    for (int i = 0; i < n; ++i)
+    // every query attends its thread's whole chain and no thread is listed twice: the planner
+    // may count per group of blocks instead of per block
+    const bool by_runs = cacheable && c->track_runs && c->plan_by_runs;
+    for (int i = 0; i < n; ++i) {
       c->pq[i] = PlanQuery{c->row(qslots[i]), qslots[i],
                            qlens ? qlens[i] : c->slots[qslots[i]].len};
+      if (by_runs) {
+        c->pq[i].runs = c->runs[qslots[i]].data();
+        c->pq[i].n_runs = (int32_t)c->runs[qslots[i]].size();
+      }
+    }
     // Single-row items (no GQA group, private tail): the vector kernel keeps up to 16 CTAs per
     // SM in flight and wins when there are many of them; with few, the warp-stream kernel's
     // deeper per-warp rings do better (measured crossover near 900 queries).
@@ -394,14 +486,15 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
     // finishing items land in the single-row vector kernel or the warp-stream kernel
     const bool fuse_final = c->use_ws && c->plan_min_rows <= 2;
     if (!c->planner.build(c->pq.data(), n, c->lay.slot_capacity, cacheable, c->plan_min_rows,
-                          fuse_final,
-                          &c->plan))
+                          fuse_final, &c->plan, by_runs))
       return APAR_ERR_WORKSPACE_TOO_SMALL;
     if ((int64_t)c->plan.users.size() > c->lay.entry_capacity ||
         (int64_t)c->plan.items.size() > c->lay.entry_capacity)
       return APAR_ERR_WORKSPACE_TOO_SMALL;
+    c->last.attn_plan_host_us = std::chrono::duration_cast<std::chrono::microseconds>(
+                                    std::chrono::steady_clock::now() - t_plan).count();
   }
-  apar_status rc = sync_device_tables(c, qslots, n, st);
+  apar_status rc = tables_in_sync ? APAR_OK : sync_device_tables(c, qslots, n, st);
   if (rc) return rc;
 
   const Plan& p = c->plan;
@@ -423,6 +516,7 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
         memcpy(s->host, (const char*)part.src + done, chunk);
         rc = send(c, s, c->ws(part.dst) + done, chunk, st);
         if (rc) return rc;
+        c->last.attn_upload_bytes += (int64_t)chunk;
         done += chunk;
       }
     }
@@ -439,8 +533,10 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
   }
 
   int launches = 0;
+  if (c->time_start) APAR_CUDA(c, cudaEventRecord(c->time_start, st));
   rc = launch_plan(c, 0, q, out, sm_scale, st, &launches);
   if (rc) return rc;
+  if (c->time_stop) APAR_CUDA(c, cudaEventRecord(c->time_stop, st));
   c->attn_book_seq = c->book_seq;
   c->kernels_total += launches;
   c->last.attn_kernels += launches;
@@ -455,17 +551,23 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
   return APAR_OK;
 }
 
-apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
+apar_status create_impl(const apar_config* cfg, bool external, bool host_only, apar_ctx** out) {
   if (!cfg || !out) return APAR_ERR_INVALID_ARG;
   if (!supported(cfg)) return APAR_ERR_UNSUPPORTED;
-  if (!cfg->k_pool || !cfg->v_pool || !cfg->workspace) return APAR_ERR_INVALID_ARG;
-  if (((uintptr_t)cfg->k_pool | (uintptr_t)cfg->v_pool) & 255) return APAR_ERR_INVALID_ARG;
-  if ((uintptr_t)cfg->workspace & 255) return APAR_ERR_INVALID_ARG;
   const Layout lay = make_layout(cfg);
-  if (cfg->workspace_bytes < lay.total) return APAR_ERR_WORKSPACE_TOO_SMALL;
+  if (!host_only) {
+    if (!cfg->k_pool || !cfg->v_pool || !cfg->workspace) return APAR_ERR_INVALID_ARG;
+    if (((uintptr_t)cfg->k_pool | (uintptr_t)cfg->v_pool) & 255) return APAR_ERR_INVALID_ARG;
+    if ((uintptr_t)cfg->workspace & 255) return APAR_ERR_INVALID_ARG;
+    if (cfg->workspace_bytes < lay.total) return APAR_ERR_WORKSPACE_TOO_SMALL;
+  }
   apar_ctx* c = new (std::nothrow) apar_ctx();
   if (!c) return APAR_ERR_INVALID_ARG;
   c->cfg = *cfg;
+  c->host_only = host_only;
+  c->track_runs = !external;
+  c->runs.resize(cfg->max_threads);
+  c->own_open.assign(cfg->max_threads, 0);
   c->lay = lay;
   c->shape = Shape{cfg->num_q_heads, cfg->num_kv_heads, cfg->num_q_heads / cfg->num_kv_heads,
                    cfg->max_blocks_per_thread};
@@ -488,9 +590,15 @@ apar_status create_impl(const apar_config* cfg, bool external, apar_ctx** out) {
   c->use_pdl = pdl ? atoi(pdl) : 1;
   c->use_ws = !(path && (!strcmp(path, "mma") || !strcmp(path, "umma")));
   c->auto_path = !path || !strcmp(path, "auto") || !*path;
+  const char* planner = getenv("APAR_PLANNER");          // testing: "tables" = per-block walk
+  c->plan_by_runs = !(planner && !strcmp(planner, "tables"));
   c->ring_bytes = lay.stage_cap;
   c->num_layers = std::max(1, cfg->num_layers);
   c->layer_bytes = (size_t)cfg->num_blocks * cfg->num_kv_heads * kTileBytes;
+  if (host_only) {
+    *out = c;
+    return APAR_OK;
+  }
   c->tm_k.resize(c->num_layers);
   c->tm_v.resize(c->num_layers);
   bool maps_ok = true;
@@ -527,7 +635,11 @@ size_t apar_workspace_bytes(const apar_config* cfg) {
 }
 
 apar_status apar_create(const apar_config* cfg, apar_ctx** out) {
-  return create_impl(cfg, false, out);
+  return create_impl(cfg, false, false, out);
+}
+
+apar_status apar_create_host_only(const apar_config* cfg, apar_ctx** out) {
+  return create_impl(cfg, false, true, out);
 }
 
 apar_status apar_destroy(apar_ctx* c) {
@@ -564,7 +676,7 @@ apar_status apar_fork(apar_ctx* c, int32_t n, const int32_t* parent_tid, int32_t
   if (need > (int)c->free_stack.size()) return APAR_ERR_NO_BLOCKS;
   if ((size_t)need * sizeof(CowCopy) > c->lay.stage_cap) return APAR_ERR_WORKSPACE_TOO_SMALL;
   Staging* stg = nullptr;
-  if (need) {
+  if (need && !c->host_only) {
     apar_status rc = acquire(c, &stg);
     if (rc) return rc;
   }
@@ -582,11 +694,14 @@ apar_status apar_fork(apar_ctx* c, int32_t n, const int32_t* parent_tid, int32_t
       ++c->refcnt[pt[b]];
     }
     ch.n_blocks = full;
+    run_fork(c, ps, cs, full);
     if (r) {
       const int32_t dst = alloc_block(c);
-      copies[nc++] = CowCopy{pt[full], dst, r, 0};
+      if (copies) copies[nc] = CowCopy{pt[full], dst, r, 0};
+      ++nc;
       ct[full] = dst;
       ch.n_blocks = full + 1;
+      run_add_block(c, cs, full);
       ++c->cow_blocks;
       c->cow_rows += r;
     }
@@ -607,7 +722,7 @@ apar_status apar_fork(apar_ctx* c, int32_t n, const int32_t* parent_tid, int32_t
   }
   if (n) ++c->struct_epoch;
   ++c->book_seq;
-  if (nc) {
+  if (nc && !c->host_only) {
     char* d_stage = c->ws(c->lay.stage);
     apar_status rc = send(c, stg, d_stage, (size_t)nc * sizeof(CowCopy), st);
     if (rc) return rc;
@@ -623,7 +738,8 @@ apar_status apar_fork(apar_ctx* c, int32_t n, const int32_t* parent_tid, int32_t
 
 apar_status apar_append_kv(apar_ctx* c, int32_t n, const int32_t* tid, const int32_t* n_tok,
                            const void* k_new, const void* v_new, void* cuda_stream) {
-  if (!c || n < 0 || (n > 0 && (!tid || !k_new || !v_new))) return APAR_ERR_INVALID_ARG;
+  if (!c || n < 0 || (n > 0 && (!tid || ((!k_new || !v_new) && !c->host_only))))
+    return APAR_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   for (int i = 0; i < n; ++i)
     if (slot_of(c, tid[i]) < 0) return APAR_ERR_BAD_THREAD;
@@ -649,6 +765,7 @@ apar_status apar_append_kv(apar_ctx* c, int32_t n, const int32_t* tid, const int
   const bool keep = rows <= kSlotMapRows;
   c->last_append_rows = keep ? rows : -1;
   ++c->book_seq;
+  ++c->mod_seq;
   const size_t cap_rows = c->lay.stage_cap / 4;
   Staging* stg = nullptr;
   int32_t* slots = nullptr;
@@ -678,7 +795,12 @@ apar_status apar_append_kv(apar_ctx* c, int32_t n, const int32_t* tid, const int
       if (pos % kBlock == 0) {
         // a thread without a private tail gains one: cached plans no longer describe it
         if (t.n_blocks == 0 || c->refcnt[tab[t.n_blocks - 1]] > 1) ++c->struct_epoch;
+        run_add_block(c, s, t.n_blocks);
         tab[t.n_blocks++] = alloc_block(c);
+      }
+      if (c->host_only) {
+        t.len = pos + 1;
+        continue;
       }
       if (!stg) {
         apar_status rc = acquire(c, &stg);
@@ -696,10 +818,173 @@ apar_status apar_append_kv(apar_ctx* c, int32_t n, const int32_t* tid, const int
   return flush();
 }
 
+// True while the cached step list still describes live threads whose device rows are current.
+static bool step_list_current(const apar_ctx* c) {
+  return c->step_valid && c->step_life == c->life_seq && c->step_mod == c->mod_seq;
+}
+
+apar_status apar_decode_step(apar_ctx* c, int32_t n, const int32_t* tid, const void* k_new,
+                             const void* v_new, const void* q, void* out, float sm_scale,
+                             void* cuda_stream) {
+  if (!c || n < 0 || n > c->cfg.max_threads ||
+      (n > 0 && (!tid || !k_new || !v_new || !q || !out)))
+    return APAR_ERR_INVALID_ARG;
+  if (c->host_only) return APAR_ERR_UNSUPPORTED;
+  if (n == 0) return APAR_OK;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const bool same = step_list_current(c) && (int)c->step_tids.size() == n &&
+                    memcmp(c->step_tids.data(), tid, (size_t)n * 4) == 0;
+  // ---- every check comes before the first change
+  if (!same) {
+    c->tmp_slots.resize(n);
+    for (int i = 0; i < n; ++i) {
+      const int s = slot_of(c, tid[i]);
+      if (s < 0) return APAR_ERR_BAD_THREAD;
+      c->tmp_slots[i] = s;
+    }
+    const uint32_t mk = next_mark(c);
+    for (int i = 0; i < n; ++i) {
+      if (c->mark[c->tmp_slots[i]] == mk) return APAR_ERR_INVALID_ARG;
+      c->mark[c->tmp_slots[i]] = mk;
+    }
+  }
+  const int32_t* sl = same ? c->step_slots.data() : c->tmp_slots.data();
+  int need = 0;
+  for (int i = 0; i < n; ++i) {
+    const int32_t len = c->slots[sl[i]].len;
+    if ((len & (kBlock - 1)) == 0) {
+      if (len / kBlock >= c->cfg.max_blocks_per_thread) return APAR_ERR_TABLE_FULL;
+      ++need;
+    }
+  }
+  if (need > (int)c->free_stack.size()) return APAR_ERR_NO_BLOCKS;
+  if ((size_t)need * sizeof(int4) > c->lay.stage_cap) return APAR_ERR_WORKSPACE_TOO_SMALL;
+  {
+    // a step that has to use the staging buffers (new list, new blocks) cannot be captured
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    APAR_CUDA(c, cudaStreamIsCapturing(st, &cap));
+    if (cap != cudaStreamCaptureStatusNone) {
+      if (!same || need) return APAR_ERR_INVALID_ARG;
+      int64_t attended = n;                       // chain lengths after this step
+      for (int i = 0; i < n; ++i) attended += c->slots[sl[i]].len;
+      if (!plan_reusable(c, n, tid, attended)) return APAR_ERR_INVALID_ARG;
+    }
+  }
+  apar_status rc;
+  c->last.attn_upload_bytes = (same ? 0 : (int64_t)n * 4) + (int64_t)need * sizeof(int4);
+  if (!same) {
+    // a new list: its table rows go to the device, and the device tables and lengths of its
+    // threads are brought up to date once; from then on the step kernel keeps them current
+    c->step_valid = false;
+    c->step_slots.swap(c->tmp_slots);
+    c->step_tids.assign(tid, tid + n);
+    size_t done = 0;
+    const size_t bytes = (size_t)n * 4;
+    while (done < bytes) {
+      Staging* s;
+      rc = acquire(c, &s);
+      if (rc) return rc;
+      const size_t chunk = std::min(bytes - done, c->ring_bytes);
+      memcpy(s->host, (const char*)c->step_slots.data() + done, chunk);
+      rc = send(c, s, c->ws(c->lay.step_rows) + done, chunk, st);
+      if (rc) return rc;
+      done += chunk;
+    }
+    rc = sync_device_tables(c, c->step_slots.data(), n, st);
+    if (rc) return rc;
+    c->step_valid = true;
+    c->step_life = c->life_seq;
+    c->step_mod = c->mod_seq;
+    sl = c->step_slots.data();
+  }
+  // ---- bookkeeping: only a thread that starts a new block needs more than a counter
+  Staging* stg = nullptr;
+  int4* pairs = nullptr;
+  int np = 0;
+  if (need) {
+    rc = acquire(c, &stg);
+    if (rc) return rc;
+    pairs = (int4*)stg->host;
+  }
+  for (int i = 0; i < n; ++i) {
+    ThreadRec& t = c->slots[sl[i]];
+    if ((t.len & (kBlock - 1)) == 0) {
+      int32_t* tab = c->row(sl[i]);
+      // a thread without a private tail gains one: cached plans no longer describe it
+      if (t.n_blocks == 0 || c->refcnt[tab[t.n_blocks - 1]] > 1) ++c->struct_epoch;
+      const int32_t b = alloc_block(c);
+      run_add_block(c, sl[i], t.n_blocks);
+      pairs[np++] = make_int4(i, sl[i], t.n_blocks, b);
+      tab[t.n_blocks++] = b;
+      t.synced = t.n_blocks;
+    }
+    ++t.len;
+    t.dev_len = t.len;
+  }
+  ++c->book_seq;
+  c->last_append_rows = n;
+  const void* d_pairs = nullptr;
+  if (np) {
+    if (stg->mapped) {
+      d_pairs = stg->mapped;              // read once, straight from the pinned buffer
+    } else {
+      d_pairs = c->ws(c->lay.stage);
+      rc = send(c, stg, c->ws(c->lay.stage), (size_t)np * sizeof(int4), st);
+      if (rc) return rc;
+    }
+  }
+  APAR_CUDA(c, launch_step_advance((int32_t*)c->ws(c->lay.tables), c->cfg.max_blocks_per_thread,
+                                   (int32_t*)c->ws(c->lay.lens),
+                                   (const int32_t*)c->ws(c->lay.step_rows), n, d_pairs, np,
+                                   (int32_t*)c->ws(c->lay.slot_map), st));
+  if (np && stg->mapped) {
+    rc = send(c, stg, nullptr, 0, st);    // nothing to copy: only marks the buffer in flight
+    if (rc) return rc;
+  }
+  APAR_CUDA(c, launch_append(c->cfg.k_pool, c->cfg.v_pool, k_new, v_new,
+                             (const int32_t*)c->ws(c->lay.slot_map), 0, n, c->cfg.num_kv_heads,
+                             st));
+  c->kernels_total += 2;
+  return run_attention(c, n, sl, tid, false, q, out, sm_scale, st, nullptr, true);
+}
+
+apar_status apar_steps_before_new_block(apar_ctx* c, int32_t* steps_out) {
+  if (!c || !steps_out) return APAR_ERR_INVALID_ARG;
+  if (!step_list_current(c)) return APAR_ERR_INVALID_ARG;
+  int32_t steps = INT32_MAX;
+  for (int32_t s : c->step_slots) {
+    const int32_t r = c->slots[s].len & (kBlock - 1);
+    steps = std::min(steps, r ? kBlock - r : 0);
+  }
+  *steps_out = steps;
+  return APAR_OK;
+}
+
+apar_status apar_note_step_replay(apar_ctx* c) {
+  if (!c) return APAR_ERR_INVALID_ARG;
+  // the device-resident plan and step list must be the ones the replayed kernels were
+  // captured with, and no thread may need a block (the captured step carries none)
+  if (!step_list_current(c) || c->attn_book_seq != c->book_seq || c->plan.items.empty() ||
+      c->plan_tids != c->step_tids)
+    return APAR_ERR_INVALID_ARG;
+  for (int32_t s : c->step_slots)
+    if ((c->slots[s].len & (kBlock - 1)) == 0) return APAR_ERR_INVALID_ARG;
+  for (int32_t s : c->step_slots) {
+    ThreadRec& t = c->slots[s];
+    ++t.len;
+    t.dev_len = t.len;
+  }
+  const int64_t n = (int64_t)c->step_slots.size();
+  c->last.attn_attended_tokens += n;
+  c->last.attn_unique_tokens += n;
+  return APAR_OK;
+}
+
 apar_status apar_tree_decode_attention(apar_ctx* c, int32_t n, const int32_t* tid, const void* q,
                                        void* out, float sm_scale, void* cuda_stream) {
   if (!c || n < 0 || n > c->cfg.max_threads || (n > 0 && (!tid || !q || !out)))
     return APAR_ERR_INVALID_ARG;
+  if (c->host_only) return APAR_ERR_UNSUPPORTED;
   if (n == 0) return APAR_OK;
   std::vector<int32_t> qslots(n);
   const uint32_t mk = next_mark(c);
@@ -723,6 +1008,7 @@ apar_status apar_tree_prefix_attention(apar_ctx* c, int32_t n, const int32_t* ti
                                        float sm_scale, void* cuda_stream) {
   if (!c || n < 0 || n > c->cfg.max_threads || (n > 0 && (!tid || !attend_len || !q || !out)))
     return APAR_ERR_INVALID_ARG;
+  if (c->host_only) return APAR_ERR_UNSUPPORTED;
   if (n == 0) return APAR_OK;
   std::vector<int32_t> qslots(n);
   for (int i = 0; i < n; ++i) {
@@ -741,6 +1027,7 @@ apar_status apar_tree_prefix_attention(apar_ctx* c, int32_t n, const int32_t* ti
 apar_status apar_append_kv_layer(apar_ctx* c, int32_t layer, const void* k_new, const void* v_new,
                                  void* cuda_stream) {
   if (!c || layer < 0 || layer >= c->num_layers || !k_new || !v_new) return APAR_ERR_INVALID_ARG;
+  if (c->host_only) return APAR_ERR_UNSUPPORTED;
   if (c->last_append_rows < 0) return APAR_ERR_WORKSPACE_TOO_SMALL;
   if (c->last_append_rows == 0) return APAR_OK;
   APAR_CUDA(c, launch_append((char*)c->cfg.k_pool + layer * c->layer_bytes,
@@ -754,11 +1041,15 @@ apar_status apar_append_kv_layer(apar_ctx* c, int32_t layer, const void* k_new, 
 apar_status apar_tree_decode_attention_layer(apar_ctx* c, int32_t layer, const void* q, void* out,
                                              float sm_scale, void* cuda_stream) {
   if (!c || layer < 0 || layer >= c->num_layers || !q || !out) return APAR_ERR_INVALID_ARG;
+  if (c->host_only) return APAR_ERR_UNSUPPORTED;
   // the device-resident plan, tables and lengths must still describe the pool
   if (c->attn_book_seq != c->book_seq || c->plan.items.empty()) return APAR_ERR_INVALID_ARG;
   int launches = 0;
+  if (c->time_start) APAR_CUDA(c, cudaEventRecord(c->time_start, (cudaStream_t)cuda_stream));
   apar_status rc = launch_plan(c, layer, q, out, sm_scale, (cudaStream_t)cuda_stream, &launches);
   c->kernels_total += launches;
+  if (rc == APAR_OK && c->time_stop)
+    APAR_CUDA(c, cudaEventRecord(c->time_stop, (cudaStream_t)cuda_stream));
   return rc;
 }
 
@@ -777,6 +1068,7 @@ apar_status apar_release(apar_ctx* c, int32_t n, const int32_t* tid) {
     for (int b = 0; b < t.n_blocks; ++b)
       if (--c->refcnt[tab[b]] == 0) c->free_stack.push_back(tab[b]);
     if (c->cur_node[tid[i]] >= 0) c->pnodes[c->cur_node[tid[i]]].end = t.len;
+    run_release(c, s);
     c->tid_slot[tid[i]] = -1;
     t = ThreadRec();
     c->free_slots.push_back(s);
@@ -784,6 +1076,7 @@ apar_status apar_release(apar_ctx* c, int32_t n, const int32_t* tid) {
   }
   if (n) ++c->struct_epoch;
   ++c->book_seq;
+  ++c->life_seq;
   return APAR_OK;
 }
 
@@ -807,7 +1100,7 @@ apar_status apar_tree_decode_attention_tables(const apar_config* cfg, int32_t n,
   }
   if (n == 0) return APAR_OK;
   apar_ctx* c = nullptr;
-  apar_status rc = create_impl(cfg, true, &c);
+  apar_status rc = create_impl(cfg, true, false, &c);
   if (rc) return rc;
   std::vector<int32_t> qslots(n);
   for (int i = 0; i < n; ++i) {
@@ -902,7 +1195,7 @@ apar_status apar_get_stats(apar_ctx* c, apar_stats* out) {
   out->kernels_total = c->kernels_total;
   out->peak_used_blocks = c->peak_used;
   int32_t flag = 0;   // synchronises with the device: introspection only
-  if (cudaMemcpy(&flag, c->ws(c->lay.err), 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+  if (!c->host_only && cudaMemcpy(&flag, c->ws(c->lay.err), 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
     c->last_cuda = (int32_t)cudaGetLastError();
     return APAR_ERR_CUDA;
   }
@@ -929,6 +1222,45 @@ apar_status apar_check_invariants(apar_ctx* c) {
     }
   }
   if (live != c->live) return APAR_ERR_INVALID_ARG;
+  if (c->track_runs) {
+    // group runs: they tile each table exactly; every thread that lists a group sees it at the
+    // same positions with the same blocks; only a thread's own open group may be longer than
+    // nobody else's view of it (nobody else lists it); reference counts add up
+    struct Seen { int32_t pos, n, first_block, refs; };
+    std::vector<Seen> seen(c->gid_ref.size(), Seen{-1, 0, 0, 0});
+    for (size_t s = 0; s < c->slots.size(); ++s) {
+      const ThreadRec& t = c->slots[s];
+      const std::vector<BlockRun>& rs = c->runs[s];
+      if (t.tid < 0) {
+        if (!rs.empty() || c->own_open[s]) return APAR_ERR_INVALID_ARG;
+        continue;
+      }
+      int32_t pos = 0;
+      for (size_t k = 0; k < rs.size(); ++k) {
+        const BlockRun& r = rs[k];
+        if (r.pos != pos || r.n <= 0 || r.gid < 0 || r.gid >= (int32_t)seen.size())
+          return APAR_ERR_INVALID_ARG;
+        Seen& g = seen[r.gid];
+        const int32_t* tab = c->row((int)s) + r.pos;
+        if (g.refs == 0) {
+          g = Seen{r.pos, r.n, tab[0], 1};
+        } else {
+          if (g.pos != r.pos || g.n != r.n || g.first_block != tab[0]) return APAR_ERR_INVALID_ARG;
+          ++g.refs;
+        }
+        pos += r.n;
+      }
+      if (pos != t.n_blocks) return APAR_ERR_INVALID_ARG;
+      if (c->own_open[s] && (rs.empty() || c->gid_ref[rs.back().gid] != 1))
+        return APAR_ERR_INVALID_ARG;
+      // a partial last block is never shared: it sits in the open group
+      if (t.len % kBlock && !c->own_open[s]) return APAR_ERR_INVALID_ARG;
+    }
+    for (size_t g = 0; g < seen.size(); ++g)
+      if (seen[g].refs != c->gid_ref[g]) return APAR_ERR_INVALID_ARG;
+    for (int32_t g : c->gid_free)
+      if (g < 0 || g >= (int32_t)seen.size() || c->gid_ref[g] != 0) return APAR_ERR_INVALID_ARG;
+  }
   for (int32_t id : c->free_stack) {
     if (id < 0 || id >= nb || count[id] != 0) return APAR_ERR_INVALID_ARG;
     count[id] = -1;                                   // seen in the free list
@@ -988,6 +1320,52 @@ apar_status apar_debug_plan(int32_t num_blocks, int32_t num_q_heads, int32_t num
   return APAR_OK;
 }
 
+apar_status apar_debug_plan_threads(apar_ctx* c, int32_t n, const int32_t* tid, int32_t by_groups,
+                                    int32_t mma_min_rows, int32_t fuse_final, int32_t* items_out,
+                                    int32_t cap_items, int32_t* users_out, int32_t cap_users,
+                                    int32_t* merges_out, int32_t cap_merges, int64_t* counts_out) {
+  if (!c || n <= 0 || !tid || !counts_out || cap_items < 0 || cap_users < 0 || cap_merges < 0 ||
+      (cap_items && !items_out) || (cap_users && !users_out) || (cap_merges && !merges_out))
+    return APAR_ERR_INVALID_ARG;
+  std::vector<PlanQuery> pq(n);
+  const uint32_t mk = next_mark(c);
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, tid[i]);
+    if (s < 0) return APAR_ERR_BAD_THREAD;
+    if (c->slots[s].len == 0) return APAR_ERR_EMPTY_CONTEXT;
+    if (c->mark[s] == mk && by_groups) return APAR_ERR_INVALID_ARG;   // needs distinct threads
+    c->mark[s] = mk;
+    pq[i] = PlanQuery{c->row(s), s, c->slots[s].len};
+    if (by_groups) {
+      pq[i].runs = c->runs[s].data();
+      pq[i].n_runs = (int32_t)c->runs[s].size();
+    }
+  }
+  if (by_groups && !c->track_runs) return APAR_ERR_INVALID_ARG;
+  Plan plan;
+  if (!c->planner.build(pq.data(), n, c->lay.slot_capacity, false, mma_min_rows, fuse_final != 0,
+                        &plan, by_groups != 0))
+    return APAR_ERR_WORKSPACE_TOO_SMALL;
+  c->plan_epoch = 0;            // the planner's scratch was reused: drop the cached plan
+  counts_out[0] = (int64_t)plan.items.size();
+  counts_out[1] = (int64_t)plan.users.size();
+  counts_out[2] = (int64_t)plan.merges.size();
+  counts_out[3] = plan.total_slots;
+  counts_out[4] = plan.unique_tokens;
+  counts_out[5] = plan.attended_tokens;
+  if ((int64_t)cap_items < counts_out[0] || (int64_t)cap_users < counts_out[1] ||
+      (int64_t)cap_merges < counts_out[2])
+    return APAR_ERR_WORKSPACE_TOO_SMALL;
+  if (!plan.items.empty()) memcpy(items_out, plan.items.data(), plan.items.size() * sizeof(WorkItem));
+  if (!plan.users.empty()) memcpy(users_out, plan.users.data(), plan.users.size() * sizeof(UserRef));
+  for (size_t i = 0; i < plan.merges.size(); ++i) {
+    merges_out[3 * i] = plan.merges[i].query;
+    merges_out[3 * i + 1] = plan.merges[i].slot_begin;
+    merges_out[3 * i + 2] = plan.merges[i].n;
+  }
+  return APAR_OK;
+}
+
 apar_status apar_stream_read(const void* src, size_t bytes, void* sink, void* stream) {
   if (!src || !sink || (reinterpret_cast<uintptr_t>(src) & 15) ||
       (reinterpret_cast<uintptr_t>(sink) & 7))
@@ -998,6 +1376,13 @@ apar_status apar_stream_read(const void* src, size_t bytes, void* sink, void* st
     return APAR_ERR_CUDA;
   return launch_stream_read(src, bytes, sink, sms, (cudaStream_t)stream) == cudaSuccess
              ? APAR_OK : APAR_ERR_CUDA;
+}
+
+apar_status apar_set_timing_events(apar_ctx* c, void* start, void* stop) {
+  if (!c || (start == nullptr) != (stop == nullptr)) return APAR_ERR_INVALID_ARG;
+  c->time_start = (cudaEvent_t)start;
+  c->time_stop = (cudaEvent_t)stop;
+  return APAR_OK;
 }
 
 int32_t apar_last_cuda_error(apar_ctx* c) { return c ? c->last_cuda : 0; }

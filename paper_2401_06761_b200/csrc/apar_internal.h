@@ -114,6 +114,13 @@ cudaError_t launch_sync(int32_t* d_tables, int table_stride, int32_t* d_lens,
                         const TableDelta* d_deltas, const int32_t* d_data, int n_deltas,
                         const int32_t* d_len_pairs, int n_pairs, cudaStream_t st);
 
+// One decode step on the device: lens[row] += 1 for the n rows in d_step_rows, slot of each new
+// row into d_slot_map; d_pairs (int4: list position, row, table position, block id) are the
+// blocks the host allocated for threads that start a new block this step.
+cudaError_t launch_step_advance(int32_t* d_tables, int table_stride, int32_t* d_lens,
+                                const int32_t* d_step_rows, int n, const void* d_pairs,
+                                int n_pairs, int32_t* d_slot_map, cudaStream_t st);
+
 struct AttnArgs {
   const void* q; void* out;
   const void* k_pool; const void* v_pool;
@@ -146,10 +153,24 @@ int make_pool_tensor_maps(void* k_pool, void* v_pool, int64_t num_blocks, int nu
 cudaError_t launch_merge(const AttnArgs& a, const MergeRef* d_merge, int n_merge, cudaStream_t st);
 
 // ---- planner (planner.cpp) ----
+// A run of consecutive table positions whose blocks are held by the same set of threads
+// ("group"): blocks become shared only through fork, so the host keeps, per thread, its table
+// as a short list of such runs (see apar_api.cu) and the planner can count per group instead
+// of per block.
+struct BlockRun {
+  int32_t gid;            // group id (dense, recycled)
+  int32_t pos;            // first table position
+  int32_t n;              // blocks
+};
+
 struct PlanQuery {
   const int32_t* table;   // host block ids of the query's thread
   int32_t table_row;      // row in the device table
   int32_t len;            // tokens
+  // optional: the same table as runs of groups; when every query of a call has them (and no
+  // query is listed twice or cut short), the planner walks these instead of the block ids
+  const BlockRun* runs = nullptr;
+  int32_t n_runs = 0;
 };
 
 struct Plan {
@@ -175,11 +196,17 @@ class Planner {
   // Returns false if the partial rows cannot fit `slot_capacity` even without splitting.
   // fuse_final: the last item of a query whose chain ends in a private run of at most 16 rows
   // finishes the query itself (see WorkItem::fin_n); such queries need no merge entry.
+  // by_runs: walk the queries' group runs (keys are group ids) instead of their block ids.
   bool build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_tails,
-             int mma_min_rows, bool fuse_final, Plan* out);
+             int mma_min_rows, bool fuse_final, Plan* out, bool by_runs = false);
+  void set_num_sms(int n) { num_sms_ = n > 0 ? n : 148; }
 
  private:
-  int num_blocks_ = 0, group_ = 1, hint_kv_heads_ = 1;
+  template <bool kRuns>
+  void find_segments(const PlanQuery* q, int n, bool open_tails, int64_t* unique,
+                     int64_t* attended);
+  void ensure_keys(size_t n);
+  int num_blocks_ = 0, group_ = 1, hint_kv_heads_ = 1, num_sms_ = 148;
   uint32_t epoch_ = 0;
   std::vector<uint32_t> stamp_;
   std::vector<int32_t> cnt_, seg_of_;

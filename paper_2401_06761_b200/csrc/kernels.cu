@@ -95,6 +95,45 @@ cudaError_t launch_sync(int32_t* d_tables, int table_stride, int32_t* d_lens,
   return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------ decode step: lengths and slots
+// One thread per entry of the step's thread list: the device length of the thread's table row
+// goes up by one and the pool slot of its new row (block * 16 + offset) is written to the slot
+// map that the scatter kernels of all layers read.  A thread that starts a new block this step
+// gets the block from the host: pair j = (list position, table row, table position, block id),
+// written into the device table here; its slot is the first row of that block.  The two kinds
+// of work touch disjoint words, so one launch does both.
+__global__ void __launch_bounds__(256) step_advance_kernel(int32_t* __restrict__ tables, int stride,
+                                                           int32_t* __restrict__ lens,
+                                                           const int32_t* __restrict__ step_rows,
+                                                           int n, const int4* __restrict__ pairs,
+                                                           int n_pairs,
+                                                           int32_t* __restrict__ slot_map) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) {
+    const int row = step_rows[i];
+    const int len = lens[row];
+    lens[row] = len + 1;
+    if (len & (kBlock - 1))
+      slot_map[i] = tables[(size_t)row * stride + (len >> 4)] * kBlock + (len & (kBlock - 1));
+  }
+  if (i < n_pairs) {
+    const int4 p = pairs[i];
+    tables[(size_t)p.y * stride + p.z] = p.w;
+    slot_map[p.x] = p.w * kBlock;
+  }
+}
+
+cudaError_t launch_step_advance(int32_t* d_tables, int table_stride, int32_t* d_lens,
+                                const int32_t* d_step_rows, int n, const void* d_pairs,
+                                int n_pairs, int32_t* d_slot_map, cudaStream_t st) {
+  const int work = n > n_pairs ? n : n_pairs;
+  if (work <= 0) return cudaSuccess;
+  step_advance_kernel<<<(work + 255) / 256, 256, 0, st>>>(d_tables, table_stride, d_lens,
+                                                          d_step_rows, n, (const int4*)d_pairs,
+                                                          n_pairs, d_slot_map);
+  return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ attention, vector path
 __device__ __forceinline__ void bf16x8_to_float(const uint4& u, float* f) {
   f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xffff0000u);

@@ -30,19 +30,37 @@ void Planner::init(int num_blocks, int group, int num_kv_heads) {
 static inline int64_t round_up16(int64_t x) { return (x + 15) / 16 * 16; }
 constexpr int kMaxFoldedParts = 8;   // partial results a finishing item may fold by itself
 
-bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_tails,
-                    int mma_min_rows, bool fuse_final, Plan* out) {
-  if (++epoch_ == 0) {
-    std::fill(stamp_.begin(), stamp_.end(), 0u);
-    epoch_ = 1;
-  }
-  // ---- pass 1: how many queries list each block; which blocks are ragged for someone
+void Planner::ensure_keys(size_t n) {
+  if (stamp_.size() >= n) return;
+  n = std::max(n, stamp_.size() * 2);
+  stamp_.resize(n, 0);
+  cnt_.resize(n, 0);
+  seg_of_.resize(n, -1);
+  partial_.resize(n, 0);
+}
+
+// Passes 1 and 2: how many queries list each key, then each query's table cut into runs of
+// equal count (segments).  kRuns = false: a key is a block id and an entry one table position.
+// kRuns = true: a key is a group id and an entry one BlockRun; the caller guarantees that no
+// query is listed twice and every query attends its thread's whole chain, so the only ragged
+// block of a query is the last one of its own, unshared group.
+template <bool kRuns>
+void Planner::find_segments(const PlanQuery* q, int n, bool open_tails, int64_t* unique_out,
+                            int64_t* attended_out) {
+  auto n_entries = [&](int i) {
+    return kRuns ? q[i].n_runs : (q[i].len + kBlock - 1) / kBlock;
+  };
+  auto key_of = [&](int i, int e) { return kRuns ? q[i].runs[e].gid : q[i].table[e]; };
+  auto pos_of = [&](int i, int e) { return kRuns ? q[i].runs[e].pos : e; };
+  auto end_of = [&](int i, int e) { return kRuns ? q[i].runs[e].pos + q[i].runs[e].n : e + 1; };
+  // ---- pass 1: how many queries list each key; which blocks are ragged for someone
   int64_t attended = 0;
   for (int i = 0; i < n; ++i) {
-    const int32_t len = q[i].len, nb = (len + kBlock - 1) / kBlock;
-    attended += len;
-    for (int p = 0; p < nb; ++p) {
-      const int32_t b = q[i].table[p];
+    const int ne = n_entries(i);
+    attended += q[i].len;
+    for (int e = 0; e < ne; ++e) {
+      const int32_t b = key_of(i, e);
+      if (kRuns) ensure_keys((size_t)b + 1);
       if (stamp_[b] != epoch_) {
         stamp_[b] = epoch_;
         cnt_[b] = 0;
@@ -51,7 +69,7 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
       }
       ++cnt_[b];
     }
-    if (len % kBlock) partial_[q[i].table[nb - 1]] = 1;
+    if (!kRuns && q[i].len % kBlock) partial_[q[i].table[ne - 1]] = 1;
   }
   // ---- pass 2: runs -> segments; a query's SegUser entries are contiguous, in chain order
   segs_.clear();
@@ -61,19 +79,20 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
   for (int i = 0; i < n; ++i) {
     qbeg_[i] = (int32_t)seg_users_.size();
     const int32_t len = q[i].len, nb = (len + kBlock - 1) / kBlock;
-    const int32_t* tab = q[i].table;
-    int p0 = 0;
-    while (p0 < nb) {
-      const int32_t b0 = tab[p0];
+    const int ne = n_entries(i);
+    int e0 = 0;
+    while (e0 < ne) {
+      const int32_t b0 = key_of(i, e0);
       const bool priv0 = partial_[b0] || cnt_[b0] == 1;
       const int32_t key0 = priv0 ? 0 : cnt_[b0];
-      int p1 = p0 + 1;
-      while (p1 < nb) {
-        const int32_t b = tab[p1];
+      int e1 = e0 + 1;
+      while (e1 < ne) {
+        const int32_t b = key_of(i, e1);
         const int32_t key = (partial_[b] || cnt_[b] == 1) ? 0 : cnt_[b];
         if (key != key0) break;
-        ++p1;
+        ++e1;
       }
+      const int32_t p0 = pos_of(i, e0), p1 = end_of(i, e1 - 1);
       const int32_t t0 = p0 * kBlock, t1 = std::min(p1 * kBlock, len);
       int32_t s = -1;
       if (!priv0) {
@@ -98,14 +117,27 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
       }
       ++segs_[s].n_users;
       seg_users_.push_back(SegUser{s, i, 0});
-      p0 = p1;
+      e0 = e1;
     }
   }
   qbeg_[n] = (int32_t)seg_users_.size();
+  *unique_out = unique;
+  *attended_out = attended;
+}
+
+bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_tails,
+                    int mma_min_rows, bool fuse_final, Plan* out, bool by_runs) {
+  if (++epoch_ == 0) {
+    std::fill(stamp_.begin(), stamp_.end(), 0u);
+    epoch_ = 1;
+  }
+  int64_t unique = 0, attended = 0;
+  if (by_runs) find_segments<true>(q, n, open_tails, &unique, &attended);
+  else find_segments<false>(q, n, open_tails, &unique, &attended);
 
   // ---- chunk length: enough items to fill the machine, never below 128 tokens
   const int64_t kInf = (int64_t)1 << 40;
-  int64_t chunk = std::max<int64_t>(128, round_up16(unique * hint_kv_heads_ / (148 * 8)));
+  int64_t chunk = std::max<int64_t>(128, round_up16(unique * hint_kv_heads_ / (num_sms_ * 8)));
   // `chunk` is sized for the kernels that keep a CTA's loads in flight through TMA rings.  The
   // single-row kernel has no such staging and needs several CTAs per SM to cover the latency:
   // when its runs, dealt out four kv heads to a CTA, would give fewer than four CTAs per SM,
@@ -121,7 +153,7 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
       if (single_row(g))
         vec_chunks += (g.tok_end - g.tok_begin + chunk - 1) / chunk * ((g.n_users + max_users - 1) / max_users);
     const int64_t head_groups = (hint_kv_heads_ + 3) / 4;
-    while (vec_chunks > 0 && vec_div < 8 && vec_chunks * vec_div * head_groups < 4 * 148) vec_div *= 2;
+    while (vec_chunks > 0 && vec_div < 8 && vec_chunks * vec_div * head_groups < 4 * num_sms_) vec_div *= 2;
   }
   auto seg_chunk = [&](const Seg& g) -> int64_t {
     if (chunk >= kInf) return kInf;

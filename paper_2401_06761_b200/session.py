@@ -90,6 +90,17 @@ class PagedSession:
                                      self._stream())
         return out
 
+    def decode_step(self, tids, k_rows: torch.Tensor, v_rows: torch.Tensor, q: torch.Tensor,
+                    out: torch.Tensor = None, sm_scale=None):
+        assert k_rows.is_cuda and k_rows.is_contiguous() and v_rows.is_contiguous()
+        assert q.is_cuda and q.is_contiguous() and q.dtype == torch.bfloat16
+        if out is None:
+            out = torch.empty_like(q)
+        B.apar_decode_step(self.ctx, tids, k_rows.data_ptr(), v_rows.data_ptr(), q.data_ptr(),
+                           out.data_ptr(), self.sm_scale if sm_scale is None else sm_scale,
+                           self._stream())
+        return out
+
     def prefix_attention(self, tids, attend_len, q: torch.Tensor, sm_scale=None):
         assert q.is_cuda and q.is_contiguous() and q.dtype == torch.bfloat16
         out = torch.empty_like(q)

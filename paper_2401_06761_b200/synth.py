@@ -340,6 +340,25 @@ def lifecycle_schedule(seed: int, n_requests: int, n_steps: int, max_live: int =
     return steps, request_of
 
 
+def lifecycle_longest_thread(steps) -> int:
+    """Most tokens any thread of the schedule ever holds (its whole chain), for sizing block
+    tables: a thread starts with its prompt or its parent's length and gains a token per step."""
+    length, live, longest = {}, [], 0
+    for st in steps:
+        for key, _, prompt in st.arrive:
+            length[key] = prompt
+            live.append(key)
+        for parent, child in st.fork:
+            length[child] = length[parent]
+            live.append(child)
+        for key in live:
+            length[key] += 1
+            longest = max(longest, length[key])
+        for key in st.finish:
+            live.remove(key)
+    return longest
+
+
 def run_lifecycle(steps, request_of, backend, rows, early_release: bool = True, on_step=None):
     """Drive `backend` through the schedule.  `rows(n)` supplies (k, v) for n new token rows.
     With early_release a thread's cache is released the moment it finishes (Section 2.3);
