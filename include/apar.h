@@ -188,6 +188,43 @@ apar_status apar_tree_prefix_attention(apar_ctx* ctx, int32_t n, const int32_t* 
                                        const void* q /*[device]*/, void* out /*[device]*/,
                                        float sm_scale, void* cuda_stream);
 
+/* Verification of speculated tokens with tree attention (Section 3.2 "Implementation": the
+ * Medusa setting predicts the next few tokens with extra heads and verifies them in one pass
+ * with a tree mask among the candidates).  Thread tid[i] holds n_cand[i] candidate tokens as the
+ * LAST n_cand[i] rows of its chain (put there with apar_append_kv, n_tok = n_cand[i]).
+ * Candidate j of that thread is one query; it attends every committed token of the chain
+ * (positions below len - n_cand[i], through the shared blocks exactly as in decode attention,
+ * so candidates of sibling threads still read a shared prompt once) and, among the candidates,
+ * exactly those whose bit is set in its mask: bit x of anc_mask means "sees candidate x of the
+ * same thread".  Bit j (itself) must be set; bits >= n_cand[i] must be clear.  A chain of
+ * candidates is a lower-triangular mask, a tree of them sets for each node the bits of its
+ * ancestors.  q, out [device] bf16 [sum n_cand][num_q_heads][128], candidates of tid[0] first.
+ *   n_cand [host] [n], 1..64 each and <= len(tid[i]); anc_mask [host] uint64 [sum n_cand];
+ *   tids distinct; sum n_cand <= max_threads.
+ * Layer 0; apar_tree_decode_attention_layer replays the same verification on other layers.
+ * Errors: INVALID_ARG (also a bad mask), BAD_THREAD, WORKSPACE_TOO_SMALL, CUDA. */
+apar_status apar_tree_verify_attention(apar_ctx* ctx, int32_t n, const int32_t* tid /*[host]*/,
+                                       const int32_t* n_cand /*[host]*/,
+                                       const uint64_t* anc_mask /*[host]*/,
+                                       const void* q /*[device]*/, void* out /*[device]*/,
+                                       float sm_scale, void* cuda_stream);
+/* Outcome of a verification: of the n_cand[i] candidate rows at the end of thread tid[i], the
+ * n_keep[i] rows keep_idx (indices into the candidates, strictly increasing; all threads'
+ * lists one after the other) stay, moved up so that they follow the committed rows in order
+ * (K and V, all kv heads, every layer; by a kernel on the stream), and the thread ends after
+ * them.  Blocks that hold no remaining row go back to the free list in table order.  The
+ * paper's own Medusa path keeps one contiguous cache for a whole batch and therefore masks
+ * mispredicted slots in later attention (Appendix C.1); with a block table per thread every
+ * thread simply keeps its own accepted length, so nothing is ever masked afterwards.
+ * The blocks from the first candidate on must be held by this thread alone (INVALID_ARG if a
+ * fork has shared them since).  tids distinct.
+ * Errors: INVALID_ARG, BAD_THREAD, WORKSPACE_TOO_SMALL, CUDA. */
+apar_status apar_accept_candidates(apar_ctx* ctx, int32_t n, const int32_t* tid /*[host]*/,
+                                   const int32_t* n_cand /*[host]*/,
+                                   const int32_t* n_keep /*[host]*/,
+                                   const int32_t* keep_idx /*[host] [sum n_keep]*/,
+                                   void* cuda_stream);
+
 /* The same decode step for the other attention layers of a model (Algorithm 1's Sample runs
  * every layer over the same sequences; the paper states nothing per layer).  Both calls reuse
  * what the most recent apar_append_kv / apar_tree_decode_attention of this context prepared on

@@ -134,6 +134,32 @@ class BlockModel:
             del self.tables[t]
             del self.lens[t]
 
+    def accept(self, tids, n_cand, n_keep):
+        """Outcome of a predict-verify step (Section 3.2 "Implementation", the Medusa setting):
+        the last n_cand rows of a thread are speculated tokens, n_keep of them are kept (the
+        accepted ones, moved up behind the committed rows) and the rest is dropped.  Blocks
+        that hold no remaining row go back to the pool, in table order.  The blocks from the
+        first candidate on must belong to this thread alone (nobody forked from it meanwhile).
+        Returns nothing: which rows are kept does not matter to the tables."""
+        self._check_live(tids)
+        if len(set(tids)) != len(tids):
+            raise BookkeepingError("INVALID_ARG")
+        B = self.block_size
+        for t, k, keep in zip(tids, n_cand, n_keep):
+            if not (1 <= k <= 64 and k <= self.lens[t] and 0 <= keep <= k):
+                raise BookkeepingError("INVALID_ARG")
+            first = (self.lens[t] - k) // B
+            if any(self.refcount[b] != 1 for b in self.tables[t][first:]):
+                raise BookkeepingError("INVALID_ARG")
+        for t, k, keep in zip(tids, n_cand, n_keep):
+            new_len = self.lens[t] - k + keep
+            blocks = -(-new_len // B)
+            for b in self.tables[t][blocks:]:
+                self.refcount[b] = 0
+                self.free.append(b)
+            del self.tables[t][blocks:]
+            self.lens[t] = new_len
+
     # ------------------------------------------------------------ counters
     def free_list(self):
         """Block ids in the order they would be handed out next."""

@@ -67,6 +67,11 @@ _SIGS = {
                                                C.c_float, C.c_void_p]),
     "apar_tree_prefix_attention": (C.c_int32, [_ctx, C.c_int32, _i32p, _i32p, C.c_void_p,
                                                C.c_void_p, C.c_float, C.c_void_p]),
+    "apar_tree_verify_attention": (C.c_int32, [_ctx, C.c_int32, _i32p, _i32p,
+                                               C.POINTER(C.c_uint64), C.c_void_p, C.c_void_p,
+                                               C.c_float, C.c_void_p]),
+    "apar_accept_candidates": (C.c_int32, [_ctx, C.c_int32, _i32p, _i32p, _i32p, _i32p,
+                                           C.c_void_p]),
     "apar_append_kv_layer": (C.c_int32, [_ctx, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "apar_tree_decode_attention_layer": (C.c_int32, [_ctx, C.c_int32, C.c_void_p, C.c_void_p,
                                                      C.c_float, C.c_void_p]),
@@ -177,6 +182,24 @@ def apar_tree_prefix_attention(ctx, tid, attend_len, q: int, out: int, sm_scale:
     tids, n = _arr(tid)
     lens, _ = _arr(attend_len)
     _check(lib.apar_tree_prefix_attention(ctx, n, tids, lens, q, out, sm_scale, stream))
+
+
+def apar_tree_verify_attention(ctx, tid, n_cand, anc_mask, q: int, out: int, sm_scale: float,
+                               stream=0):
+    """anc_mask: one Python int (uint64 bit mask) per candidate, all threads' candidates in order."""
+    tids, n = _arr(tid)
+    cands, _ = _arr(n_cand)
+    masks = (C.c_uint64 * max(len(anc_mask), 1))(*anc_mask)
+    _check(lib.apar_tree_verify_attention(ctx, n, tids, cands, masks, q, out, sm_scale, stream))
+
+
+def apar_accept_candidates(ctx, tid, n_cand, keep, stream=0):
+    """keep: per thread, the list of candidate indices that stay (increasing)."""
+    tids, n = _arr(tid)
+    cands, _ = _arr(n_cand)
+    counts, _ = _arr([len(k) for k in keep])
+    flat, _ = _arr([x for k in keep for x in k])
+    _check(lib.apar_accept_candidates(ctx, n, tids, cands, counts, flat, stream))
 
 
 def apar_append_kv_layer(ctx, layer: int, k_new: int, v_new: int, stream=0):

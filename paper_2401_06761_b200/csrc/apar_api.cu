@@ -26,7 +26,7 @@ constexpr int kSlotMapRows = 262144;  // new-row slots of the last append kept f
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {            // partition of the caller's workspace
-  size_t err, tables, lens, stage, slot_map, step_rows, plan_items, plan_users, plan_merges, part_ml, part_o, total;
+  size_t err, tables, lens, stage, slot_map, step_rows, verify, plan_items, plan_users, plan_merges, part_ml, part_o, total;
   size_t stage_cap;        // bytes of the transient staging area
   int64_t slot_capacity;   // partial rows (before the head dimension)
   int64_t entry_capacity;  // (item, user) pairs a plan may hold
@@ -58,6 +58,7 @@ Layout make_layout(const apar_config* c) {
   L.stage = take(L.stage_cap);
   L.slot_map = take((size_t)std::max(kSlotMapRows, c->max_threads) * 4);
   L.step_rows = take((size_t)c->max_threads * 4);
+  L.verify = take((size_t)c->max_threads * sizeof(VerifyDesc));
   L.plan_items = take((size_t)L.entry_capacity * sizeof(WorkItem));
   L.plan_users = take((size_t)L.entry_capacity * sizeof(UserRef));
   L.plan_merges = take((size_t)c->max_threads * sizeof(MergeRef));
@@ -125,6 +126,7 @@ struct apar_ctx {
   int num_layers = 1;
   uint64_t book_seq = 1, attn_book_seq = 0;   // bookkeeping calls so far / at the last plan
   int64_t last_append_rows = -1;              // rows of the last append kept in the slot map
+  int plan_verify_n = 0;                      // candidate descriptors that belong to the plan
   int32_t last_cuda = 0;
   bool host_only = false;                     // bookkeeping only: no device, nothing is launched
   // Every thread's table as runs of groups (blocks held by the same set of threads).  A
@@ -433,6 +435,12 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
     APAR_CUDA(c, launch_attention_vec(a, p.n_vec - p.n_vec_final, p.n_vec_final, single_row, st));
     ++*launches_out;
   }
+  // candidate tokens of a verification step: their own partial result per query
+  if (c->plan_verify_n > 0) {
+    APAR_CUDA(c, launch_verify_tail(a, (const VerifyDesc*)c->ws(c->lay.verify), c->plan_verify_n,
+                                    st));
+    ++*launches_out;
+  }
   if (!p.merges.empty()) {
     APAR_CUDA(c, launch_merge(a, (const MergeRef*)c->ws(c->lay.plan_merges),
                               (int)p.merges.size(), st));
@@ -455,7 +463,7 @@ bool plan_reusable(const apar_ctx* c, int n, const int32_t* tids, int64_t attend
 apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32_t* tids,
                           bool has_dups, const void* q, void* out, float sm_scale,
                           cudaStream_t st, const int32_t* qlens = nullptr,
-                          bool tables_in_sync = false) {
+                          bool tables_in_sync = false, std::vector<VerifyDesc>* verify = nullptr) {
   c->last.attn_kernels = 0;
   int64_t attended = 0;
   for (int i = 0; i < n; ++i) attended += qlens ? qlens[i] : c->slots[qslots[i]].len;
@@ -477,14 +485,16 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
         c->pq[i].runs = c->runs[qslots[i]].data();
         c->pq[i].n_runs = (int32_t)c->runs[qslots[i]].size();
       }
+      if (verify) c->pq[i].extra_parts = 1;
     }
+    c->plan_verify_n = 0;
     // Single-row items (no GQA group, private tail): the vector kernel keeps up to 16 CTAs per
     // SM in flight and wins when there are many of them; with few, the warp-stream kernel's
     // deeper per-warp rings do better (measured crossover near 900 queries).
     c->plan_min_rows = c->mma_min_rows;
     if (c->auto_path && c->shape.group == 1 && n <= kFewQueries) c->plan_min_rows = 1;
     // finishing items land in the single-row vector kernel or the warp-stream kernel
-    const bool fuse_final = c->use_ws && c->plan_min_rows <= 2;
+    const bool fuse_final = c->use_ws && c->plan_min_rows <= 2 && !verify;
     if (!c->planner.build(c->pq.data(), n, c->lay.slot_capacity, cacheable, c->plan_min_rows,
                           fuse_final, &c->plan, by_runs))
       return APAR_ERR_WORKSPACE_TOO_SMALL;
@@ -519,6 +529,19 @@ apar_status run_attention(apar_ctx* c, int n, const int32_t* qslots, const int32
         c->last.attn_upload_bytes += (int64_t)chunk;
         done += chunk;
       }
+    }
+    if (verify) {
+      // every candidate's descriptor learns where its partial result goes
+      if ((size_t)n * sizeof(VerifyDesc) > c->ring_bytes) return APAR_ERR_WORKSPACE_TOO_SMALL;
+      for (int i = 0; i < n; ++i) (*verify)[i].slot = p.extra_slot[i];
+      Staging* s;
+      rc = acquire(c, &s);
+      if (rc) return rc;
+      memcpy(s->host, verify->data(), (size_t)n * sizeof(VerifyDesc));
+      rc = send(c, s, c->ws(c->lay.verify), (size_t)n * sizeof(VerifyDesc), st);
+      if (rc) return rc;
+      c->last.attn_upload_bytes += (int64_t)n * sizeof(VerifyDesc);
+      c->plan_verify_n = n;
     }
     if (cacheable) {
       c->plan_tids.assign(tids, tids + n);
@@ -1022,6 +1045,153 @@ apar_status apar_tree_prefix_attention(apar_ctx* c, int32_t n, const int32_t* ti
   }
   return run_attention(c, n, qslots.data(), tid, true, q, out, sm_scale,
                        (cudaStream_t)cuda_stream, attend_len);
+}
+
+apar_status apar_tree_verify_attention(apar_ctx* c, int32_t n, const int32_t* tid,
+                                       const int32_t* n_cand, const uint64_t* anc_mask,
+                                       const void* q, void* out, float sm_scale,
+                                       void* cuda_stream) {
+  if (!c || n < 0 || (n > 0 && (!tid || !n_cand || !anc_mask || !q || !out)))
+    return APAR_ERR_INVALID_ARG;
+  if (c->host_only) return APAR_ERR_UNSUPPORTED;
+  if (n == 0) return APAR_OK;
+  int64_t total = 0;
+  for (int i = 0; i < n; ++i) {
+    if (slot_of(c, tid[i]) < 0) return APAR_ERR_BAD_THREAD;
+    if (n_cand[i] < 1 || n_cand[i] > 64) return APAR_ERR_INVALID_ARG;
+    total += n_cand[i];
+  }
+  if (total > c->cfg.max_threads) return APAR_ERR_INVALID_ARG;
+  const uint32_t mk = next_mark(c);
+  std::vector<int32_t> qslots((size_t)total), qlens((size_t)total);
+  std::vector<VerifyDesc> descs((size_t)total);
+  int64_t seen = 0, k0 = 0;
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, tid[i]);
+    if (c->mark[s] == mk) return APAR_ERR_INVALID_ARG;          // a thread listed twice
+    c->mark[s] = mk;
+    const int32_t k = n_cand[i], len = c->slots[s].len;
+    if (k > len) return APAR_ERR_INVALID_ARG;                   // candidates are appended rows
+    const uint64_t valid = k == 64 ? ~0ull : ((1ull << k) - 1);
+    for (int j = 0; j < k; ++j) {
+      const uint64_t m = anc_mask[k0 + j];
+      if ((m & ~valid) || !((m >> j) & 1ull)) return APAR_ERR_INVALID_ARG;
+      qslots[k0 + j] = s;
+      qlens[k0 + j] = len - k;
+      descs[k0 + j] = VerifyDesc{s, len - k, k, -1, m, (int32_t)(k0 + j), 0};
+      seen += __builtin_popcountll(m);
+    }
+    k0 += k;
+  }
+  apar_status rc = run_attention(c, (int)total, qslots.data(), nullptr, true, q, out, sm_scale,
+                                 (cudaStream_t)cuda_stream, qlens.data(), false, &descs);
+  if (rc == APAR_OK) {
+    c->last.attn_attended_tokens += seen;
+    c->last.attn_unique_tokens += total;
+  }
+  return rc;
+}
+
+apar_status apar_accept_candidates(apar_ctx* c, int32_t n, const int32_t* tid,
+                                   const int32_t* n_cand, const int32_t* n_keep,
+                                   const int32_t* keep_idx, void* cuda_stream) {
+  if (!c || n < 0 || (n > 0 && (!tid || !n_cand || !n_keep))) return APAR_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  for (int i = 0; i < n; ++i)
+    if (slot_of(c, tid[i]) < 0) return APAR_ERR_BAD_THREAD;
+  const uint32_t mk = next_mark(c);
+  int64_t n_moves = 0, n_groups = 0, kofs = 0;
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, tid[i]);
+    if (c->mark[s] == mk) return APAR_ERR_INVALID_ARG;
+    c->mark[s] = mk;
+    const ThreadRec& t = c->slots[s];
+    const int32_t k = n_cand[i], keep = n_keep[i];
+    if (k < 1 || k > 64 || k > t.len || keep < 0 || keep > k || (keep > 0 && !keep_idx))
+      return APAR_ERR_INVALID_ARG;
+    int moved = 0;
+    for (int j = 0; j < keep; ++j) {
+      const int32_t x = keep_idx[kofs + j];
+      if (x < j || x >= k || (j > 0 && x <= keep_idx[kofs + j - 1])) return APAR_ERR_INVALID_ARG;
+      if (x != j) ++moved;
+    }
+    // rows are moved and blocks are given back inside the thread's own tail only
+    const int32_t* tab = c->row(s);
+    for (int b = (t.len - k) / kBlock; b < t.n_blocks; ++b)
+      if (c->refcnt[tab[b]] != 1) return APAR_ERR_INVALID_ARG;
+    n_moves += moved;
+    if (moved) ++n_groups;
+    kofs += keep;
+  }
+  const size_t bytes = (size_t)n_moves * sizeof(RowMove) + (size_t)(n_groups + 1) * 4;
+  if (bytes > c->lay.stage_cap) return APAR_ERR_WORKSPACE_TOO_SMALL;
+  Staging* stg = nullptr;
+  RowMove* moves = nullptr;
+  int32_t* gbeg = nullptr;
+  if (n_moves && !c->host_only) {
+    apar_status rc = acquire(c, &stg);
+    if (rc) return rc;
+    moves = (RowMove*)stg->host;
+    gbeg = (int32_t*)(stg->host + (size_t)n_moves * sizeof(RowMove));
+  }
+  int64_t nm = 0, ng = 0;
+  kofs = 0;
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, tid[i]);
+    ThreadRec& t = c->slots[s];
+    int32_t* tab = c->row(s);
+    const int32_t k = n_cand[i], keep = n_keep[i], base = t.len - k;
+    bool opened = false;
+    for (int j = 0; j < keep; ++j) {
+      const int32_t x = keep_idx[kofs + j];
+      if (x == j) continue;
+      if (moves) {
+        if (!opened) gbeg[ng++] = (int32_t)nm;
+        const int32_t ps = base + x, pd = base + j;
+        moves[nm] = RowMove{tab[ps / kBlock] * kBlock + ps % kBlock,
+                            tab[pd / kBlock] * kBlock + pd % kBlock};
+      }
+      opened = true;
+      ++nm;
+    }
+    kofs += keep;
+    // the thread ends after its last kept row; blocks past that go back to the pool
+    const int32_t new_len = base + keep, new_nb = (new_len + kBlock - 1) / kBlock;
+    for (int b = new_nb; b < t.n_blocks; ++b) {
+      c->refcnt[tab[b]] = 0;
+      c->free_stack.push_back(tab[b]);
+    }
+    std::vector<BlockRun>& rs = c->runs[s];
+    const int32_t open_gid = c->own_open[s] ? rs.back().gid : -1;
+    while (!rs.empty() && rs.back().pos >= new_nb) {
+      if (--c->gid_ref[rs.back().gid] == 0) c->gid_free.push_back(rs.back().gid);
+      rs.pop_back();
+    }
+    if (!rs.empty() && rs.back().pos + rs.back().n > new_nb) rs.back().n = new_nb - rs.back().pos;
+    c->own_open[s] = (open_gid >= 0 && !rs.empty() && rs.back().gid == open_gid) ? 1 : 0;
+    t.len = new_len;
+    t.n_blocks = new_nb;
+    t.synced = std::min(t.synced, new_nb);
+    t.dev_len = -1;
+  }
+  if (n) ++c->struct_epoch;
+  ++c->book_seq;
+  ++c->mod_seq;
+  if (nm && moves) {
+    gbeg[ng] = (int32_t)nm;
+    char* d_stage = c->ws(c->lay.stage);
+    apar_status rc = send(c, stg, d_stage, bytes, st);
+    if (rc) return rc;
+    for (int l = 0; l < c->num_layers; ++l) {
+      APAR_CUDA(c, launch_row_moves((char*)c->cfg.k_pool + l * c->layer_bytes,
+                                    (char*)c->cfg.v_pool + l * c->layer_bytes,
+                                    (const RowMove*)d_stage,
+                                    (const int32_t*)(d_stage + (size_t)n_moves * sizeof(RowMove)),
+                                    (int)ng, c->cfg.num_kv_heads, st));
+      ++c->kernels_total;
+    }
+  }
+  return APAR_OK;
 }
 
 apar_status apar_append_kv_layer(apar_ctx* c, int32_t layer, const void* k_new, const void* v_new,

@@ -56,6 +56,22 @@ struct CowCopy {
   int32_t src_block, dst_block, rows, pad;
 };
 
+// One candidate token of a verification step (a query of its own): it sits at chain position
+// base + index of thread `row`, which holds n_cand candidates from `base` on, and attends,
+// among them, exactly those whose bit is set in `mask` (its own bit included).  The committed
+// prefix [0, base) is covered by ordinary work items; `slot` is where this partial result goes
+// (-1: there is no prefix, write the output).
+struct VerifyDesc {
+  int32_t row, base, n_cand, slot;
+  uint64_t mask;
+  int32_t query, pad;
+};
+
+// Rows to move when candidates are accepted: row src of the thread's chain becomes row dst.
+struct RowMove {
+  int32_t src_slot, dst_slot;     // pool slots (block * 16 + offset)
+};
+
 struct Shape {
   int32_t num_q_heads, num_kv_heads, group;
   int32_t table_stride;        // ints per device table row
@@ -150,6 +166,14 @@ cudaError_t launch_attention_ws(const AttnArgs& a, int item_begin, int n_items, 
 // Returns 0 on success.
 int make_pool_tensor_maps(void* k_pool, void* v_pool, int64_t num_blocks, int num_kv_heads,
                           CUtensorMap* tm_k, CUtensorMap* tm_v);
+// Candidate part of a verification step: one partial result (or the output) per VerifyDesc.
+cudaError_t launch_verify_tail(const AttnArgs& a, const VerifyDesc* d_desc, int n_desc,
+                               cudaStream_t st);
+// Moves token rows inside one layer of the pools (K and V, all kv heads); moves are grouped:
+// group g is moves [begin[g], begin[g+1]) and is carried out as "read all, then write all".
+cudaError_t launch_row_moves(void* k_pool, void* v_pool, const RowMove* d_moves,
+                             const int32_t* d_group_begin, int n_groups, int num_kv_heads,
+                             cudaStream_t st);
 cudaError_t launch_merge(const AttnArgs& a, const MergeRef* d_merge, int n_merge, cudaStream_t st);
 
 // ---- planner (planner.cpp) ----
@@ -171,6 +195,10 @@ struct PlanQuery {
   // query is listed twice or cut short), the planner walks these instead of the block ids
   const BlockRun* runs = nullptr;
   int32_t n_runs = 0;
+  // 1: one more partial result of this query is produced outside the plan's items (the
+  // candidate tokens of a verification step); a slot is reserved for it (Plan::extra_slot)
+  // and the query is merged.  len may then be 0 (nothing but that result).
+  int32_t extra_parts = 0;
 };
 
 struct Plan {
@@ -182,6 +210,7 @@ struct Plan {
   int32_t n_mma_tiles[4] = {0, 0, 0, 0};   // mma items needing 1, 2, 3, 4 query tiles
   std::vector<UserRef> users;
   std::vector<MergeRef> merges;
+  std::vector<int32_t> extra_slot;   // per query with extra_parts: its slot, -1 = writes the output
   int64_t total_slots = 0;         // partial rows (before the head dimension)
   int64_t unique_tokens = 0, attended_tokens = 0;
   int32_t chunk_tokens = 0;

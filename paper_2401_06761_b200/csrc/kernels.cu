@@ -450,6 +450,130 @@ cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items,
   return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------ verification: candidate part
+// One CTA per (candidate query, kv head); warp w takes the query heads w, w + 4, ... of the
+// group.  The candidates are at most 64 rows that were appended a moment ago, so they are read
+// straight from global memory, two tokens per step (one per half-warp, lane c of a half
+// holding dims [8c, 8c + 8) as in the vector path); a token outside the mask is skipped.
+__global__ void __launch_bounds__(128) verify_tail_kernel(const AttnArgs a,
+                                                          const VerifyDesc* __restrict__ descs) {
+  const VerifyDesc d = descs[blockIdx.x];
+  const int kvh = blockIdx.y;
+  const int G = a.shape.group, HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int half = lane >> 4, c = lane & 15;
+  const int32_t* table = a.d_tables + (size_t)d.row * a.shape.table_stride;
+  for (int hg = warp; hg < G; hg += 4) {
+    const int head = kvh * G + hg;
+    float qf[8], o[8];
+    {
+      const uint4 qv = __ldg((const uint4*)a.q + ((size_t)d.query * HQ + head) * 16 + c);
+      bf16x8_to_float(qv, qf);
+#pragma unroll
+      for (int x = 0; x < 8; ++x) { qf[x] *= a.scale_log2e; o[x] = 0.f; }
+    }
+    float m = -INFINITY, l = 0.f;
+    for (int i0 = 0; i0 < d.n_cand; i0 += 2) {
+      const int i = i0 + half;
+      const bool on = i < d.n_cand && ((d.mask >> i) & 1ull);
+      float s = -INFINITY;
+      uint4 vv = make_uint4(0u, 0u, 0u, 0u);
+      if (on) {
+        const int pos = d.base + i;
+        const size_t rowoff =
+            (((size_t)table[pos >> 4] * HKV + kvh) * kBlock + (pos & (kBlock - 1))) * 16 + c;
+        const uint4 kk = ld_stream((const uint4*)a.k_pool + rowoff);
+        vv = ld_stream((const uint4*)a.v_pool + rowoff);
+        float kf[8];
+        bf16x8_to_float(kk, kf);
+        s = 0.f;
+#pragma unroll
+        for (int x = 0; x < 8; ++x) s = fmaf(qf[x], kf[x], s);
+      }
+      // sum over the 16 lanes of a half (both halves shuffle, masked-off ones carry -inf)
+      float t = on ? s : 0.f;
+      t += __shfl_xor_sync(0xffffffffu, t, 8);
+      t += __shfl_xor_sync(0xffffffffu, t, 4);
+      t += __shfl_xor_sync(0xffffffffu, t, 2);
+      t += __shfl_xor_sync(0xffffffffu, t, 1);
+      s = on ? t : -INFINITY;
+      const float other = __shfl_xor_sync(0xffffffffu, s, 16);
+      const float mn = fmaxf(m, fmaxf(s, other));
+      if (mn == -INFINITY) continue;               // both tokens masked, nothing seen yet
+      const float corr = exp2f(m - mn);             // m = -inf gives 0
+      const float p = on ? exp2f(s - mn) : 0.f;
+      const float p_other = other == -INFINITY ? 0.f : exp2f(other - mn);
+      m = mn;
+      l = l * corr + p + p_other;                   // kept identical in both halves
+      float vf[8];
+      bf16x8_to_float(vv, vf);
+#pragma unroll
+      for (int x = 0; x < 8; ++x) o[x] = fmaf(p, vf[x], o[x] * corr);
+    }
+#pragma unroll
+    for (int x = 0; x < 8; ++x) o[x] += __shfl_xor_sync(0xffffffffu, o[x], 16);
+    if (half == 0) {
+      if (d.slot < 0) {
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(o[0] * inv, o[1] * inv);
+        __nv_bfloat162 p1 = __floats2bfloat162_rn(o[2] * inv, o[3] * inv);
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(o[4] * inv, o[5] * inv);
+        __nv_bfloat162 p3 = __floats2bfloat162_rn(o[6] * inv, o[7] * inv);
+        uint4 packed;
+        packed.x = *(uint32_t*)&p0; packed.y = *(uint32_t*)&p1;
+        packed.z = *(uint32_t*)&p2; packed.w = *(uint32_t*)&p3;
+        ((uint4*)((__nv_bfloat16*)a.out + ((size_t)d.query * HQ + head) * kDim))[c] = packed;
+      } else {
+        const size_t prow = (size_t)d.slot * HQ + head;
+        float4* dst = (float4*)(a.part_o + prow * kDim) + 2 * c;
+        dst[0] = make_float4(o[0], o[1], o[2], o[3]);
+        dst[1] = make_float4(o[4], o[5], o[6], o[7]);
+        if (c == 0) a.part_ml[prow] = make_float2(m, l);
+      }
+    }
+  }
+}
+
+cudaError_t launch_verify_tail(const AttnArgs& a, const VerifyDesc* d_desc, int n_desc,
+                               cudaStream_t st) {
+  if (n_desc <= 0) return cudaSuccess;
+  verify_tail_kernel<<<dim3(n_desc, a.shape.num_kv_heads), 128, 0, st>>>(a, d_desc);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ accepted candidates: row moves
+// One CTA per (group of moves, kv head, K|V).  A group holds the rows one thread keeps (at
+// most 64); sources and destinations of a group may overlap, so every source row is read into
+// shared memory before the first destination row is written.
+__global__ void __launch_bounds__(256) row_move_kernel(uint4* __restrict__ k_pool,
+                                                       uint4* __restrict__ v_pool,
+                                                       const RowMove* __restrict__ moves,
+                                                       const int32_t* __restrict__ group_begin,
+                                                       int num_kv_heads) {
+  __shared__ uint4 rows[64 * 16];
+  const int m0 = group_begin[blockIdx.x], m1 = group_begin[blockIdx.x + 1];
+  uint4* pool = blockIdx.z ? v_pool : k_pool;
+  const int h = blockIdx.y;
+  for (int x = threadIdx.x; x < (m1 - m0) * 16; x += blockDim.x) {
+    const int slot = moves[m0 + (x >> 4)].src_slot;
+    rows[x] = pool[(((size_t)(slot >> 4) * num_kv_heads + h) * kBlock + (slot & 15)) * 16 + (x & 15)];
+  }
+  __syncthreads();
+  for (int x = threadIdx.x; x < (m1 - m0) * 16; x += blockDim.x) {
+    const int slot = moves[m0 + (x >> 4)].dst_slot;
+    pool[(((size_t)(slot >> 4) * num_kv_heads + h) * kBlock + (slot & 15)) * 16 + (x & 15)] = rows[x];
+  }
+}
+
+cudaError_t launch_row_moves(void* k_pool, void* v_pool, const RowMove* d_moves,
+                             const int32_t* d_group_begin, int n_groups, int num_kv_heads,
+                             cudaStream_t st) {
+  if (n_groups <= 0) return cudaSuccess;
+  row_move_kernel<<<dim3(n_groups, num_kv_heads, 2), 256, 0, st>>>(
+      (uint4*)k_pool, (uint4*)v_pool, d_moves, d_group_begin, num_kv_heads);
+  return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ staging upload
 // Moves a staged host buffer (pinned, mapped) into device memory with SM loads over PCIe
 // instead of a copy engine.  The library's uploads are small (slot lists, table deltas, plan

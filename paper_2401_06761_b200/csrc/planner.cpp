@@ -172,6 +172,7 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
         seg_users_[k].ord = ord;
         ord += (int32_t)((g.tok_end - g.tok_begin + ck - 1) / ck);
       }
+      ord += q[i].extra_parts;        // results the caller computes itself (see PlanQuery)
       n_parts_[i] = ord;
       if (ord >= 2) total_slots += ord;
     }
@@ -182,6 +183,7 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
 
   // ---- partial slots and merges
   out->merges.clear();
+  out->extra_slot.assign(n, -1);
   part_off_.assign(n, -1);
   int32_t off = 0;
   fused_.assign(n, 0);
@@ -191,8 +193,11 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
       // the chain ends in a private run: its last item can finish the query on its own
       const Seg& last = segs_[seg_users_[qbeg_[i + 1] - 1].seg];
       // (folding is serial work of one CTA: chains cut into many pieces go to the merge kernel)
-      if (fuse_final && last.priv && group_ <= 16 && n_parts_[i] - 1 <= kMaxFoldedParts)
+      if (fuse_final && last.priv && group_ <= 16 && n_parts_[i] - 1 <= kMaxFoldedParts &&
+          q[i].extra_parts == 0)
         fused_[i] = 1;
+      // the caller's own partial result takes the last slot of the query
+      if (q[i].extra_parts) out->extra_slot[i] = off + n_parts_[i] - 1;
       if (!fused_[i]) out->merges.push_back(MergeRef{i, off, n_parts_[i], 0});
       off += n_parts_[i];
     }

@@ -35,6 +35,9 @@ class HostLibrary:
     def release(self, tids):
         B.apar_release(self.ctx, tids)
 
+    def accept(self, tids, n_cand, keep):
+        B.apar_accept_candidates(self.ctx, tids, n_cand, keep, 0)
+
     def close(self):
         B.apar_destroy(self.ctx)
 
@@ -81,11 +84,21 @@ def test_random_replay_matches_the_pool_model(seed):
                 kids, _ = m.fork(parents)
                 assert lib.fork(parents) == kids
                 live += kids
-            elif op < 0.85:
+            elif op < 0.7:
                 sub = rnd.sample(live, rnd.randrange(1, len(live) + 1))
                 cnt = [rnd.choice([0, 1, 1, 1, 2, 15, 16, 17, 40]) for _ in sub]
                 m.append(sub, cnt)
                 lib.append(sub, None if all(c == 1 for c in cnt) else cnt)
+            elif op < 0.85:
+                # predict-verify: speculated rows at the end of some threads, part of them kept
+                sub = rnd.sample(live, rnd.randrange(1, min(4, len(live)) + 1))
+                cnt = [rnd.randrange(1, 40) for _ in sub]
+                m.append(sub, cnt)
+                lib.append(sub, cnt)
+                same_state(lib, m)
+                keep = [sorted(rnd.sample(range(k), rnd.randrange(0, k + 1))) for k in cnt]
+                m.accept(sub, cnt, [len(k) for k in keep])
+                lib.accept(sub, cnt, keep)
             elif len(live) > 2:
                 gone = rnd.sample(live, rnd.randrange(1, 3))
                 m.release(gone)
@@ -96,7 +109,7 @@ def test_random_replay_matches_the_pool_model(seed):
                 if op < 0.3:
                     lib.fork(parents)
                 elif op < 0.85:
-                    lib.append(sub, cnt)
+                    lib.append(sub, cnt)      # (an accept only ever follows its own append)
                 else:
                     lib.release(gone)
             assert le.value.code == e.code
@@ -156,4 +169,36 @@ def test_benchmark_forests_on_the_host(config, nreq, monkeypatch):
     with pytest.raises(B.AparError) as e:
         B.apar_decode_step(lib.ctx, step.live_handles, 0, 0, 0, 0, 1.0, 0)
     assert e.value.code in ("UNSUPPORTED", "INVALID_ARG")
+    lib.close()
+
+
+def test_accept_events_of_the_golden_file_through_the_library():
+    """The hand-worked predict-verify events (tests/golden/accept_candidates.txt), library side."""
+    from test_oracle_bookkeeping import accept_events, load_golden
+    g = load_golden("accept_candidates.txt")
+    lib = HostLibrary(8, 2, g["num_blocks"], 8, 16)
+    in_use, peak = [], []
+    for ev in accept_events():
+        if ev[0] == "new+append":
+            (t,) = lib.new_threads(1)
+            lib.append([t], [ev[1]])
+        elif ev[0] == "append":
+            lib.append([ev[1]], [ev[2]])
+        elif ev[0] == "fork":
+            lib.fork([ev[1]])
+        elif ev[0] == "accept":
+            lib.accept([ev[1]], [ev[2]], [list(range(ev[3]))])
+        else:
+            with pytest.raises(B.AparError) as e:
+                lib.accept([ev[1]], [ev[2]], [list(range(ev[3]))])
+            assert e.value.code == "INVALID_ARG"
+        B.apar_check_invariants(lib.ctx)
+        st = B.apar_get_stats(lib.ctx)
+        in_use.append(st["used_blocks"])
+        peak.append(st["peak_used_blocks"])
+    assert in_use == g["in_use_after_event"] and peak == g["peak_after_event"]
+    for t, table in g["table"].items():
+        assert B.apar_get_thread(lib.ctx, t) == (g["len"][t], table)
+    assert B.apar_get_refcounts(lib.ctx, g["num_blocks"]) == g["refcount"]
+    assert B.apar_get_free_list(lib.ctx, g["num_blocks"]) == g["free_list"]
     lib.close()

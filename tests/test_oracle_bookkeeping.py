@@ -23,7 +23,7 @@ def load_golden(name):
             out[parts[0]][int(parts[1])] = vals if parts[0] == "table" else vals[0]
         elif parts[0] == "copies":
             out["copies"] = [tuple(int(x) for x in c.split()) for c in val.split(",") if c.strip()]
-        elif parts[0] in ("refcount", "in_use_after_event", "peak_after_event"):
+        elif parts[0] in ("refcount", "in_use_after_event", "peak_after_event", "free_list"):
             out[parts[0]] = [int(x) for x in val.split()]
         else:
             out[parts[0]] = int(val)
@@ -195,3 +195,37 @@ def test_failed_calls_change_nothing():
     with pytest.raises(BookkeepingError) as e:
         m2.fork([x, y])                 # needs 2 copies, 1 block free
     assert e.value.code == "NO_BLOCKS" and len(m2.tables) == 2 and len(m2.free) == 1
+
+
+def accept_events():
+    """The events of tests/golden/accept_candidates.txt."""
+    return [("new+append", 37), ("append", 0, 5), ("accept", 0, 5, 2), ("append", 0, 12),
+            ("accept", 0, 12, 1), ("fork", 0), ("append", 0, 30), ("accept", 0, 30, 0),
+            ("append", 1, 10), ("accept", 1, 10, 10), ("accept-refused", 0, 9, 0)]
+
+
+def test_accept_of_speculated_rows_against_the_hand_worked_events():
+    g = load_golden("accept_candidates.txt")
+    m = BlockModel(g["num_blocks"], g["block_size"], 8, 16)
+    in_use, peak = [], []
+    for ev in accept_events():
+        if ev[0] == "new+append":
+            (t,) = m.new_threads(1)
+            m.append([t], [ev[1]])
+        elif ev[0] == "append":
+            m.append([ev[1]], [ev[2]])
+        elif ev[0] == "fork":
+            m.fork([ev[1]])
+        elif ev[0] == "accept":
+            m.accept([ev[1]], [ev[2]], [ev[3]])
+        else:
+            before = (dict(m.lens), {t: list(b) for t, b in m.tables.items()}, list(m.free))
+            with pytest.raises(BookkeepingError) as e:
+                m.accept([ev[1]], [ev[2]], [ev[3]])
+            assert e.value.code == "INVALID_ARG"
+            assert before == (m.lens, m.tables, m.free)
+        in_use.append(m.used_blocks())
+        peak.append(m.peak_used)
+    assert in_use == g["in_use_after_event"] and peak == g["peak_after_event"]
+    assert m.tables == g["table"] and m.lens == g["len"]
+    assert m.refcount == g["refcount"] and m.free_list() == g["free_list"]
