@@ -21,6 +21,8 @@ constexpr int kRing = 12;             // pinned staging buffers in flight: enoug
                                       // while the GPU still runs the one before
 constexpr int kFewQueries = 768;      // up to here single-row items go to the warp-stream kernel
 constexpr int kSlotsPerThread = 6;    // partial-result rows provisioned per live thread
+constexpr int kMinSlots = 1184;       // and never fewer than this (8 per SM of a 148-SM part), so
+                                      // that a few very long threads still spread over the machine
 constexpr int kSlotMapRows = 262144;  // new-row slots of the last append kept for other layers
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -45,9 +47,7 @@ bool supported(const apar_config* c) {
 Layout make_layout(const apar_config* c) {
   Layout L;
   const size_t table_bytes = (size_t)c->max_threads * c->max_blocks_per_thread * 4;
-  // partial rows: several per live thread, and never fewer than one per (SM, resident CTA)
-  // so that a few very long threads can still be spread over the whole machine
-  L.slot_capacity = std::max<int64_t>((int64_t)c->max_threads * kSlotsPerThread, 148 * 8);
+  L.slot_capacity = std::max<int64_t>((int64_t)c->max_threads * kSlotsPerThread, kMinSlots);
   L.entry_capacity = L.slot_capacity + c->max_threads;
   L.stage_cap = std::min<size_t>(std::max<size_t>(table_bytes / 4 + (64 << 10), 1 << 20), 64 << 20);
   size_t off = 0;
@@ -105,7 +105,7 @@ struct apar_ctx {
   // ---- staging
   Staging ring[kRing];
   size_t ring_bytes = 0;
-  int ring_next = 0;
+  int ring_next = 0, ring_n = kRing;   // buffers in use (a one-call context needs few)
   // ---- planning
   Planner planner;
   Plan plan;
@@ -117,7 +117,8 @@ struct apar_ctx {
   int mma_min_rows = INT_MAX;
   int plan_min_rows = INT_MAX;          // the value the current plan was built with
   bool auto_path = true;                // no kernel family forced
-  int umma_min_tiles = 2;               // items with at least this many 16-row tiles use tcgen05
+  int umma_heads = 0;                   // > 0: kv heads per CTA of the tcgen05 kernel (testing)
+  int num_sms = 148;
   int use_pdl = 1;                      // warp-stream launches may start before the kernel before
                                         // them has finished (0: ordinary launches only)
   bool use_ws = true;                   // single-tile items use the warp-stream kernel
@@ -166,7 +167,7 @@ namespace {
 // Next pinned buffer, once the copy that last used it has completed.
 apar_status acquire(apar_ctx* c, Staging** out) {
   Staging* s = &c->ring[c->ring_next];
-  c->ring_next = (c->ring_next + 1) % kRing;
+  c->ring_next = (c->ring_next + 1) % c->ring_n;
   if (s->in_flight) {
     APAR_CUDA(c, cudaEventSynchronize(s->done));
     s->in_flight = false;
@@ -372,6 +373,8 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
   a.tm_k = &c->tm_k[layer];
   a.tm_v = &c->tm_v[layer];
   a.d_error = (int*)c->ws(c->lay.err);
+  a.num_sms = c->num_sms;
+  a.umma_heads = c->umma_heads;
   // The first attention kernel of the call is launched the ordinary way (it starts after the
   // table sync and the append have completed).  A warp-stream launch that follows another
   // attention kernel may start while that kernel is still in its last wave, and orders itself
@@ -382,39 +385,24 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
   const int chain = c->use_pdl ? 1 : 0;
   bool first = true;
   if (p.n_mma) {
-    // items are ordered 4, 3, 2, 1 query tiles: the first umma_min_tiles.. classes go to tcgen05
-    int32_t sync_counts[4], n_umma = 0;
-    for (int k = 0; k < 4; ++k) {
-      const bool umma = k + 1 >= c->umma_min_tiles;
-      sync_counts[k] = umma ? 0 : p.n_mma_tiles[k];
-      if (umma) n_umma += p.n_mma_tiles[k];
-    }
+    // items are ordered 4, 3, 2, 1 query tiles.  Single-tile items (last in the list) go to the
+    // warp-stream kernel, whole items (all kv heads) per CTA, unless the tcgen05 kernel is
+    // forced for everything; their finishing items wait until every other item is launched.
+    const int n_ws = c->use_ws ? p.n_mma_tiles[0] : 0;
+    const int n_umma = p.n_mma - n_ws;
     if (n_umma) {
       a.pdl = 0;
       APAR_CUDA(c, launch_attention_umma(a, p.n_vec, n_umma, st));
       ++*launches_out;
       first = false;
     }
-    if (c->use_ws && sync_counts[0] > 0) {
-      // single-tile items are last in the list: whole items (all kv heads) per CTA; the
-      // finishing ones wait until every other item has been launched
-      const int first_item = p.n_vec + p.n_mma - sync_counts[0];
-      const int n_plain = sync_counts[0] - p.n_mma1_final;
-      if (n_plain > 0) {
-        a.pdl = first ? 0 : chain;
-        APAR_CUDA(c, launch_attention_ws(a, first_item, n_plain, st));
-        ++*launches_out;
-        first = false;
-      }
-      sync_counts[0] = 0;
+    const int n_plain = n_ws - (c->use_ws ? p.n_mma1_final : 0);
+    if (n_plain > 0) {
+      a.pdl = first ? 0 : chain;
+      APAR_CUDA(c, launch_attention_ws(a, p.n_vec + n_umma, n_plain, st));
+      ++*launches_out;
+      first = false;
     }
-    a.pdl = 0;
-    APAR_CUDA(c, launch_attention_mma(a, p.n_vec + n_umma, sync_counts, st));
-    for (int k = 0; k < 4; ++k)
-      if (sync_counts[k] > 0) {
-        ++*launches_out;
-        first = false;
-      }
   }
   const bool single_row = c->shape.group == 1 && c->plan_min_rows <= 2;
   a.pdl = 0;
@@ -603,15 +591,17 @@ apar_status create_impl(const apar_config* cfg, bool external, bool host_only, a
   for (int i = 0; i < cfg->max_threads; ++i) c->free_slots[i] = cfg->max_threads - 1 - i;
   c->mark.assign(cfg->max_threads, 0);
   c->planner.init(cfg->num_blocks, c->shape.group, cfg->num_kv_heads);
-  // APAR_ATTN_PATH (testing aid) forces one kernel family for every item it can take:
-  // "vec" CUDA cores, "mma" mma.sync, "umma" tcgen05.  Default ("auto"): 1 row vec, up to 16
-  // rows warp-stream (mma.sync, whole item per CTA), more rows tcgen05.
+  // Testing switches, read once here.  APAR_ATTN_PATH forces one kernel family for every item
+  // it can take: "vec" CUDA cores only, "umma" tcgen05 for every multi-row item, "ws" the
+  // warp-stream kernel also for single rows.  Default ("auto"): 1 row vector kernel (warp-
+  // stream when the call has few queries), up to 16 rows warp-stream, more rows tcgen05.
   const char* path = getenv("APAR_ATTN_PATH");
   c->mma_min_rows = (path && !strcmp(path, "vec")) ? INT_MAX : (path && !strcmp(path, "ws")) ? 1 : 2;
-  c->umma_min_tiles = (path && !strcmp(path, "mma")) ? 5 : (path && !strcmp(path, "umma")) ? 1 : 2;
-  const char* pdl = getenv("APAR_PDL");                  // testing: 0 = ordinary launches only
+  const char* pdl = getenv("APAR_PDL");                  // 0 = ordinary launches only
   c->use_pdl = pdl ? atoi(pdl) : 1;
-  c->use_ws = !(path && (!strcmp(path, "mma") || !strcmp(path, "umma")));
+  c->use_ws = !(path && !strcmp(path, "umma"));
+  const char* heads = getenv("APAR_UMMA_HEADS");         // kv heads per CTA of the tcgen05 kernel
+  c->umma_heads = heads ? atoi(heads) : 0;
   c->auto_path = !path || !strcmp(path, "auto") || !*path;
   const char* planner = getenv("APAR_PLANNER");          // testing: "tables" = per-block walk
   c->plan_by_runs = !(planner && !strcmp(planner, "tables"));
@@ -621,6 +611,13 @@ apar_status create_impl(const apar_config* cfg, bool external, bool host_only, a
   if (host_only) {
     *out = c;
     return APAR_OK;
+  }
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      c->num_sms = sms;
+    c->planner.set_num_sms(c->num_sms);
   }
   c->tm_k.resize(c->num_layers);
   c->tm_v.resize(c->num_layers);
@@ -634,7 +631,8 @@ apar_status create_impl(const apar_config* cfg, bool external, bool host_only, a
     delete c;
     return APAR_ERR_CUDA;
   }
-  for (int i = 0; i < kRing; ++i) {
+  c->ring_n = external ? 2 : kRing;
+  for (int i = 0; i < c->ring_n; ++i) {
     cudaError_t e = cudaHostAlloc((void**)&c->ring[i].host, c->ring_bytes, cudaHostAllocMapped);
     if (e == cudaSuccess)
       e = cudaHostGetDevicePointer((void**)&c->ring[i].mapped, c->ring[i].host, 0);
@@ -1467,7 +1465,7 @@ apar_status apar_debug_plan(int32_t num_blocks, int32_t num_q_heads, int32_t num
   planner.init(num_blocks, num_q_heads / num_kv_heads, num_kv_heads);
   Plan plan;
   if (!planner.build(pq.data(), n_threads,
-                     std::max<int64_t>((int64_t)kSlotsPerThread * n_threads, 148 * 8), false,
+                     std::max<int64_t>((int64_t)kSlotsPerThread * n_threads, kMinSlots), false,
                      mma_min_rows, fuse_final != 0, &plan))
     return APAR_ERR_WORKSPACE_TOO_SMALL;
   counts_out[0] = (int64_t)plan.items.size();

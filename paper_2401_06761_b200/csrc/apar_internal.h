@@ -151,13 +151,11 @@ struct AttnArgs {
   // 1: this launch is allowed to start before the launch before it on the stream has finished
   // (programmatic dependent launch); its kernel then orders itself with pdl_wait()
   int pdl = 0;
+  int num_sms = 148;                  // of the device the context lives on
+  int umma_heads = 0;                 // > 0: kv heads per CTA of the tcgen05 kernel (testing)
 };
 // single_row: every item carries exactly one query row.
 cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items, bool single_row,
-                                 cudaStream_t st);
-// Tensor-core path.  Items start at item_begin, grouped by the number of 16-row query tiles
-// they need: first counts[3] items with 4 tiles, then counts[2] with 3, counts[1], counts[0].
-cudaError_t launch_attention_mma(const AttnArgs& a, int item_begin, const int32_t* counts,
                                  cudaStream_t st);
 // Blackwell tcgen05/TMEM path for items with up to 64 rows (any number of query tiles).
 cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st);

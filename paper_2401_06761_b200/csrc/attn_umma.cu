@@ -19,13 +19,12 @@
 //              signals completion with tcgen05.commit on mbarriers.  Owns the TMEM allocation.
 // All waits are bounded; a wait that gives up raises an error word and every role unwinds to
 // the common exit where TMEM is released.
-#include <cstdlib>
-
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include "apar_internal.h"
+#include "ptx.cuh"
 
 namespace apar {
 namespace {
@@ -41,7 +40,6 @@ constexpr int kPOff = kQOff + kKV;                 // P operand: [64 rows][64 to
 constexpr int kBarOff = kPOff + kHalf;
 constexpr int kUserOff = kBarOff + 256;             // the item's UserRef entries (at most 64)
 constexpr int kSmem = kUserOff + 64 * 8 + 1024;
-constexpr uint32_t kSpin = 1u << 20;
 constexpr int kTmemCols = 256;                     // S0 | S1 | O
 constexpr int kWavesMin = 6, kHeadsMax = 2;        // see launch_attention_umma
 constexpr float kRefSlack = 8.f;                   // P stays below 2^8 before the reference moves
@@ -50,48 +48,6 @@ enum Bar { KFULL0 = 0, KEMPTY0 = KFULL0 + kKStages, VFULL0 = KEMPTY0 + kKStages,
            VEMPTY0 = VFULL0 + kVStages, SFULL0 = VEMPTY0 + kVStages, SFREE0 = SFULL0 + 2,
            PFULL = SFREE0 + 2, PFREE, QFULL, ODONE, NBARS };
 
-__device__ __forceinline__ uint32_t s32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void bar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void bar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ void bar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool bar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      " selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  On giving up it records where (code = wait site * 1000 + tile) in the error word.
-__device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* cta_abort,
-                                         int* err_word, int code) {
-  for (uint32_t i = 0; i < kSpin; ++i) {
-    if (bar_try(bar, parity)) return true;
-    if ((i & 255) == 255 && *cta_abort) return false;
-  }
-  *cta_abort = 1;
-  atomicCAS(err_word, 0, code);
-  return false;
-}
-__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
-                                       uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"((uint64_t)map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void fence_async_smem() {
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
 __device__ __forceinline__ void tc_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -169,16 +125,6 @@ __device__ __forceinline__ void tmem_wait_st() {
 __device__ __forceinline__ uint32_t swz_off(int row, int c) {   // as in the mma.sync path
   return (uint32_t)((c >> 3) * kHalf + row * 128 + (((c & 7) ^ (row & 7)) << 4));
 }
-__device__ __forceinline__ float ex2(float x) {   // 2^x, flushes to zero, 2^-inf = 0
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *(uint32_t*)&v;
-}
-
 // One CTA owns one work item and `heads_per_cta` consecutive kv heads of it, which it works
 // through one after the other.  All of them share the item's block table, token range and
 // users; only the Q rows and the output rows differ.  The mbarrier phases run on across the
@@ -660,12 +606,11 @@ cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items
   // uneven last waves than the hidden start-up saves (the kernel is bound by HBM, not by the
   // latencies that running on into the next head hides).
   const int hkv = a.shape.num_kv_heads;
-  const char* force = getenv("APAR_UMMA_HEADS");      // testing
   int u = 1;
   for (int c = 2; c <= kHeadsMax && c <= hkv; c *= 2)
     if (hkv % c == 0 && (long long)n_items * (hkv / c) >= (long long)kWavesMin * 2 * sm_count[dev])
       u = c;
-  if (force && atoi(force) >= 1 && hkv % atoi(force) == 0) u = atoi(force);
+  if (a.umma_heads >= 1 && hkv % a.umma_heads == 0) u = a.umma_heads;   // forced (testing)
   return launch_kernel(attn_umma_kernel, dim3(n_items, hkv / u), dim3(192), kSmem, st, a.pdl != 0,
                        *a.tm_k, *a.tm_v, a, item_begin, u);
 }

@@ -17,6 +17,7 @@
 #include <cuda_runtime.h>
 
 #include "apar_internal.h"
+#include "ptx.cuh"
 
 namespace apar {
 namespace {
@@ -27,48 +28,8 @@ constexpr int kRingBytes = 4 * kSlots * kSlotBytes; // 128 KiB
 constexpr int kUsersOffW = kRingBytes;              // UserRef[16]
 constexpr int kBarsOffW = kUsersOffW + 16 * 8;      // full[4][kSlots], empty[4][kSlots]
 constexpr int kSmemW = kBarsOffW + 2 * 4 * kSlots * 8 + 64 + 1024;
-constexpr uint32_t kSpinW = 1u << 20;
 constexpr float kSlack = 8.f;                       // the reference max moves only past 2^8
 
-__device__ __forceinline__ uint32_t sm32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void wb_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void wb_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ void wb_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool wb_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      " selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait; records (site * 1000 + detail) in the error word when it gives up.
-__device__ __forceinline__ bool wb_wait(uint32_t bar, uint32_t parity, volatile int* cta_abort,
-                                        int* err_word, int code) {
-  for (uint32_t i = 0; i < kSpinW; ++i) {
-    if (wb_try(bar, parity)) return true;
-    if ((i & 255) == 255 && *cta_abort) return false;
-  }
-  *cta_abort = 1;
-  atomicCAS(err_word, 0, code);
-  return false;
-}
-__device__ __forceinline__ void tma2d(uint32_t dst, const CUtensorMap* map, int x, int y,
-                                      uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"((uint64_t)map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
 __device__ __forceinline__ void ldsm4(uint32_t addr, uint32_t (&r)[4]) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
@@ -85,15 +46,6 @@ __device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], 
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ float ex2f(float x) {   // 2^x, flushes to zero, 2^-inf = 0
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t packbf(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *(uint32_t*)&v;
-}
 // (row of the block, 16-byte chunk c of 16) inside a [2 halves][16 rows][64 dims] tile written
 // by TMA with the 128-byte swizzle.
 __device__ __forceinline__ uint32_t blk_off(int row, int c) {
@@ -104,8 +56,8 @@ __global__ void __launch_bounds__(160, 2)
 attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                const AttnArgs a, int item_begin, int heads_per_cta) {
   extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (sm32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* bp = smem_raw + (base - sm32(smem_raw));
+  const uint32_t base = (s32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* bp = smem_raw + (base - s32(smem_raw));
   UserRef* s_users = (UserRef*)(bp + kUsersOffW);
   const uint32_t bars = base + kBarsOffW;
   auto full_bar = [&](int w, int s) { return bars + 8u * (w * kSlots + s); };
@@ -131,8 +83,8 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_v) : "memory");
     for (int i = 0; i < 4 * kSlots; ++i) {
-      wb_init(bars + 8u * i, 1);
-      wb_init(bars + 8u * (4 * kSlots + i), 1);
+      bar_init(bars + 8u * i, 1);
+      bar_init(bars + 8u * (4 * kSlots + i), 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -160,11 +112,11 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         if (c + 1 < total) bid_next = table[b1];            // one block ahead of its use
         const int s = c % kSlots;
         if (c >= kSlots &&
-            !wb_wait(empty_bar(w, s), ((c / kSlots) - 1) & 1, cta_abort, a.d_error, 8000 + w))
+            !bar_wait(empty_bar(w, s), ((c / kSlots) - 1) & 1, cta_abort, a.d_error, 8000 + w))
           break;
-        if (op == 0) wb_expect_tx(full_bar(w, s), kSlotBytes);
+        if (op == 0) bar_expect_tx(full_bar(w, s), kSlotBytes);
         const int h = h_begin + w + 4 * hi;
-        tma2d(base + (w * kSlots + s) * kSlotBytes + (op >> 1) * kTileBytes + (op & 1) * 2048, map,
+        tma_2d(base + (w * kSlots + s) * kSlotBytes + (op >> 1) * kTileBytes + (op & 1) * 2048, map,
               (op & 1) * 64, (bid * HKV + h) * kBlock, full_bar(w, s));
         b = b1;
         if (b == 0) ++hi;
@@ -215,7 +167,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 
     for (int b = 0; b < n_blk; ++b, ++c) {
       const int s = c % kSlots;
-      if (!wb_wait(full_bar(w, s), (c / kSlots) & 1, cta_abort, a.d_error, 9000 + w)) {
+      if (!bar_wait(full_bar(w, s), (c / kSlots) & 1, cta_abort, a.d_error, 9000 + w)) {
         alive = false;
         break;
       }
@@ -256,7 +208,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       const bool mv0 = mx0 > ref0 + kSlack || ref0 == -INFINITY;
       const bool mv1 = mx1 > ref1 + kSlack || ref1 == -INFINITY;
       if (__any_sync(0xffffffffu, mv0 || mv1)) {
-        const float f0 = mv0 ? ex2f(ref0 - mx0) : 1.f, f1 = mv1 ? ex2f(ref1 - mx1) : 1.f;
+        const float f0 = mv0 ? ex2(ref0 - mx0) : 1.f, f1 = mv1 ? ex2(ref1 - mx1) : 1.f;
         if (mv0) ref0 = mx0;
         if (mv1) ref1 = mx1;
         l0 *= f0;
@@ -269,15 +221,15 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       float p[2][4];
 #pragma unroll
       for (int n = 0; n < 2; ++n) {
-        p[n][0] = ex2f(sc[n][0] - ref0);
-        p[n][1] = ex2f(sc[n][1] - ref0);
-        p[n][2] = ex2f(sc[n][2] - ref1);
-        p[n][3] = ex2f(sc[n][3] - ref1);
+        p[n][0] = ex2(sc[n][0] - ref0);
+        p[n][1] = ex2(sc[n][1] - ref0);
+        p[n][2] = ex2(sc[n][2] - ref1);
+        p[n][3] = ex2(sc[n][3] - ref1);
       }
       l0 += p[0][0] + p[0][1] + p[1][0] + p[1][1];
       l1 += p[0][2] + p[0][3] + p[1][2] + p[1][3];
-      uint32_t pa[4] = {packbf(p[0][0], p[0][1]), packbf(p[0][2], p[0][3]),
-                        packbf(p[1][0], p[1][1]), packbf(p[1][2], p[1][3])};
+      uint32_t pa[4] = {pack2(p[0][0], p[0][1]), pack2(p[0][2], p[0][3]),
+                        pack2(p[1][0], p[1][1]), pack2(p[1][2], p[1][3])};
       {
         const int row = (jm & 1) * 8 + jr;
 #pragma unroll
@@ -289,7 +241,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         }
       }
       __syncwarp();
-      if (lane == 0) wb_arrive(empty_bar(w, s));
+      if (lane == 0) bar_arrive(empty_bar(w, s));
     }
     if (!alive) break;
     // ---- this head's rows: straight from the accumulator fragments
@@ -315,8 +267,8 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           const float2 ml = a.part_ml[prow];
           const float2* src = (const float2*)(a.part_o + prow * kDim) + tq;
           const float mn = fmaxf(M, ml.x);
-          const float f0 = M == -INFINITY ? 0.f : ex2f(M - mn);
-          const float f1 = ml.x == -INFINITY ? 0.f : ex2f(ml.x - mn);
+          const float f0 = M == -INFINITY ? 0.f : ex2(M - mn);
+          const float f1 = ml.x == -INFINITY ? 0.f : ex2(ml.x - mn);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const float2 x = src[4 * j];
@@ -331,7 +283,7 @@ attn_ws_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
           uint32_t* dst = (uint32_t*)a.out + ((size_t)ur.query * HQ + head) * 64 + tq;
 #pragma unroll
           for (int j = 0; j < 16; ++j)
-            dst[4 * j] = packbf(o[j][2 * half] * inv, o[j][2 * half + 1] * inv);
+            dst[4 * j] = pack2(o[j][2 * half] * inv, o[j][2 * half + 1] * inv);
         } else {
           const size_t prow = (size_t)(ur.slot + it.slot_add) * HQ + head;
           float2* dst = (float2*)(a.part_o + prow * kDim) + tq;
@@ -366,7 +318,7 @@ cudaError_t launch_attention_ws(const AttnArgs& a, int item_begin, int n_items, 
   // heads are dealt out over several CTAs (in multiples of the four consumer warps).
   const int hkv = a.shape.num_kv_heads;
   const int max_groups = (hkv + 3) / 4;
-  const int want = (4 * 148 + n_items - 1) / n_items;
+  const int want = (4 * a.num_sms + n_items - 1) / n_items;
   const int groups = want < 1 ? 1 : (want > max_groups ? max_groups : want);
   const int heads_per_cta = ((hkv + groups - 1) / groups + 3) / 4 * 4;
   const int grid_y = (hkv + heads_per_cta - 1) / heads_per_cta;

@@ -439,7 +439,7 @@ cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items,
     // several CTAs (multiples of the four warps) until the machine is full
     const int hkv = a.shape.num_kv_heads;
     const int max_groups = (hkv + 3) / 4;
-    const int want = (5 * 148 + n_items - 1) / n_items;
+    const int want = (5 * a.num_sms + n_items - 1) / n_items;
     const int groups = want < 1 ? 1 : (want > max_groups ? max_groups : want);
     const int heads_per_cta = ((hkv + groups - 1) / groups + 3) / 4 * 4;
     const dim3 grid(n_items, (hkv + heads_per_cta - 1) / heads_per_cta);

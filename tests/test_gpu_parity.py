@@ -72,7 +72,7 @@ def _make(spec, path, monkeypatch, extra_blocks=0):
     return sess, orc, Both(sess, orc)
 
 
-@pytest.mark.parametrize("path", ["vec", "mma", "umma", "ws", "auto"])
+@pytest.mark.parametrize("path", ["vec", "umma", "ws", "auto"])
 @pytest.mark.parametrize("config,nreq", [(1, 1), (2, 3), (3, 6), (4, 2), (5, 24)])
 def test_config_step_parity(config, nreq, path, monkeypatch):
     spec = synth.forest_spec(config, n_requests=nreq)
@@ -100,7 +100,7 @@ def test_config_step_parity(config, nreq, path, monkeypatch):
     sess.close()
 
 
-@pytest.mark.parametrize("path", ["vec", "mma", "umma", "auto"])
+@pytest.mark.parametrize("path", ["vec", "umma", "ws", "auto"])
 def test_random_event_replay_with_plan_reuse(path, monkeypatch):
     shape = synth.LayerShape(8, 2)
     monkeypatch.setenv("APAR_ATTN_PATH", path)
@@ -146,7 +146,7 @@ def test_random_event_replay_with_plan_reuse(path, monkeypatch):
     sess.close()
 
 
-@pytest.mark.parametrize("path", ["vec", "mma", "umma", "auto"])
+@pytest.mark.parametrize("path", ["vec", "umma", "ws", "auto"])
 @pytest.mark.parametrize("hq,hkv,n_children,prompt", [(4, 4, 40, 100), (16, 2, 12, 333),
                                                       (8, 8, 2, 1), (8, 1, 70, 48)])
 def test_wide_forks(hq, hkv, n_children, prompt, path, monkeypatch):
@@ -173,7 +173,7 @@ def test_wide_forks(hq, hkv, n_children, prompt, path, monkeypatch):
     sess.close()
 
 
-@pytest.mark.parametrize("path", ["vec", "mma", "umma", "auto"])
+@pytest.mark.parametrize("path", ["vec", "umma", "ws", "auto"])
 def test_long_thread_is_split_and_merged(path, monkeypatch):
     shape = synth.LayerShape(8, 2)
     monkeypatch.setenv("APAR_ATTN_PATH", path)
@@ -293,7 +293,7 @@ def test_error_codes_match_the_model_and_change_nothing():
     sess.close()
 
 
-@pytest.mark.parametrize("path", ["vec", "mma", "umma", "auto"])
+@pytest.mark.parametrize("path", ["vec", "umma", "ws", "auto"])
 @pytest.mark.parametrize("hq,hkv,kids", [(4, 4, 5), (16, 2, 6), (8, 8, 1)])
 def test_scores_that_keep_growing_move_the_softmax_reference(hq, hkv, kids, path, monkeypatch):
     """Every later token scores far higher than all earlier ones, so the running maximum rises by

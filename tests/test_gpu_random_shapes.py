@@ -20,7 +20,8 @@ def test_random_forest_random_shape(seed, monkeypatch):
     rnd = random.Random(1000 + seed)
     for case in range(5):
         hq, hkv = rnd.choice(SHAPES)
-        monkeypatch.setenv("APAR_ATTN_PATH", rnd.choice(["auto", "auto", "umma", "ws", "vec", "mma"]))
+        monkeypatch.setenv("APAR_ATTN_PATH", rnd.choice(["auto", "auto", "umma", "ws", "vec"]))
+        monkeypatch.setenv("APAR_PLANNER", rnd.choice(["groups", "groups", "tables"]))
         monkeypatch.setenv("APAR_UMMA_HEADS", rnd.choice(["1", "2", "4", "8"]))
         monkeypatch.setenv("APAR_PDL", rnd.choice(["0", "1"]))
         shape = synth.LayerShape(hq, hkv)
