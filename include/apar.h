@@ -383,7 +383,9 @@ apar_status apar_check_invariants(apar_ctx* ctx);
  *                 run finishes its query (folds the other partial results)
  *   items_out [host] [cap_items][8] int32: table_row, tok_begin, tok_end, user_begin, n_users,
  *             slot_add, fin_n, fin_begin (the fields of a work item; table_row = index of the
- *             thread whose table the item walks)
+ *             thread whose table the item walks; fin_n holds the number of folded partial
+ *             results in its low 8 bits and, from bit 8 on, one bit per folded part that is
+ *             set when that part comes from an item of 2..16 rows)
  *   users_out [host] [cap_users][2] int32: query (thread index), partial slot or -1
  *   merges_out [host] [cap_merges][3] int32: query, first partial slot, number of slots
  *   counts_out [host] [6] int64: items, users, merges, partial slots, unique tokens,

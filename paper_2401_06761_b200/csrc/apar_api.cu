@@ -28,7 +28,7 @@ constexpr int kSlotMapRows = 262144;  // new-row slots of the last append kept f
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {            // partition of the caller's workspace
-  size_t err, tables, lens, stage, slot_map, step_rows, verify, plan_items, plan_users, plan_merges, part_ml, part_o, total;
+  size_t err, ticket, tables, lens, stage, slot_map, step_rows, verify, plan_items, plan_users, plan_merges, part_ml, part_flag, part_o, total;
   size_t stage_cap;        // bytes of the transient staging area
   int64_t slot_capacity;   // partial rows (before the head dimension)
   int64_t entry_capacity;  // (item, user) pairs a plan may hold
@@ -53,6 +53,7 @@ Layout make_layout(const apar_config* c) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   L.err = take(256);
+  L.ticket = take(256);
   L.tables = take(table_bytes);
   L.lens = take((size_t)c->max_threads * 4);
   L.stage = take(L.stage_cap);
@@ -63,6 +64,7 @@ Layout make_layout(const apar_config* c) {
   L.plan_users = take((size_t)L.entry_capacity * sizeof(UserRef));
   L.plan_merges = take((size_t)c->max_threads * sizeof(MergeRef));
   L.part_ml = take((size_t)L.slot_capacity * c->num_q_heads * sizeof(float2));
+  L.part_flag = take((size_t)L.slot_capacity * c->num_q_heads * sizeof(int32_t));
   L.part_o = take((size_t)L.slot_capacity * c->num_q_heads * kDim * sizeof(float));
   L.total = off;
   return L;
@@ -118,6 +120,8 @@ struct apar_ctx {
   int plan_min_rows = INT_MAX;          // the value the current plan was built with
   bool auto_path = true;                // no kernel family forced
   int umma_heads = 0;                   // > 0: kv heads per CTA of the tcgen05 kernel (testing)
+  int umma_mode = 0;                    // 1: one CTA per (item, heads); 2: persistent CTAs
+  int ws_mode = 0;                      // 1: one CTA per item; 2: persistent warps
   int num_sms = 148;
   int use_pdl = 1;                      // warp-stream launches may start before the kernel before
                                         // them has finished (0: ordinary launches only)
@@ -375,6 +379,9 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
   a.d_error = (int*)c->ws(c->lay.err);
   a.num_sms = c->num_sms;
   a.umma_heads = c->umma_heads;
+  a.umma_mode = c->umma_mode;
+  a.ws_mode = c->ws_mode;
+  a.d_ticket = (int*)c->ws(c->lay.ticket);
   // The first attention kernel of the call is launched the ordinary way (it starts after the
   // table sync and the append have completed).  A warp-stream launch that follows another
   // attention kernel may start while that kernel is still in its last wave, and orders itself
@@ -384,11 +391,23 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
   // launched the ordinary way, which also orders them after everything before them.
   const int chain = c->use_pdl ? 1 : 0;
   bool first = true;
+  // unit counters of the persistent kernels, one word per launch; a memset between two
+  // attention kernels would keep the later one from starting early, so all are cleared here
+  APAR_CUDA(c, cudaMemsetAsync(a.d_ticket, 0, 4 * sizeof(int), st));
+  // Single-tile items go to the warp-stream kernel (unless the tcgen05 kernel is forced for
+  // everything).  Its persistent form takes plain and finishing items in ONE launch: the unit
+  // counter hands out the plain ones first, and a finishing unit waits for the ready flag of
+  // each partial result that a plain unit of the same launch produces.
+  const int n_ws = (c->use_ws && p.n_mma) ? p.n_mma_tiles[0] : 0;
+  const int n_ws_final = c->use_ws ? p.n_mma1_final : 0;
+  const bool ws_merged = c->ws_mode != 1 && n_ws_final > 0 && n_ws > n_ws_final;
+  if (ws_merged) {
+    a.part_flag = (int*)c->ws(c->lay.part_flag);
+    APAR_CUDA(c, cudaMemsetAsync(a.part_flag, 0,
+                                 (size_t)p.total_slots * c->shape.num_q_heads * sizeof(int), st));
+  }
   if (p.n_mma) {
-    // items are ordered 4, 3, 2, 1 query tiles.  Single-tile items (last in the list) go to the
-    // warp-stream kernel, whole items (all kv heads) per CTA, unless the tcgen05 kernel is
-    // forced for everything; their finishing items wait until every other item is launched.
-    const int n_ws = c->use_ws ? p.n_mma_tiles[0] : 0;
+    // items are ordered 4, 3, 2, 1 query tiles, finishing items last
     const int n_umma = p.n_mma - n_ws;
     if (n_umma) {
       a.pdl = 0;
@@ -396,14 +415,15 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
       ++*launches_out;
       first = false;
     }
-    const int n_plain = n_ws - (c->use_ws ? p.n_mma1_final : 0);
-    if (n_plain > 0) {
+    const int n_now = ws_merged ? n_ws : n_ws - n_ws_final;
+    if (n_now > 0) {
       a.pdl = first ? 0 : chain;
-      APAR_CUDA(c, launch_attention_ws(a, p.n_vec + n_umma, n_plain, st));
+      APAR_CUDA(c, launch_attention_ws(a, p.n_vec + n_umma, n_now, st, 1));
       ++*launches_out;
       first = false;
     }
   }
+  a.part_flag = nullptr;
   const bool single_row = c->shape.group == 1 && c->plan_min_rows <= 2;
   a.pdl = 0;
   if (p.n_vec - p.n_vec_final > 0) {
@@ -412,9 +432,9 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
     first = false;
   }
   // finishing items: everything they fold has been enqueued before them on this stream
-  if (p.n_mma1_final > 0) {
+  if (p.n_mma1_final > 0 && !ws_merged) {
     a.pdl = first ? 0 : chain;
-    APAR_CUDA(c, launch_attention_ws(a, p.n_vec + p.n_mma - p.n_mma1_final, p.n_mma1_final, st));
+    APAR_CUDA(c, launch_attention_ws(a, p.n_vec + p.n_mma - p.n_mma1_final, p.n_mma1_final, st, 2));
     ++*launches_out;
     first = false;
   }
@@ -602,6 +622,10 @@ apar_status create_impl(const apar_config* cfg, bool external, bool host_only, a
   c->use_ws = !(path && !strcmp(path, "umma"));
   const char* heads = getenv("APAR_UMMA_HEADS");         // kv heads per CTA of the tcgen05 kernel
   c->umma_heads = heads ? atoi(heads) : 0;
+  const char* mode = getenv("APAR_UMMA_MODE");           // "grid" | "persist"
+  c->umma_mode = (mode && !strcmp(mode, "grid")) ? 1 : (mode && !strcmp(mode, "persist")) ? 2 : 0;
+  mode = getenv("APAR_WS_MODE");                         // "grid" | "persist"
+  c->ws_mode = (mode && !strcmp(mode, "grid")) ? 1 : (mode && !strcmp(mode, "persist")) ? 2 : 0;
   c->auto_path = !path || !strcmp(path, "auto") || !*path;
   const char* planner = getenv("APAR_PLANNER");          // testing: "tables" = per-block walk
   c->plan_by_runs = !(planner && !strcmp(planner, "tables"));

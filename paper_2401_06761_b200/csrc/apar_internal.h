@@ -28,8 +28,15 @@ struct WorkItem {
   // fin_n > 0: this is the last item of its (single) query's chain; instead of writing a
   // partial it folds partial slots [fin_begin, fin_begin + fin_n), which earlier launches of
   // the same call completed, into its own state and writes the final output.
+  // Bits 8.. of fin_n: bit (8 + j) is set when folded part j is produced by a single-tile
+  // item, which a multi-row finishing item may share a kernel launch with; the kernel then
+  // waits for that part's ready flag instead of relying on launch order.
   int32_t fin_n, fin_begin;
 };
+__host__ __device__ inline int fin_count(const WorkItem& w) { return w.fin_n & 0xff; }
+__host__ __device__ inline uint32_t fin_same_class(const WorkItem& w) {
+  return (uint32_t)w.fin_n >> 8;
+}
 
 // A query that reads a work item.  slot < 0: the item covers the query's whole chain and
 // writes the final output; otherwise partial row (slot + item.slot_add) receives (m, l, o).
@@ -143,6 +150,9 @@ struct AttnArgs {
   const int32_t* d_tables; const int32_t* d_lens;
   const WorkItem* d_items; const UserRef* d_users;
   float* part_o; float2* part_ml;     // [slots][num_q_heads][128], [slots][num_q_heads]
+  // [slots][num_q_heads] ready flags, or nullptr: set (to 1, after the partial row) by the
+  // plain units of a warp-stream launch that also holds finishing units; cleared by the host
+  int* part_flag = nullptr;
   Shape shape;
   float scale_log2e;                  // sm_scale * log2(e)
   const CUtensorMap* tm_k = nullptr;  // [host] TMA descriptors of the pools (tensor-core path)
@@ -153,6 +163,11 @@ struct AttnArgs {
   int pdl = 0;
   int num_sms = 148;                  // of the device the context lives on
   int umma_heads = 0;                 // > 0: kv heads per CTA of the tcgen05 kernel (testing)
+  int umma_mode = 0;                  // tcgen05 kernel: 0 default, 1 one CTA per (item, heads),
+                                      // 2 persistent CTAs that claim units from *d_ticket
+  int ws_mode = 0;                    // warp-stream kernel: 0 default, 1 one CTA per item, 2 persistent
+  int* d_ticket = nullptr;            // [device] unit counters of the persistent forms (4 words),
+                                      // zeroed before the first attention kernel of a call
 };
 // single_row: every item carries exactly one query row.
 cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items, bool single_row,
@@ -160,7 +175,10 @@ cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items,
 // Blackwell tcgen05/TMEM path for items with up to 64 rows (any number of query tiles).
 cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st);
 // Warp-stream path for items with at most 16 rows per kv head; one CTA per item, all kv heads.
-cudaError_t launch_attention_ws(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st);
+// ticket_index: which word of a.d_ticket the persistent form counts units in (each launch of
+// a call its own: 1 plain items, 2 finishing items; word 0 belongs to the tcgen05 kernel).
+cudaError_t launch_attention_ws(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st,
+                                int ticket_index);
 // Returns 0 on success.
 int make_pool_tensor_maps(void* k_pool, void* v_pool, int64_t num_blocks, int num_kv_heads,
                           CUtensorMap* tm_k, CUtensorMap* tm_v);

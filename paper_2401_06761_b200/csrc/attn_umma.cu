@@ -19,6 +19,8 @@
 //              signals completion with tcgen05.commit on mbarriers.  Owns the TMEM allocation.
 // All waits are bounded; a wait that gives up raises an error word and every role unwinds to
 // the common exit where TMEM is released.
+#include <algorithm>
+
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -582,6 +584,552 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   }
 }
 
+
+// ---------------------------------------------------------------------------- persistent form
+// The same roles and the same per-tile pipeline, but a CTA does not end with its work item: two
+// CTAs per SM stay resident and claim units - one (work item, kv head) each - from a device
+// counter, longest items first.  The producer claims the next unit while the current one is
+// still streaming and publishes its description (item fields, users, first block ids) in a
+// small ring in shared memory, so that across a unit boundary the K/V rings never run dry, the
+// MMA thread issues the next unit's Q K^T while the softmax warps still write the previous
+// unit's rows out, and barrier initialisation, TMEM allocation and CTA start-up are paid once
+// per CTA instead of once per unit.  All four softmax warps take part in every unit (rows past
+// the unit's own are zero queries whose results are dropped), so that every barrier has a
+// fixed number of arrivals whatever the unit's width.
+constexpr int kDescSlots = 3;
+constexpr int kClaimTiles = 8;      // the next unit is claimed this many K tiles before the end
+struct UnitDesc {
+  int32_t table_row, tok_begin, n_tok, n_tiles;     // n_tiles == 0: no more units
+  int32_t kvh, n_users, slot_add, pad;
+  UserRef users[64];
+  int32_t ids[64];                                  // first block ids of the run
+};
+constexpr int kDescOff = kUserOff;
+constexpr int kSmemP = kDescOff + kDescSlots * (int)sizeof(UnitDesc) + 1024;
+enum BarP { DFULL0 = NBARS, DEMPTY0 = DFULL0 + kDescSlots, NBARS_P = DEMPTY0 + kDescSlots };
+static_assert(8 * NBARS_P + 16 <= 256, "barrier area");
+
+__global__ void __launch_bounds__(192, 2)
+attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
+                         const __grid_constant__ CUtensorMap tm_v, const AttnArgs a,
+                         int item_begin, int n_units, int* __restrict__ ticket) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (s32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* bp = smem_raw + (base - s32(smem_raw));
+  const uint32_t bars = base + kBarOff;
+  auto bar = [&](int i) { return bars + 8u * i; };
+  volatile int* cta_abort = (volatile int*)(bp + kBarOff + 8 * NBARS_P);
+  volatile uint32_t* tmem_slot = (volatile uint32_t*)(bp + kBarOff + 8 * NBARS_P + 8);
+  UnitDesc* descs = (UnitDesc*)(bp + kDescOff);
+
+  const int G = a.shape.group, HQ = a.shape.num_q_heads, HKV = a.shape.num_kv_heads;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    *cta_abort = *(volatile int*)a.d_error;
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_k) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_v) : "memory");
+    for (int s = 0; s < kKStages; ++s) {
+      bar_init(bar(KFULL0 + s), 1);
+      bar_init(bar(KEMPTY0 + s), 1);
+    }
+    for (int s = 0; s < kVStages; ++s) {
+      bar_init(bar(VFULL0 + s), 1);
+      bar_init(bar(VEMPTY0 + s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      bar_init(bar(SFULL0 + b), 1);
+      bar_init(bar(SFREE0 + b), 4);
+    }
+    bar_init(bar(PFULL), 4);
+    bar_init(bar(PFREE), 1);
+    bar_init(bar(QFULL), 4);
+    bar_init(bar(ODONE), 4);
+    for (int d = 0; d < kDescSlots; ++d) {
+      bar_init(bar(DFULL0 + d), 1);
+      bar_init(bar(DEMPTY0 + d), 5);               // four softmax warps and the MMA thread
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(s32((const void*)tmem_slot)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  if (*cta_abort) {
+    if (warp == 5)
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem),
+                   "r"(kTmemCols) : "memory");
+    return;
+  }
+  const uint32_t tm_o = tmem + 128u;
+  if (threadIdx.x == 0) pdl_launch_dependents();
+
+  if (warp == 4) {
+    // ---------------------------------------------------------------- producer + unit fetch
+    // Fetch of the next unit, one phase per call so that the global-memory round trips of its
+    // chain (ticket -> work item -> lengths, users, block ids) pass while K/V tiles are issued.
+    int f_phase = 0, f_units = 0;     // descriptors published so far (the end mark included)
+    bool f_end = false;
+    int f_tick = 0;
+    int4 f_item = make_int4(0, 0, 0, 0);
+    int f_row = 0, f_tok_begin = 0, f_tok_end = 0, f_user_begin = 0, f_n_users = 0, f_slot_add = 0;
+    int f_len = 0, f_id0 = 0, f_id1 = 0;
+    UserRef f_u0 = UserRef{0, -1}, f_u1 = UserRef{0, -1};
+    auto fetch_step = [&](bool may_claim) {
+      if (f_phase == 0) {
+        if (f_end || !may_claim) return;
+        if (lane == 0) f_tick = atomicAdd(ticket, 1);
+        f_phase = 1;
+      } else if (f_phase == 1) {
+        f_tick = __shfl_sync(0xffffffffu, f_tick, 0);
+        if (f_tick >= n_units) {
+          f_phase = 3;                              // publish the end mark
+        } else {
+          const int4* ip = (const int4*)(a.d_items + item_begin + f_tick / HKV);
+          if (lane < 2) f_item = __ldg(ip + lane);
+          f_phase = 2;
+        }
+      } else if (f_phase == 2) {
+        f_row = __shfl_sync(0xffffffffu, f_item.x, 0);
+        f_tok_begin = __shfl_sync(0xffffffffu, f_item.y, 0);
+        f_tok_end = __shfl_sync(0xffffffffu, f_item.z, 0);
+        f_user_begin = __shfl_sync(0xffffffffu, f_item.w, 0);
+        f_n_users = __shfl_sync(0xffffffffu, f_item.x, 1);
+        f_slot_add = __shfl_sync(0xffffffffu, f_item.y, 1);
+        if (f_tok_end < 0 && lane == 0) f_len = a.d_lens[f_row];
+        const int32_t* tab = a.d_tables + (size_t)f_row * a.shape.table_stride;
+        const int p0 = f_tok_begin / kBlock + lane;          // stays inside the table row
+        f_id0 = p0 < a.shape.table_stride ? tab[p0] : 0;
+        f_id1 = p0 + 32 < a.shape.table_stride ? tab[p0 + 32] : 0;
+        if (lane < f_n_users) f_u0 = a.d_users[f_user_begin + lane];
+        if (lane + 32 < f_n_users) f_u1 = a.d_users[f_user_begin + lane + 32];
+        f_phase = 3;
+      } else {
+        const int slot = f_units % kDescSlots;
+        int ok = f_units < kDescSlots ||
+                 bar_try(bar(DEMPTY0 + slot), ((f_units / kDescSlots) - 1) & 1);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) return;
+        UnitDesc* d = descs + slot;
+        const bool end = f_tick >= n_units;
+        if (end) {
+          if (lane == 0) d->n_tiles = 0;
+          f_end = true;
+        } else {
+          const int tok_end = f_tok_end < 0 ? __shfl_sync(0xffffffffu, f_len, 0) : f_tok_end;
+          if (lane == 0) {
+            d->table_row = f_row;
+            d->tok_begin = f_tok_begin;
+            d->n_tok = tok_end - f_tok_begin;
+            d->n_tiles = (tok_end - f_tok_begin + kTileTok - 1) / kTileTok;
+            d->kvh = f_tick % HKV;
+            d->n_users = f_n_users;
+            d->slot_add = f_slot_add;
+          }
+          d->ids[lane] = f_id0;
+          d->ids[lane + 32] = f_id1;
+          if (lane < f_n_users) d->users[lane] = f_u0;
+          if (lane + 32 < f_n_users) d->users[lane + 32] = f_u1;
+        }
+        __syncwarp();
+        if (lane == 0) bar_arrive(bar(DFULL0 + slot));
+        ++f_units;
+        f_phase = 0;
+      }
+    };
+
+    // K and V tiles are two independent sequences over the units; each has its own cursor.
+    struct Cursor {
+      int unit = 0, t = 0, n_tiles = 0, n_blk = 0, kvh = 0;   // unit ordinal, tile in the unit
+      bool active = false, done = false;
+      const int32_t* table = nullptr;
+      int id_cur = 0, id_next = 0;
+    } kc, vc;
+    auto open_unit = [&](Cursor& c) {
+      const UnitDesc* d = descs + c.unit % kDescSlots;
+      const int n_tiles = d->n_tiles;
+      if (n_tiles == 0) {
+        c.done = true;
+        return;
+      }
+      c.n_tiles = n_tiles;
+      c.n_blk = (d->n_tok + kBlock - 1) / kBlock;
+      c.kvh = d->kvh;
+      c.table = a.d_tables + (size_t)d->table_row * a.shape.table_stride + d->tok_begin / kBlock;
+      c.id_cur = d->ids[lane];
+      c.id_next = d->ids[lane + 32];
+      c.t = 0;
+      c.active = true;
+    };
+    // Issues tile c.t of the cursor's unit into ring slot (g mod stages) if that slot is free.
+    auto issue = [&](Cursor& c, int g, int stages, int empty0, int full0, uint32_t ring,
+                     const CUtensorMap* map) -> bool {
+      const int s = g % stages;
+      int ready = g < stages || bar_try(bar(empty0 + s), ((g / stages) - 1) & 1);
+      ready = __shfl_sync(0xffffffffu, ready, 0);
+      if (!ready) return false;
+      const int t = c.t;
+      if (t > 0 && (t & 7) == 0) {
+        c.id_cur = c.id_next;
+        const int nxt = (t + 8) * kTileBlocks + lane;
+        c.id_next = nxt < c.n_blk ? c.table[nxt] : 0;
+      }
+      const int blk = t * kTileBlocks + (lane >> 1);
+      const int bid = __shfl_sync(0xffffffffu, c.id_cur, blk & 31);
+      if (lane == 0)
+        bar_expect_tx(bar(full0 + s),
+                      (uint32_t)min(kTileBlocks, c.n_blk - t * kTileBlocks) * kTileBytes);
+      __syncwarp();
+      if (lane < 2 * kTileBlocks && blk < c.n_blk)
+        tma_2d(ring + s * kKV + (lane & 1) * kHalf + (lane >> 1) * (kBlock * 128), map,
+               (lane & 1) * 64, (bid * HKV + c.kvh) * kBlock, bar(full0 + s));
+      if (++c.t == c.n_tiles) {
+        c.active = false;
+        ++c.unit;
+      }
+      return true;
+    };
+
+    int kg = 0, vg = 0;               // tiles issued so far, all units
+    uint32_t idle = 0;
+    // the first unit: its fetch is driven to the end at once
+    for (int i = 0; i < 4 && f_units == 0; ++i) fetch_step(true);
+    while (!vc.done) {
+      bool did = false;
+      if (!kc.active && !kc.done && kc.unit < f_units) open_unit(kc);
+      bool did_k = false;
+      if (kc.active && issue(kc, kg, kKStages, KEMPTY0, KFULL0, base, &tm_k)) {
+        ++kg;
+        did = did_k = true;
+      }
+      if (!vc.active && !vc.done && vc.unit < f_units) open_unit(vc);
+      if (vc.active && issue(vc, vg, kVStages, VEMPTY0, VFULL0, base + kVOff, &tm_v)) {
+        ++vg;
+        did = true;
+      }
+      // claim the next unit towards the end of the K stream of the current one (or at once
+      // when the K cursor has nothing to do); one phase per tile issued or per idle pass
+      const bool near_end = !kc.active || kc.n_tiles - kc.t <= kClaimTiles;
+      const bool room = f_units <= kc.unit + (kc.active ? 1 : 0);
+      if (did_k || !kc.active) fetch_step(near_end && room);
+      if (did) {
+        idle = 0;
+      } else {
+        ++idle;
+        int stop = idle > kSpin || ((idle & 255) == 0 && *cta_abort);
+        if (__shfl_sync(0xffffffffu, stop, 0)) {
+          if (lane == 0 && idle > kSpin) {
+            *cta_abort = 1;
+            atomicCAS(a.d_error, 0, 6000 + (kg % 25) * 40 + vg % 40);
+          }
+          break;
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------------------------------------------------------- MMA issuer
+    constexpr uint32_t kIdescQK = instr_desc(kTileTok, false);
+    constexpr uint32_t kIdescPV = instr_desc(kDim, true);
+    if (lane == 0) {
+      int qk_g = 0, pv_g = 0;                 // tiles issued, all units
+      int qu = 0, qt = 0, q_tiles = -1;       // Q K^T cursor: unit ordinal, tile, tiles (-1: unknown)
+      int pu = 0, pt = 0, p_tiles = -1, p_tok = 0;
+      bool q_done = false;
+      uint32_t idle = 0;
+      while (true) {
+        bool did = false;
+        if (!q_done && q_tiles < 0 && bar_try(bar(DFULL0 + qu % kDescSlots), (qu / kDescSlots) & 1)) {
+          q_tiles = descs[qu % kDescSlots].n_tiles;
+          if (q_tiles == 0) q_done = true;
+        }
+        if (!q_done && q_tiles > 0) {
+          const int g = qk_g, s = g % kKStages, b = g & 1;
+          if (bar_try(bar(KFULL0 + s), (g / kKStages) & 1) &&
+              (g < 2 || bar_try(bar(SFREE0 + b), ((g >> 1) - 1) & 1)) &&
+              (qt > 0 || bar_try(bar(QFULL), qu & 1))) {
+            tc_fence_after();
+            const uint32_t kb = base + s * kKV, qb = base + kQOff;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint32_t off = (ks >> 2) * kHalf + (ks & 3) * 32;
+              umma_bf16(tmem + 64u * b, smem_desc(qb + off, 16, 1024),
+                        smem_desc(kb + off, 16, 1024), kIdescQK, ks > 0);
+            }
+            umma_commit(bar(SFULL0 + b));
+            umma_commit(bar(KEMPTY0 + s));
+            ++qk_g;
+            if (++qt == q_tiles) {
+              qt = 0;
+              ++qu;
+              q_tiles = -1;
+            }
+            did = true;
+          }
+        }
+        if (pv_g < qk_g) {
+          if (p_tiles < 0) {                  // (published: the Q K^T cursor has read it before)
+            p_tiles = descs[pu % kDescSlots].n_tiles;
+            p_tok = descs[pu % kDescSlots].n_tok;
+          }
+          const int g = pv_g, s = g % kVStages;
+          if (bar_try(bar(PFULL), g & 1) && bar_try(bar(VFULL0 + s), (g / kVStages) & 1) &&
+              (pt > 0 || pu == 0 || bar_try(bar(ODONE), (pu - 1) & 1))) {
+            tc_fence_after();
+            const uint32_t vb = base + kVOff + s * kKV, pb = base + kPOff;
+            const int nk = min(kTileBlocks, (p_tok - pt * kTileTok + kBlock - 1) / kBlock);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              if (kk < nk)
+                umma_bf16(tm_o, smem_desc(pb + kk * 32, 16, 1024),
+                          smem_desc(vb + kk * (kBlock * 128), kHalf, 1024), kIdescPV,
+                          (pt | kk) != 0);
+            umma_commit(bar(PFREE));
+            umma_commit(bar(VEMPTY0 + s));
+            ++pv_g;
+            if (++pt == p_tiles) {
+              bar_arrive(bar(DEMPTY0 + pu % kDescSlots));     // done with this description
+              pt = 0;
+              ++pu;
+              p_tiles = -1;
+            }
+            did = true;
+          }
+        }
+        if (q_done && pv_g == qk_g) break;
+        if (did) {
+          idle = 0;
+        } else if (++idle > kSpin || ((idle & 255) == 0 && *cta_abort)) {
+          if (idle > kSpin) atomicCAS(a.d_error, 0, 7000 + (qk_g % 25) * 40 + pv_g % 40);
+          *cta_abort = 1;
+          break;
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------------------------------------------------------- softmax warps 0-3
+    const int row = warp * 16 + (lane & 15);
+    const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+    const float c = a.scale_log2e;
+    const int g8 = lane >> 2, qd = lane & 3;
+    // rows 16w .. 16w+15 of unit description d into the A-operand layout (rows past the unit's
+    // own as zeros)
+    auto stage_q = [&](const UnitDesc* d) {
+      const int R = d->n_users * G, kvh = d->kvh;
+      uint4 qv[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int i = lane + 32 * k, r = warp * 16 + (i >> 4), cc = i & 15;
+        qv[k] = make_uint4(0u, 0u, 0u, 0u);
+        if (r < R)
+          qv[k] = __ldg((const uint4*)a.q +
+                        ((size_t)d->users[r / G].query * HQ + kvh * G + r % G) * 16 + cc);
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int i = lane + 32 * k;
+        *(uint4*)(bp + kQOff + swz_off(warp * 16 + (i >> 4), i & 15)) = qv[k];
+      }
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) bar_arrive(bar(QFULL));
+    };
+    bool alive = bar_wait(bar(DFULL0), 0, cta_abort, a.d_error, 1000);
+    if (alive && descs[0].n_tiles > 0) stage_q(descs);
+    int g0 = 0;                                       // tiles of earlier units
+    for (int u = 0; alive; ++u) {
+      const UnitDesc* d = descs + u % kDescSlots;     // published: waited for below / above
+      const int n_tiles = d->n_tiles;
+      if (n_tiles == 0) break;
+      const int n_tok = d->n_tok, R = d->n_users * G, kvh = d->kvh, slot_add = d->slot_add;
+      float ref_lo = -INFINITY, ref_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+      for (int t = 0; t < n_tiles; ++t) {
+        const int g = g0 + t, b = g & 1;
+        if (!bar_wait(bar(SFULL0 + b), (g >> 1) & 1, cta_abort, a.d_error, 2000 + t % 1000)) {
+          alive = false;
+          break;
+        }
+        tc_fence_after();
+        uint32_t sr[32];
+        TMEM_LD_16x256((tmem + 64u * b) | lane_sel, sr);
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) bar_arrive(bar(SFREE0 + b));
+        const int tile_tok = min(kTileTok, n_tok - t * kTileTok);
+        float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const bool in = 8 * k + 2 * qd + e < tile_tok;
+            const float x_lo = in ? __uint_as_float(sr[4 * k + e]) * c : -INFINITY;
+            const float x_hi = in ? __uint_as_float(sr[4 * k + 2 + e]) * c : -INFINITY;
+            sr[4 * k + e] = __float_as_uint(x_lo);
+            sr[4 * k + 2 + e] = __float_as_uint(x_hi);
+            mx_lo = fmaxf(mx_lo, x_lo);
+            mx_hi = fmaxf(mx_hi, x_hi);
+          }
+        }
+        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+        const bool move_lo = mx_lo > ref_lo + kRefSlack || ref_lo == -INFINITY;
+        const bool move_hi = mx_hi > ref_hi + kRefSlack || ref_hi == -INFINITY;
+        const float new_lo = move_lo ? mx_lo : ref_lo, new_hi = move_hi ? mx_hi : ref_hi;
+        const bool rescale = t > 0 && __any_sync(0xffffffffu, move_lo || move_hi);
+        if (rescale) {
+          if (!bar_wait(bar(PFREE), (g - 1) & 1, cta_abort, a.d_error, 3000 + t % 1000)) {
+            alive = false;
+            break;
+          }
+          tc_fence_after();
+          const float f_lo = move_lo ? ex2(ref_lo - new_lo) : 1.f;
+          const float f_hi = move_hi ? ex2(ref_hi - new_hi) : 1.f;
+          l_lo *= f_lo;
+          l_hi *= f_hi;
+          const float fa = __shfl_sync(0xffffffffu, f_lo, 4 * (lane & 7));
+          const float fb = __shfl_sync(0xffffffffu, f_hi, 4 * (lane & 7));
+          const float f = (lane & 8) ? fb : fa;
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint32_t orow[32];
+            TMEM_LD_32((tm_o + 32u * q4) | lane_sel, orow, 0);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) orow[j] = __float_as_uint(__uint_as_float(orow[j]) * f);
+            TMEM_ST_32((tm_o + 32u * q4) | lane_sel, orow);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+        }
+        ref_lo = new_lo;
+        ref_hi = new_hi;
+        uint32_t pk_lo[8], pk_hi[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const float a0 = ex2(__uint_as_float(sr[4 * k]) - ref_lo);
+          const float a1 = ex2(__uint_as_float(sr[4 * k + 1]) - ref_lo);
+          const float b0 = ex2(__uint_as_float(sr[4 * k + 2]) - ref_hi);
+          const float b1 = ex2(__uint_as_float(sr[4 * k + 3]) - ref_hi);
+          l_lo += a0 + a1;
+          l_hi += b0 + b1;
+          pk_lo[k] = pack2(a0, a1);
+          pk_hi[k] = pack2(b0, b1);
+        }
+        if (g > 0 && !rescale &&
+            !bar_wait(bar(PFREE), (g - 1) & 1, cta_abort, a.d_error, 3000 + t % 1000)) {
+          alive = false;
+          break;
+        }
+        {
+          const int r_lo = warp * 16 + g8;
+          uint8_t* p_lo = bp + kPOff + r_lo * 128 + 4 * qd;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const int off = (k ^ (r_lo & 7)) << 4;
+            *(uint32_t*)(p_lo + off) = pk_lo[k];
+            *(uint32_t*)(p_lo + 8 * 128 + off) = pk_hi[k];
+          }
+        }
+        if (tile_tok < kTileTok && warp == 0) {
+          const int vs = g % kVStages;
+          if (!bar_wait(bar(VFULL0 + vs), (g / kVStages) & 1, cta_abort, a.d_error,
+                        4000 + t % 1000)) {
+            alive = false;
+            break;
+          }
+          uint8_t* vptr = bp + kVOff + vs * kKV;
+          const int first = tile_tok, last = ((tile_tok + kBlock - 1) / kBlock) * kBlock;
+          for (int x = lane; x < (last - first) * 16; x += 32)
+            *(uint4*)(vptr + swz_off(first + (x >> 4), x & 15)) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) bar_arrive(bar(PFULL));
+      }
+      if (!alive) break;
+      // This warp has seen the unit's last S tile, so every Q K^T of the unit has completed:
+      // the next unit's rows can take the Q buffer while the last P V is still running.
+      const UnitDesc* dn = descs + (u + 1) % kDescSlots;
+      if (!bar_wait(bar(DFULL0 + (u + 1) % kDescSlots), ((u + 1) / kDescSlots) & 1, cta_abort,
+                    a.d_error, 1000 + (u + 1) % 1000))
+        break;
+      // the users of this unit are read below: copy what the write-out needs before the
+      // description can be reused (it cannot before this warp's own arrival, see the end)
+      if (dn->n_tiles > 0) stage_q(dn);
+      if (!bar_wait(bar(PFREE), (g0 + n_tiles - 1) & 1, cta_abort, a.d_error, 5000)) break;
+      tc_fence_after();
+      l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+      l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+      l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+      l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+      const float la = __shfl_sync(0xffffffffu, l_lo, 4 * (lane & 7));
+      const float lb = __shfl_sync(0xffffffffu, l_hi, 4 * (lane & 7));
+      const float ra = __shfl_sync(0xffffffffu, ref_lo, 4 * (lane & 7));
+      const float rb = __shfl_sync(0xffffffffu, ref_hi, 4 * (lane & 7));
+      const float l = (lane & 8) ? lb : la, ref = (lane & 8) ? rb : ra;
+      {
+        const bool mine = lane < 16 && row < R;
+        UserRef ur = UserRef{0, -1};
+        if (mine) ur = d->users[row / G];
+        const int head = kvh * G + row % G;
+        const float inv = 1.f / l;
+        uint4* dst_out = (uint4*)((__nv_bfloat16*)a.out + ((size_t)ur.query * HQ + head) * kDim);
+        const size_t prow = (size_t)(ur.slot + slot_add) * HQ + head;
+        float4* dst_part = (float4*)(a.part_o + prow * kDim);
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          uint32_t orow[32];
+          TMEM_LD_32((tm_o + 32u * q4) | lane_sel, orow, 0);
+          tmem_wait_ld();
+          if (mine) {
+            if (ur.slot < 0) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8)
+                dst_out[4 * q4 + (j >> 3)] = make_uint4(
+                    pack2(__uint_as_float(orow[j]) * inv, __uint_as_float(orow[j + 1]) * inv),
+                    pack2(__uint_as_float(orow[j + 2]) * inv, __uint_as_float(orow[j + 3]) * inv),
+                    pack2(__uint_as_float(orow[j + 4]) * inv, __uint_as_float(orow[j + 5]) * inv),
+                    pack2(__uint_as_float(orow[j + 6]) * inv, __uint_as_float(orow[j + 7]) * inv));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                dst_part[8 * q4 + (j >> 2)] =
+                    make_float4(__uint_as_float(orow[j]), __uint_as_float(orow[j + 1]),
+                                __uint_as_float(orow[j + 2]), __uint_as_float(orow[j + 3]));
+            }
+          }
+        }
+        if (mine && ur.slot >= 0) a.part_ml[prow] = make_float2(ref, l);
+      }
+      // O has been read and this unit's description is no longer needed by this warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        bar_arrive(bar(ODONE));
+        bar_arrive(bar(DEMPTY0 + u % kDescSlots));
+      }
+      g0 += n_tiles;
+    }
+  }
+  // ---- common exit: every role arrives here, then the allocating warp frees TMEM
+  if (a.pdl && threadIdx.x == 0) pdl_wait();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem),
+                 "r"(kTmemCols) : "memory");
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items,
@@ -596,16 +1144,26 @@ cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items
     cudaError_t e = cudaFuncSetAttribute(attn_umma_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_umma_persist_kernel,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemP);
+    if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
+  }
+  const int hkv = a.shape.num_kv_heads;
+  if (a.umma_mode != 1 && a.d_ticket != nullptr) {
+    // persistent form: two resident CTAs per SM claim (item, kv head) units from a counter
+    const long long n_units = (long long)n_items * hkv;
+    const int grid = (int)std::min<long long>(n_units, 2LL * sm_count[dev]);
+    return launch_kernel(attn_umma_persist_kernel, dim3(grid), dim3(192), kSmemP, st,
+                         a.pdl != 0, *a.tm_k, *a.tm_v, a, item_begin, (int)n_units, a.d_ticket);
   }
   // Heads per CTA: up to kHeadsMax, if that leaves at least kWavesMin CTAs for each of the
   // machine's CTA slots (two per SM), so that the hardware scheduler can still even out the
   // load.  Measured: two heads per CTA take 2-3 % off the kernel, four or eight cost more in
   // uneven last waves than the hidden start-up saves (the kernel is bound by HBM, not by the
   // latencies that running on into the next head hides).
-  const int hkv = a.shape.num_kv_heads;
   int u = 1;
   for (int c = 2; c <= kHeadsMax && c <= hkv; c *= 2)
     if (hkv % c == 0 && (long long)n_items * (hkv / c) >= (long long)kWavesMin * 2 * sm_count[dev])

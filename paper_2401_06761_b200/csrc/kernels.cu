@@ -395,7 +395,7 @@ __global__ void __launch_bounds__(128) attn_vec_heads_kernel(const AttnArgs a, i
     for (int d = 0; d < 8; ++d) o[d] += __shfl_xor_sync(0xffffffffu, o[d], 16);
     if (half == 0) {
       // a finishing item folds the partial results of the rest of the chain into its own
-      for (int j = 0; j < it.fin_n; ++j) {
+      for (int j = 0; j < fin_count(it); ++j) {
         const size_t prow = (size_t)(it.fin_begin + j) * HQ + h;
         const float2 ml = a.part_ml[prow];
         const float4* src = (const float4*)(a.part_o + prow * kDim) + 2 * c;
@@ -410,7 +410,7 @@ __global__ void __launch_bounds__(128) attn_vec_heads_kernel(const AttnArgs a, i
         l = l * f0 + ml.y * f1;
         m = mn;
       }
-      if (ur.slot < 0 || it.fin_n > 0) {
+      if (ur.slot < 0 || fin_count(it) > 0) {
         const float inv = l > 0.f ? 1.f / l : 0.f;      // no tokens at all: zeros
         __nv_bfloat162 p0 = __floats2bfloat162_rn(o[0] * inv, o[1] * inv);
         __nv_bfloat162 p1 = __floats2bfloat162_rn(o[2] * inv, o[3] * inv);

@@ -243,7 +243,27 @@ bool Planner::build(const PlanQuery* q, int n, int64_t slot_capacity, bool open_
           // private runs hold exactly one query; is this the end of a fused query's chain?
           const int qi = out->users[g.user_off].query;
           if (fused_[qi] && g.tok_end == q[qi].len) {
-            it.fin_n = n_parts_[qi] - 1;
+            // which of the folded parts come from single-tile items (same kernel class as a
+            // multi-row finishing item, hence possibly the same launch): bit = part ordinal
+            uint32_t same_class = 0;
+            for (int k = qbeg_[qi]; k < qbeg_[qi + 1]; ++k) {
+              const Seg& sg = segs_[seg_users_[k].seg];
+              int nu_k = sg.n_users;
+              if (sg.n_users > max_users) {           // wide run: the user group that holds qi
+                int j = 0;
+                while (j < sg.n_users && out->users[sg.user_off + j].query != qi) ++j;
+                nu_k = std::min(max_users, sg.n_users - j / max_users * max_users);
+              }
+              const int rows_k = nu_k * group_;
+              if (rows_k < mma_min_rows || rows_k > 16) continue;
+              const int32_t nck = (int32_t)((sg.tok_end - sg.tok_begin + seg_chunk(sg) - 1) /
+                                            seg_chunk(sg));
+              for (int x = 0; x < nck; ++x) {
+                const int part = seg_users_[k].ord + x;
+                if (part < n_parts_[qi] - 1) same_class |= 1u << part;
+              }
+            }
+            it.fin_n = (n_parts_[qi] - 1) | (int32_t)(same_class << 8);
             it.fin_begin = part_off_[qi];
             (to_mma ? mma1_final_ : vec_final_).push_back(it);
             continue;

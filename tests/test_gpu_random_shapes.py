@@ -22,6 +22,8 @@ def test_random_forest_random_shape(seed, monkeypatch):
         hq, hkv = rnd.choice(SHAPES)
         monkeypatch.setenv("APAR_ATTN_PATH", rnd.choice(["auto", "auto", "umma", "ws", "vec"]))
         monkeypatch.setenv("APAR_PLANNER", rnd.choice(["groups", "groups", "tables"]))
+        monkeypatch.setenv("APAR_UMMA_MODE", rnd.choice(["persist", "grid"]))
+        monkeypatch.setenv("APAR_WS_MODE", rnd.choice(["persist", "grid"]))
         monkeypatch.setenv("APAR_UMMA_HEADS", rnd.choice(["1", "2", "4", "8"]))
         monkeypatch.setenv("APAR_PDL", rnd.choice(["0", "1"]))
         shape = synth.LayerShape(hq, hkv)

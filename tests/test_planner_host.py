@@ -99,7 +99,13 @@ def check_plan(m, threads, hq, hkv, mma_min_rows, fuse_final):
         rows_used |= set(slots)
         last = items[parts[-1][3]]
         if last[6]:                           # the chain's last item finishes the query
-            assert last[6] == len(parts) - 1 and last[7] == slots[0] and q not in merged
+            assert last[6] & 0xff == len(parts) - 1 and last[7] == slots[0] and q not in merged
+            # bits 8..: the folded parts that come from single-tile items (2..16 rows), which
+            # may share a kernel launch with the finishing item
+            g = hq // hkv
+            want = sum(1 << j for j, p in enumerate(parts[:-1])
+                       if mma_min_rows <= items[p[3]][4] * g <= 16)
+            assert last[6] >> 8 == want
         else:
             assert merged[q] == (slots[0], len(parts))
         for p in parts[:-1]:
