@@ -225,6 +225,27 @@ apar_status apar_accept_candidates(apar_ctx* ctx, int32_t n, const int32_t* tid 
                                    const int32_t* keep_idx /*[host] [sum n_keep]*/,
                                    void* cuda_stream);
 
+/* Tree-masked attention for whole runs of consecutive tokens: prompt prefill into the paged
+ * pool and the training mask of Section 2.2 (Fig. 2: a token attends the tokens of its
+ * ancestors and, causally, those of its own node).  Segment i is the q_count[i] tokens of
+ * thread tid[i] at chain positions q_begin[i] .. q_begin[i] + q_count[i] - 1 (their K, V rows
+ * must already be in the pool: append first); the query at position p attends positions
+ * 0 .. p of that thread's chain.  A prompt is one segment from position 0; every node of a
+ * paragraph tree is one segment of its thread that starts where the node's own tokens start.
+ * q, out [device] bf16 [sum q_count][num_q_heads][128], segments in order.  The queries of a
+ * segment are processed 64 rows at a time (64 / group tokens x group heads) on the tensor
+ * cores; a tile reads its chain once for all of its rows and masks every row at its own
+ * position.  Any number of queries per call (they are launched in batches that fit the
+ * workspace); `layer` selects the pool layer.  Invalidates the cached decode plan.
+ * Errors: INVALID_ARG (also a range outside the thread), BAD_THREAD, WORKSPACE_TOO_SMALL (more
+ * than 12 x max_threads x num_q_heads queries in one call), CUDA. */
+apar_status apar_tree_prefill_attention(apar_ctx* ctx, int32_t layer, int32_t n,
+                                        const int32_t* tid /*[host]*/,
+                                        const int32_t* q_begin /*[host]*/,
+                                        const int32_t* q_count /*[host]*/,
+                                        const void* q /*[device]*/, void* out /*[device]*/,
+                                        float sm_scale, void* cuda_stream);
+
 /* The same decode step for the other attention layers of a model (Algorithm 1's Sample runs
  * every layer over the same sequences; the paper states nothing per layer).  Both calls reuse
  * what the most recent apar_append_kv / apar_tree_decode_attention of this context prepared on

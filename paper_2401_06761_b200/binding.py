@@ -72,6 +72,8 @@ _SIGS = {
                                                C.c_float, C.c_void_p]),
     "apar_accept_candidates": (C.c_int32, [_ctx, C.c_int32, _i32p, _i32p, _i32p, _i32p,
                                            C.c_void_p]),
+    "apar_tree_prefill_attention": (C.c_int32, [_ctx, C.c_int32, C.c_int32, _i32p, _i32p, _i32p,
+                                                C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]),
     "apar_append_kv_layer": (C.c_int32, [_ctx, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "apar_tree_decode_attention_layer": (C.c_int32, [_ctx, C.c_int32, C.c_void_p, C.c_void_p,
                                                      C.c_float, C.c_void_p]),
@@ -200,6 +202,15 @@ def apar_accept_candidates(ctx, tid, n_cand, keep, stream=0):
     counts, _ = _arr([len(k) for k in keep])
     flat, _ = _arr([x for k in keep for x in k])
     _check(lib.apar_accept_candidates(ctx, n, tids, cands, counts, flat, stream))
+
+
+def apar_tree_prefill_attention(ctx, layer: int, tid, q_begin, q_count, q: int, out: int,
+                                sm_scale: float, stream=0):
+    tids, n = _arr(tid)
+    begins, _ = _arr(q_begin)
+    counts, _ = _arr(q_count)
+    _check(lib.apar_tree_prefill_attention(ctx, layer, n, tids, begins, counts, q, out, sm_scale,
+                                           stream))
 
 
 def apar_append_kv_layer(ctx, layer: int, k_new: int, v_new: int, stream=0):

@@ -391,9 +391,6 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
   // launched the ordinary way, which also orders them after everything before them.
   const int chain = c->use_pdl ? 1 : 0;
   bool first = true;
-  // unit counters of the persistent kernels, one word per launch; a memset between two
-  // attention kernels would keep the later one from starting early, so all are cleared here
-  APAR_CUDA(c, cudaMemsetAsync(a.d_ticket, 0, 4 * sizeof(int), st));
   // Single-tile items go to the warp-stream kernel (unless the tcgen05 kernel is forced for
   // everything).  Its persistent form takes plain and finishing items in ONE launch: the unit
   // counter hands out the plain ones first, and a finishing unit waits for the ready flag of
@@ -401,11 +398,9 @@ apar_status launch_plan(apar_ctx* c, int layer, const void* q, void* out, float 
   const int n_ws = (c->use_ws && p.n_mma) ? p.n_mma_tiles[0] : 0;
   const int n_ws_final = c->use_ws ? p.n_mma1_final : 0;
   const bool ws_merged = c->ws_mode != 1 && n_ws_final > 0 && n_ws > n_ws_final;
-  if (ws_merged) {
-    a.part_flag = (int*)c->ws(c->lay.part_flag);
-    APAR_CUDA(c, cudaMemsetAsync(a.part_flag, 0,
-                                 (size_t)p.total_slots * c->shape.num_q_heads * sizeof(int), st));
-  }
+  // (flags and unit counters look after themselves: the flags carry the number of the launch
+  // that wrote them, the counters are put back to zero by the last warp of a launch)
+  if (ws_merged) a.part_flag = (int*)c->ws(c->lay.part_flag);
   if (p.n_mma) {
     // items are ordered 4, 3, 2, 1 query tiles, finishing items last
     const int n_umma = p.n_mma - n_ws;
@@ -650,7 +645,10 @@ apar_status create_impl(const apar_config* cfg, bool external, bool host_only, a
     maps_ok = make_pool_tensor_maps((char*)cfg->k_pool + l * c->layer_bytes,
                                     (char*)cfg->v_pool + l * c->layer_bytes, cfg->num_blocks,
                                     cfg->num_kv_heads, &c->tm_k[l], &c->tm_v[l]) == 0;
-  if (!maps_ok || cudaMemset(c->ws(lay.err), 0, 256) != cudaSuccess) {
+  if (!maps_ok || cudaMemset(c->ws(lay.err), 0, 256) != cudaSuccess ||
+      cudaMemset(c->ws(lay.ticket), 0, 256) != cudaSuccess ||
+      cudaMemset(c->ws(lay.part_flag), 0,
+                 (size_t)lay.slot_capacity * cfg->num_q_heads * sizeof(int32_t)) != cudaSuccess) {
     c->last_cuda = (int32_t)cudaGetLastError();
     delete c;
     return APAR_ERR_CUDA;
@@ -1213,6 +1211,159 @@ apar_status apar_accept_candidates(apar_ctx* c, int32_t n, const int32_t* tid,
       ++c->kernels_total;
     }
   }
+  return APAR_OK;
+}
+
+apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
+                                        const int32_t* tid, const int32_t* q_begin,
+                                        const int32_t* q_count, const void* q, void* out,
+                                        float sm_scale, void* cuda_stream) {
+  if (!c || n < 0 || layer < 0 || layer >= c->num_layers ||
+      (n > 0 && (!tid || !q_begin || !q_count || !q || !out)))
+    return APAR_ERR_INVALID_ARG;
+  if (c->host_only) return APAR_ERR_UNSUPPORTED;
+  if (n == 0) return APAR_OK;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  std::vector<int32_t> seg_slot(n);
+  int64_t total_q = 0, attended = 0;
+  for (int i = 0; i < n; ++i) {
+    const int s = slot_of(c, tid[i]);
+    if (s < 0) return APAR_ERR_BAD_THREAD;
+    if (q_begin[i] < 0 || q_count[i] < 1 ||
+        (int64_t)q_begin[i] + q_count[i] > c->slots[s].len)
+      return APAR_ERR_INVALID_ARG;
+    seg_slot[i] = s;
+    total_q += q_count[i];
+    attended += (int64_t)q_count[i] * q_begin[i] + (int64_t)q_count[i] * (q_count[i] + 1) / 2;
+  }
+  if (total_q > INT32_MAX) return APAR_ERR_INVALID_ARG;
+  apar_status rc = sync_device_tables(c, seg_slot.data(), n, st);
+  if (rc) return rc;
+  c->plan_epoch = 0;                    // the plan area of the workspace is reused below
+  c->attn_book_seq = 0;
+  c->plan_verify_n = 0;
+
+  // Work items: the queries of a segment in tiles of 64 rows (64 / group tokens); a tile reads
+  // the chain from its start to the tile's last token once, for all of its rows, and every row
+  // stops at its own position (the mask is applied by the kernel).  Longest tiles first.
+  const int G = c->shape.group, per_tile = std::max(1, kMaxRowsPerItem / G);
+  struct Tile { int32_t seg, first, count; };
+  std::vector<Tile> tiles;
+  for (int i = 0; i < n; ++i)
+    for (int j = 0; j < q_count[i]; j += per_tile)
+      tiles.push_back(Tile{i, j, std::min(per_tile, q_count[i] - j)});
+  std::stable_sort(tiles.begin(), tiles.end(), [&](const Tile& x, const Tile& y) {
+    return q_begin[x.seg] + x.first + x.count > q_begin[y.seg] + y.first + y.count;
+  });
+  std::vector<int64_t> seg_qbase(n);
+  {
+    int64_t b = 0;
+    for (int i = 0; i < n; ++i) { seg_qbase[i] = b; b += q_count[i]; }
+  }
+  AttnArgs a;
+  a.q = q;
+  a.out = out;
+  a.k_pool = (const char*)c->cfg.k_pool + (size_t)layer * c->layer_bytes;
+  a.v_pool = (const char*)c->cfg.v_pool + (size_t)layer * c->layer_bytes;
+  a.d_tables = (const int32_t*)c->ws(c->lay.tables);
+  a.d_lens = (const int32_t*)c->ws(c->lay.lens);
+  a.d_items = (const WorkItem*)c->ws(c->lay.plan_items);
+  a.d_users = (const UserRef*)c->ws(c->lay.plan_users);
+  a.part_o = (float*)c->ws(c->lay.part_o);
+  a.part_ml = nullptr;
+  a.shape = c->shape;
+  a.scale_log2e = sm_scale * 1.4426950408889634f;
+  a.tm_k = &c->tm_k[layer];
+  a.tm_v = &c->tm_v[layer];
+  a.d_error = (int*)c->ws(c->lay.err);
+  a.num_sms = c->num_sms;
+  a.d_ticket = (int*)c->ws(c->lay.ticket);
+  // visible length per query, indexed by query number: the partial-result area is free here
+  // (every tile covers its rows' whole chains, so nothing is merged)
+  int32_t* d_limit = (int32_t*)c->ws(c->lay.part_ml);
+  a.q_limit = d_limit;
+
+  auto upload = [&](const void* src, size_t bytes, char* dst) -> apar_status {
+    size_t done = 0;
+    while (done < bytes) {
+      Staging* s;
+      apar_status r = acquire(c, &s);
+      if (r) return r;
+      const size_t chunk = std::min(bytes - done, c->ring_bytes);
+      memcpy(s->host, (const char*)src + done, chunk);
+      r = send(c, s, dst + done, chunk, st);
+      if (r) return r;
+      done += chunk;
+    }
+    return APAR_OK;
+  };
+  // batches that fit the plan area; limits are addressed by the global query number, so the
+  // limit array is uploaded whole, in pieces of the area's size if need be (then batch by batch)
+  const int64_t cap = c->lay.entry_capacity;
+  const int64_t limit_cap = c->lay.slot_capacity * c->shape.num_q_heads * 2;
+  if (total_q > limit_cap) return APAR_ERR_WORKSPACE_TOO_SMALL;
+  std::vector<int32_t> limits((size_t)total_q);
+  for (int i = 0; i < n; ++i)
+    for (int j = 0; j < q_count[i]; ++j) limits[(size_t)(seg_qbase[i] + j)] = q_begin[i] + j + 1;
+  rc = upload(limits.data(), limits.size() * 4, (char*)d_limit);
+  if (rc) return rc;
+  std::vector<WorkItem> items;
+  std::vector<UserRef> users;
+  int launches = 0;
+  c->last.attn_work_items = 0;
+  size_t t0 = 0;
+  while (t0 < tiles.size()) {
+    items.clear();
+    users.clear();
+    size_t t1 = t0;
+    while (t1 < tiles.size() && (int64_t)users.size() + tiles[t1].count <= cap &&
+           (int64_t)items.size() < cap) {
+      const Tile& t = tiles[t1];
+      WorkItem it;
+      it.table_row = seg_slot[t.seg];
+      it.tok_begin = 0;
+      it.tok_end = q_begin[t.seg] + t.first + t.count;
+      it.user_begin = (int32_t)users.size();
+      it.n_users = t.count;
+      it.slot_add = 0;
+      it.fin_n = it.fin_begin = 0;
+      items.push_back(it);
+      for (int k = 0; k < t.count; ++k)
+        users.push_back(UserRef{(int32_t)(seg_qbase[t.seg] + t.first + k), -1});
+      ++t1;
+    }
+    rc = upload(items.data(), items.size() * sizeof(WorkItem), c->ws(c->lay.plan_items));
+    if (rc) return rc;
+    rc = upload(users.data(), users.size() * sizeof(UserRef), c->ws(c->lay.plan_users));
+    if (rc) return rc;
+    if (c->time_start && t0 == 0) APAR_CUDA(c, cudaEventRecord(c->time_start, st));
+    APAR_CUDA(c, launch_attention_umma(a, 0, (int)items.size(), st));
+    ++launches;
+    c->last.attn_work_items += (int64_t)items.size();
+    t0 = t1;
+  }
+  if (c->time_stop) APAR_CUDA(c, cudaEventRecord(c->time_stop, st));
+  c->kernels_total += launches;
+  c->last.attn_kernels = launches;
+  c->last.attn_threads = total_q;
+  c->last.attn_attended_tokens = attended;
+  int64_t unique = 0;                   // rows of the pools that are read: per listed thread,
+  {                                     // its chain up to the last query position
+    const uint32_t mk = next_mark(c);
+    std::vector<int32_t> reach(c->slots.size(), 0);
+    for (int i = 0; i < n; ++i)
+      reach[seg_slot[i]] = std::max(reach[seg_slot[i]], q_begin[i] + q_count[i]);
+    for (int i = 0; i < n; ++i)
+      if (c->mark[seg_slot[i]] != mk) {
+        c->mark[seg_slot[i]] = mk;
+        unique += reach[seg_slot[i]];
+      }
+  }
+  c->last.attn_unique_tokens = unique;
+  c->last.attn_partials = 0;
+  c->last.attn_plan_reused = 0;
+  c->last.attn_vec_items = 0;
+  c->last.attn_mma_items = c->last.attn_work_items;
   return APAR_OK;
 }
 

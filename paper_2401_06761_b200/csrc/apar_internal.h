@@ -150,8 +150,8 @@ struct AttnArgs {
   const int32_t* d_tables; const int32_t* d_lens;
   const WorkItem* d_items; const UserRef* d_users;
   float* part_o; float2* part_ml;     // [slots][num_q_heads][128], [slots][num_q_heads]
-  // [slots][num_q_heads] ready flags, or nullptr: set (to 1, after the partial row) by the
-  // plain units of a warp-stream launch that also holds finishing units; cleared by the host
+  // [slots][num_q_heads] ready flags, or nullptr: written (after the partial row, with the
+  // launch's own mark) by the plain units of a warp-stream launch that also holds finishing units
   int* part_flag = nullptr;
   Shape shape;
   float scale_log2e;                  // sm_scale * log2(e)
@@ -165,9 +165,13 @@ struct AttnArgs {
   int umma_heads = 0;                 // > 0: kv heads per CTA of the tcgen05 kernel (testing)
   int umma_mode = 0;                  // tcgen05 kernel: 0 default, 1 one CTA per (item, heads),
                                       // 2 persistent CTAs that claim units from *d_ticket
+  // [device] per query: how many tokens of its chain it sees (position + 1); non-null selects
+  // the tree-mask (prefill) form of the tcgen05 kernel
+  const int32_t* q_limit = nullptr;
   int ws_mode = 0;                    // warp-stream kernel: 0 default, 1 one CTA per item, 2 persistent
-  int* d_ticket = nullptr;            // [device] unit counters of the persistent forms (4 words),
-                                      // zeroed before the first attention kernel of a call
+  int* d_ticket = nullptr;            // [device] counters of the persistent forms, zero when no
+                                      // launch is in flight: words 0-2 tcgen05 kernel, 4-6 and
+                                      // 8-10 warp-stream launches (unit counter, leavers, launches)
 };
 // single_row: every item carries exactly one query row.
 cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items, bool single_row,
@@ -175,8 +179,8 @@ cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items,
 // Blackwell tcgen05/TMEM path for items with up to 64 rows (any number of query tiles).
 cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st);
 // Warp-stream path for items with at most 16 rows per kv head; one CTA per item, all kv heads.
-// ticket_index: which word of a.d_ticket the persistent form counts units in (each launch of
-// a call its own: 1 plain items, 2 finishing items; word 0 belongs to the tcgen05 kernel).
+// ticket_index: which group of four words of a.d_ticket the persistent form uses (1 or 2; group
+// 0 belongs to the tcgen05 kernel).
 cudaError_t launch_attention_ws(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st,
                                 int ticket_index);
 // Returns 0 on success.

@@ -609,6 +609,10 @@ constexpr int kSmemP = kDescOff + kDescSlots * (int)sizeof(UnitDesc) + 1024;
 enum BarP { DFULL0 = NBARS, DEMPTY0 = DFULL0 + kDescSlots, NBARS_P = DEMPTY0 + kDescSlots };
 static_assert(8 * NBARS_P + 16 <= 256, "barrier area");
 
+// kCausal: every query has its own visible length (AttnArgs::q_limit, in chain positions): a
+// key at or beyond it is masked out for that row.  This is the tree mask of prefill / training
+// attention, where the queries of a unit are consecutive tokens of one node.
+template <bool kCausal>
 __global__ void __launch_bounds__(192, 2)
 attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
                          const __grid_constant__ CUtensorMap tm_v, const AttnArgs a,
@@ -664,6 +668,13 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
     if (warp == 5)
       asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem),
                    "r"(kTmemCols) : "memory");
+    if (threadIdx.x == 128) {                 // keeps the launch's exit count complete
+      const int gone = atomicAdd(ticket + 1, 1);
+      if (gone == (int)gridDim.x - 1) {
+        ticket[0] = 0;
+        ticket[1] = 0;
+      }
+    }
     return;
   }
   const uint32_t tm_o = tmem + 128u;
@@ -831,6 +842,15 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
         }
       }
     }
+    // ticket[0] unit counter, ticket[1] producers that have stopped claiming: the last one puts
+    // both back to zero, so that nothing has to be cleared between launches
+    if (lane == 0) {
+      const int gone = atomicAdd(ticket + 1, 1);
+      if (gone == (int)gridDim.x - 1) {
+        ticket[0] = 0;
+        ticket[1] = 0;
+      }
+    }
   } else if (warp == 5) {
     // ---------------------------------------------------------------- MMA issuer
     constexpr uint32_t kIdescQK = instr_desc(kTileTok, false);
@@ -919,8 +939,15 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
     const int g8 = lane >> 2, qd = lane & 3;
     // rows 16w .. 16w+15 of unit description d into the A-operand layout (rows past the unit's
     // own as zeros)
+    int lim_lo_next = 0, lim_hi_next = 0;             // visible keys of rows g8 / g8 + 8,
+                                                      // relative to the unit's first token
     auto stage_q = [&](const UnitDesc* d) {
       const int R = d->n_users * G, kvh = d->kvh;
+      if (kCausal) {
+        const int r_lo = warp * 16 + g8, r_hi = r_lo + 8;
+        lim_lo_next = r_lo < R ? a.q_limit[d->users[r_lo / G].query] - d->tok_begin : d->n_tok;
+        lim_hi_next = r_hi < R ? a.q_limit[d->users[r_hi / G].query] - d->tok_begin : d->n_tok;
+      }
       uint4 qv[8];
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
@@ -947,6 +974,7 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
       const int n_tiles = d->n_tiles;
       if (n_tiles == 0) break;
       const int n_tok = d->n_tok, R = d->n_users * G, kvh = d->kvh, slot_add = d->slot_add;
+      const int lim_lo = lim_lo_next, lim_hi = lim_hi_next;    // (of this unit: staged with its Q)
       float ref_lo = -INFINITY, ref_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
       for (int t = 0; t < n_tiles; ++t) {
         const int g = g0 + t, b = g & 1;
@@ -962,14 +990,17 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
         __syncwarp();
         if (lane == 0) bar_arrive(bar(SFREE0 + b));
         const int tile_tok = min(kTileTok, n_tok - t * kTileTok);
+        // keys of this tile a row may see: all that exist, or (tree mask) those before its limit
+        const int see_lo = kCausal ? min(tile_tok, lim_lo - t * kTileTok) : tile_tok;
+        const int see_hi = kCausal ? min(tile_tok, lim_hi - t * kTileTok) : tile_tok;
         float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
-            const bool in = 8 * k + 2 * qd + e < tile_tok;
-            const float x_lo = in ? __uint_as_float(sr[4 * k + e]) * c : -INFINITY;
-            const float x_hi = in ? __uint_as_float(sr[4 * k + 2 + e]) * c : -INFINITY;
+            const bool in_lo = 8 * k + 2 * qd + e < see_lo, in_hi = 8 * k + 2 * qd + e < see_hi;
+            const float x_lo = in_lo ? __uint_as_float(sr[4 * k + e]) * c : -INFINITY;
+            const float x_hi = in_hi ? __uint_as_float(sr[4 * k + 2 + e]) * c : -INFINITY;
             sr[4 * k + e] = __float_as_uint(x_lo);
             sr[4 * k + 2 + e] = __float_as_uint(x_hi);
             mx_lo = fmaxf(mx_lo, x_lo);
@@ -1144,7 +1175,10 @@ cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items
     cudaError_t e = cudaFuncSetAttribute(attn_umma_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_umma_persist_kernel,
+    e = cudaFuncSetAttribute(attn_umma_persist_kernel<false>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemP);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_umma_persist_kernel<true>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemP);
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
@@ -1152,11 +1186,15 @@ cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items
     configured[dev] = true;
   }
   const int hkv = a.shape.num_kv_heads;
-  if (a.umma_mode != 1 && a.d_ticket != nullptr) {
+  if (a.q_limit != nullptr && a.d_ticket == nullptr) return cudaErrorInvalidValue;
+  if ((a.umma_mode != 1 || a.q_limit != nullptr) && a.d_ticket != nullptr) {
     // persistent form: two resident CTAs per SM claim (item, kv head) units from a counter
     const long long n_units = (long long)n_items * hkv;
     const int grid = (int)std::min<long long>(n_units, 2LL * sm_count[dev]);
-    return launch_kernel(attn_umma_persist_kernel, dim3(grid), dim3(192), kSmemP, st,
+    if (a.q_limit != nullptr)
+      return launch_kernel(attn_umma_persist_kernel<true>, dim3(grid), dim3(192), kSmemP, st,
+                           a.pdl != 0, *a.tm_k, *a.tm_v, a, item_begin, (int)n_units, a.d_ticket);
+    return launch_kernel(attn_umma_persist_kernel<false>, dim3(grid), dim3(192), kSmemP, st,
                          a.pdl != 0, *a.tm_k, *a.tm_v, a, item_begin, (int)n_units, a.d_ticket);
   }
   // Heads per CTA: up to kHeadsMax, if that leaves at least kWavesMin CTAs for each of the

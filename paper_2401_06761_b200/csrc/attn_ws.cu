@@ -349,12 +349,35 @@ attn_ws_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  if (*cta_abort) return;
+  const bool dead_on_arrival = *cta_abort != 0;
   if (threadIdx.x == 0) pdl_launch_dependents();
 
   const int g = lane >> 2, tq = lane & 3;
   const int jm = lane >> 3, jr = lane & 7;
   const float cs = a.scale_log2e;
+  // ticket[0] unit counter, ticket[1] warps that have left, ticket[2] launches completed.  The
+  // last warp to leave puts the first two back to zero and counts the launch, so that nobody
+  // has to clear anything between launches (and a replayed CUDA graph finds the same state).
+  // The launch count only changes when every warp has left: all warps read the same value,
+  // and "ready" for a partial result of this launch is that value plus one.
+  const int ready_mark = *(volatile int*)(ticket + 2) + 1;
+  auto leave = [&]() {
+    if (lane == 0) {
+      const int gone = atomicAdd(ticket + 1, 1);
+      if (gone == (int)gridDim.x * 4 - 1) {
+        ticket[0] = 0;
+        ticket[1] = 0;
+        __threadfence();
+        atomicAdd(ticket + 2, 1);
+      }
+    }
+  };
+
+  if (dead_on_arrival) {               // an earlier kernel gave up a wait: claim nothing
+    leave();
+    if (a.pdl) pdl_wait();
+    return;
+  }
 
   // ---- background fetch of unit descriptions: ticket -> work item -> (length) -> done
   WsUnit cur, nxt, nn;
@@ -481,6 +504,7 @@ attn_ws_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
   cur = nn;
   nn_final = false;
   if (!cur.valid) {
+    leave();
     if (a.pdl) pdl_wait();
     return;
   }
@@ -621,6 +645,7 @@ attn_ws_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
             do {
               asm volatile("ld.acquire.gpu.global.s32 %0, [%1];"
                            : "=r"(ready) : "l"(a.part_flag + prow) : "memory");
+              ready = ready == ready_mark;
             } while (!ready && ++spins < kSpin && !((spins & 255) == 255 && *cta_abort));
             if (!ready) {
               if (spins >= kSpin) atomicCAS(a.d_error, 0, 9500 + w);
@@ -669,7 +694,8 @@ attn_ws_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
             if (ur.slot >= 0) {
               __threadfence();
               *(volatile int*)(a.part_flag +
-                               (size_t)(ur.slot + cur.slot_add) * HQ + cur.h * G + r % G) = 1;
+                               (size_t)(ur.slot + cur.slot_add) * HQ + cur.h * G + r % G) =
+                  ready_mark;
             }
           }
         }
@@ -713,6 +739,7 @@ attn_ws_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
     const uint32_t fb = full_bar(c % kSlots), par = (c / kSlots) & 1;
     for (uint32_t i = 0; i < kSpin && !bar_try(fb, par); ++i) {}
   }
+  leave();
   if (a.pdl) pdl_wait();               // this grid completes after its predecessor
 }
 
@@ -735,13 +762,13 @@ cudaError_t launch_attention_ws(const AttnArgs& a, int item_begin, int n_items, 
   }
   const int hkv = a.shape.num_kv_heads;
   if (a.ws_mode != 1 && a.d_ticket != nullptr) {
-    // persistent form: every warp of two resident CTAs per SM claims (item, kv head) units;
-    // the counter was zeroed by the caller before the first attention kernel of the call
+    // persistent form: every warp of two resident CTAs per SM claims (item, kv head) units
+    // (the counters put themselves back to zero at the end of every launch)
     const long long n_units = (long long)n_items * hkv;
     const int grid = (int)std::min<long long>((n_units + 3) / 4, 2LL * a.num_sms);
     return launch_kernel(attn_ws_persist_kernel, dim3(grid), dim3(128), kSmemWP, st, a.pdl != 0,
                          *a.tm_k, *a.tm_v, a, item_begin, (int)n_units,
-                         a.d_ticket + ticket_index);
+                         a.d_ticket + 4 * ticket_index);
   }
   // Whole items per CTA when there are enough of them to fill the machine; otherwise the kv
   // heads are dealt out over several CTAs (in multiples of the four consumer warps).

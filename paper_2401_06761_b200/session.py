@@ -121,6 +121,17 @@ class PagedSession:
     def accept(self, tids, n_cand, keep):
         B.apar_accept_candidates(self.ctx, tids, n_cand, keep, self._stream())
 
+    def prefill_attention(self, tids, q_begin, q_count, q: torch.Tensor, out: torch.Tensor = None,
+                          layer: int = 0, sm_scale=None):
+        assert q.is_cuda and q.is_contiguous() and q.dtype == torch.bfloat16
+        if out is None:
+            out = torch.empty_like(q)
+        B.apar_tree_prefill_attention(self.ctx, layer, tids, q_begin, q_count, q.data_ptr(),
+                                      out.data_ptr(),
+                                      self.sm_scale if sm_scale is None else sm_scale,
+                                      self._stream())
+        return out
+
     def append_layer(self, layer: int, k_rows: torch.Tensor, v_rows: torch.Tensor):
         assert k_rows.is_cuda and k_rows.is_contiguous() and v_rows.is_contiguous()
         B.apar_append_kv_layer(self.ctx, layer, k_rows.data_ptr(), v_rows.data_ptr(),
