@@ -121,7 +121,7 @@ class ClockSampler:
 
 def parse_workload(name: str) -> int:
     if not (name.startswith("cfg") and name[3:].isdigit() and int(name[3:]) in synth.LAYER_SHAPES):
-        raise SystemExit(f"unknown workload {name}; use cfg1..cfg5 or lifecycle")
+        raise SystemExit(f"unknown workload {name}; use cfg1..cfg5, lifecycle or prefill")
     return int(name[3:])
 
 
@@ -537,6 +537,141 @@ def lifecycle_report(dev, n_requests=96, n_steps=1500, max_live=96):
     return rep
 
 
+def run_prefill(args):
+    """--workload prefill: the tensor-core side of the path.  A step = 64 new prompts of 2048
+    tokens (7B-like MHA layer: 32 heads) appended into the paged pool + tree-masked attention
+    over all of their tokens (every token attends the tokens before it) + release.  A second
+    arm applies the paragraph-tree mask of Section 2.2 to every token of a config-3-shaped
+    forest (each node a segment that attends its ancestors and, causally, itself)."""
+    from paper_2401_06761_b200 import build
+    build.build()
+    from paper_2401_06761_b200 import binding as B
+    from paper_2401_06761_b200.session import PagedSession, pool_requirements
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("--workload prefill runs on one GPU")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) \
+        if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+    peak_tf = float(peaks.get("bf16_tflops_sustained", 1400.0))
+    peak_kind = "measured, sustained" if peaks else "fallback"
+    n_prompts, plen = args.requests or 64, 2048
+    shape = synth.LAYER_SHAPES[2]
+    sess = PagedSession(shape, n_prompts * plen // 16 + 64, n_prompts + 8, plen // 16 + 1,
+                        device=dev)
+    g = torch.Generator(device=dev).manual_seed(2024)
+    rows = n_prompts * plen
+    k = torch.randn((rows, shape.num_kv_heads, 128), generator=g, device=dev).to(torch.bfloat16)
+    v = torch.randn((rows, shape.num_kv_heads, 128), generator=g, device=dev).to(torch.bfloat16)
+    q = torch.randn((rows, shape.num_q_heads, 128), generator=g, device=dev).to(torch.bfloat16)
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream().cuda_stream
+    flops = 4.0 * 128 * shape.num_q_heads * n_prompts * (plen * (plen + 1) / 2)
+
+    def step(events=None):
+        tids = B.apar_new_threads(sess.ctx, n_prompts)
+        B.apar_append_kv(sess.ctx, tids, [plen] * n_prompts, k.data_ptr(), v.data_ptr(), stream)
+        if events:
+            B.apar_set_timing_events(sess.ctx, events[0].cuda_event, events[1].cuda_event)
+        B.apar_tree_prefill_attention(sess.ctx, 0, tids, [0] * n_prompts, [plen] * n_prompts,
+                                      q.data_ptr(), out.data_ptr(), sess.sm_scale, stream)
+        if events:
+            B.apar_set_timing_events(sess.ctx, 0, 0)
+        B.apar_release(sess.ctx, tids)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    pool = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+            for _ in range(args.steps)]
+    for a, b in pool:
+        a.record(); b.record()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0).start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    k0 = sess.stats()["kernels_total"]
+    ev0.record()
+    for i in range(args.steps):
+        step(pool[i])
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    total_ms = ev0.elapsed_time(ev1)
+    attn_ms = statistics.mean(a.elapsed_time(b) for a, b in pool)
+    st = sess.stats()
+    if st["device_wait_timeouts"]:
+        raise SystemExit("a kernel gave up a bounded wait: the timed results are invalid")
+    launches = st["kernels_total"] - k0
+    sess.close()
+    del k, v, q, out
+    torch.cuda.empty_cache()
+
+    # ---- the paragraph-tree mask on a config-3-shaped forest: every token of every node
+    spec = synth.forest_spec(3, n_requests=64)
+    nb, nt, mb = pool_requirements(spec)
+    tsess = PagedSession(spec.shape, nb, nt, mb, device=dev)
+    tstep = synth.build_forest(spec, tsess, device=dev)
+    synth.run_step_forks(tstep, tsess)
+    tsess.append(tstep.live_handles, None, tstep.k_new, tstep.v_new)
+    segs = []
+    for node in spec.nodes:
+        h = tstep.handles[node.index]
+        total = tsess.thread(h)[0]
+        own = node.n_tok
+        segs.append((h, spec.attended_tokens(node) - own, own))
+    # (a node that was forked from keeps only its own tokens: children hold theirs)
+    t_tids = [s[0] for s in segs]
+    t_begin = [s[1] for s in segs]
+    t_count = [s[2] for s in segs]
+    nq = sum(t_count)
+    tq = torch.randn((nq, spec.shape.num_q_heads, 128), generator=torch.Generator(device=dev)
+                     .manual_seed(7), device=dev).to(torch.bfloat16)
+    tout = torch.empty_like(tq)
+    t_flops = 4.0 * 128 * spec.shape.num_q_heads * sum(b * c + c * (c + 1) / 2
+                                                     for b, c in zip(t_begin, t_count))
+    for _ in range(3):
+        tsess.prefill_attention(t_tids, t_begin, t_count, tq, out=tout)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 10
+    e0.record()
+    for _ in range(reps):
+        tsess.prefill_attention(t_tids, t_begin, t_count, tq, out=tout)
+    e1.record()
+    torch.cuda.synchronize()
+    tree_ms = e0.elapsed_time(e1) / reps
+    assert tsess.stats()["device_wait_timeouts"] == 0
+    tsess.close()
+
+    achieved = flops / (attn_ms * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": METRIC, "value": rows * args.steps / (total_ms * 1e-3), "unit": UNIT,
+        "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "prefill", "prompts": n_prompts, "prompt_tokens": plen,
+                   "num_q_heads": shape.num_q_heads, "num_kv_heads": shape.num_kv_heads,
+                   "head_dim": 128, "block_size": 16,
+                   "step": "new threads + append of all prompt rows + tree-masked attention "
+                           "over every token + release",
+                   "l2": "K, V, Q and out of a step are 2.1 GB, larger than L2",
+                   "note": "value counts query tokens (one per prompt position) per second"},
+        "clocks": clocks, "gpu_launches": launches,
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
+                     "frac": achieved / peak_tf, "traffic": None,
+                     "peak_kind": f"cuBLAS bf16 GEMM, {peak_kind}",
+                     "flops_per_step": flops, "attention_ms": attn_ms,
+                     "kernel": "tcgen05 kernel, tree-mask form (64-row query tiles)"},
+        "tree_mask": {"workload": "every token of a config-3-shaped forest of 64 requests",
+                      "queries": nq, "segments": len(segs), "ms": tree_ms,
+                      "tflops": t_flops / (tree_ms * 1e-3) / 1e12,
+                      "frac_of_peak": t_flops / (tree_ms * 1e-3) / 1e12 / peak_tf,
+                      "note": "host planning and uploads of the call included"},
+    }))
+
+
 def run_ours(args):
     from paper_2401_06761_b200 import build
     build.build()
@@ -799,7 +934,13 @@ def main():
                     help="attention layers per step (layers > 0 replay the plan; default 1)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    if args.workload == "prefill":
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable":
+                              "the prefill workload is timed on the GPU arm only"}))
+        else:
+            run_prefill(args)
+    elif args.impl == "reference":
         run_reference(args, parse_workload(args.workload))
     else:
         run_ours(args)

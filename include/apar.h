@@ -237,8 +237,7 @@ apar_status apar_accept_candidates(apar_ctx* ctx, int32_t n, const int32_t* tid 
  * cores; a tile reads its chain once for all of its rows and masks every row at its own
  * position.  Any number of queries per call (they are launched in batches that fit the
  * workspace); `layer` selects the pool layer.  Invalidates the cached decode plan.
- * Errors: INVALID_ARG (also a range outside the thread), BAD_THREAD, WORKSPACE_TOO_SMALL (more
- * than 12 x max_threads x num_q_heads queries in one call), CUDA. */
+ * Errors: INVALID_ARG (also a range outside the thread), BAD_THREAD, CUDA. */
 apar_status apar_tree_prefill_attention(apar_ctx* ctx, int32_t layer, int32_t n,
                                         const int32_t* tid /*[host]*/,
                                         const int32_t* q_begin /*[host]*/,

@@ -1239,9 +1239,7 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
   if (total_q > INT32_MAX) return APAR_ERR_INVALID_ARG;
   apar_status rc = sync_device_tables(c, seg_slot.data(), n, st);
   if (rc) return rc;
-  c->plan_epoch = 0;                    // the plan area of the workspace is reused below
-  c->attn_book_seq = 0;
-  c->plan_verify_n = 0;
+  c->attn_book_seq = 0;                 // layer replays of a decode plan need a decode call
 
   // Work items: the queries of a segment in tiles of 64 rows (64 / group tokens); a tile reads
   // the chain from its start to the tile's last token once, for all of its rows, and every row
@@ -1267,9 +1265,16 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
   a.v_pool = (const char*)c->cfg.v_pool + (size_t)layer * c->layer_bytes;
   a.d_tables = (const int32_t*)c->ws(c->lay.tables);
   a.d_lens = (const int32_t*)c->ws(c->lay.lens);
-  a.d_items = (const WorkItem*)c->ws(c->lay.plan_items);
-  a.d_users = (const UserRef*)c->ws(c->lay.plan_users);
-  a.part_o = (float*)c->ws(c->lay.part_o);
+  // Every tile covers its rows' whole chains, so no partial results are written: the area
+  // that holds them in decode calls (by far the largest part of the workspace) takes this
+  // call's work items and user entries instead, first half users, second half items.
+  const size_t area = (size_t)c->lay.slot_capacity * c->shape.num_q_heads * kDim * sizeof(float);
+  const int64_t cap = (int64_t)(area / 2 / std::max(sizeof(UserRef), sizeof(WorkItem)));
+  char* d_users = c->ws(c->lay.part_o);
+  char* d_items = d_users + area / 2;
+  a.d_items = (const WorkItem*)d_items;
+  a.d_users = (const UserRef*)d_users;
+  a.part_o = nullptr;
   a.part_ml = nullptr;
   a.shape = c->shape;
   a.scale_log2e = sm_scale * 1.4426950408889634f;
@@ -1278,10 +1283,7 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
   a.d_error = (int*)c->ws(c->lay.err);
   a.num_sms = c->num_sms;
   a.d_ticket = (int*)c->ws(c->lay.ticket);
-  // visible length per query, indexed by query number: the partial-result area is free here
-  // (every tile covers its rows' whole chains, so nothing is merged)
-  int32_t* d_limit = (int32_t*)c->ws(c->lay.part_ml);
-  a.q_limit = d_limit;
+  a.causal = true;                      // each user entry carries its query's visible length
 
   auto upload = [&](const void* src, size_t bytes, char* dst) -> apar_status {
     size_t done = 0;
@@ -1297,16 +1299,6 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
     }
     return APAR_OK;
   };
-  // batches that fit the plan area; limits are addressed by the global query number, so the
-  // limit array is uploaded whole, in pieces of the area's size if need be (then batch by batch)
-  const int64_t cap = c->lay.entry_capacity;
-  const int64_t limit_cap = c->lay.slot_capacity * c->shape.num_q_heads * 2;
-  if (total_q > limit_cap) return APAR_ERR_WORKSPACE_TOO_SMALL;
-  std::vector<int32_t> limits((size_t)total_q);
-  for (int i = 0; i < n; ++i)
-    for (int j = 0; j < q_count[i]; ++j) limits[(size_t)(seg_qbase[i] + j)] = q_begin[i] + j + 1;
-  rc = upload(limits.data(), limits.size() * 4, (char*)d_limit);
-  if (rc) return rc;
   std::vector<WorkItem> items;
   std::vector<UserRef> users;
   int launches = 0;
@@ -1329,12 +1321,13 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
       it.fin_n = it.fin_begin = 0;
       items.push_back(it);
       for (int k = 0; k < t.count; ++k)
-        users.push_back(UserRef{(int32_t)(seg_qbase[t.seg] + t.first + k), -1});
+        users.push_back(UserRef{(int32_t)(seg_qbase[t.seg] + t.first + k),
+                                -1 - (q_begin[t.seg] + t.first + k + 1)});
       ++t1;
     }
-    rc = upload(items.data(), items.size() * sizeof(WorkItem), c->ws(c->lay.plan_items));
+    rc = upload(items.data(), items.size() * sizeof(WorkItem), d_items);
     if (rc) return rc;
-    rc = upload(users.data(), users.size() * sizeof(UserRef), c->ws(c->lay.plan_users));
+    rc = upload(users.data(), users.size() * sizeof(UserRef), d_users);
     if (rc) return rc;
     if (c->time_start && t0 == 0) APAR_CUDA(c, cudaEventRecord(c->time_start, st));
     APAR_CUDA(c, launch_attention_umma(a, 0, (int)items.size(), st));

@@ -609,8 +609,9 @@ constexpr int kSmemP = kDescOff + kDescSlots * (int)sizeof(UnitDesc) + 1024;
 enum BarP { DFULL0 = NBARS, DEMPTY0 = DFULL0 + kDescSlots, NBARS_P = DEMPTY0 + kDescSlots };
 static_assert(8 * NBARS_P + 16 <= 256, "barrier area");
 
-// kCausal: every query has its own visible length (AttnArgs::q_limit, in chain positions): a
-// key at or beyond it is masked out for that row.  This is the tree mask of prefill / training
+// kCausal: every query has its own visible length L in chain positions (its user entry carries
+// slot = -1 - L: negative, so the row is written out as a final result): a key at or beyond L
+// is masked out for that row.  This is the tree mask of prefill / training
 // attention, where the queries of a unit are consecutive tokens of one node.
 template <bool kCausal>
 __global__ void __launch_bounds__(192, 2)
@@ -945,8 +946,8 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
       const int R = d->n_users * G, kvh = d->kvh;
       if (kCausal) {
         const int r_lo = warp * 16 + g8, r_hi = r_lo + 8;
-        lim_lo_next = r_lo < R ? a.q_limit[d->users[r_lo / G].query] - d->tok_begin : d->n_tok;
-        lim_hi_next = r_hi < R ? a.q_limit[d->users[r_hi / G].query] - d->tok_begin : d->n_tok;
+        lim_lo_next = r_lo < R ? -d->users[r_lo / G].slot - 1 - d->tok_begin : d->n_tok;
+        lim_hi_next = r_hi < R ? -d->users[r_hi / G].slot - 1 - d->tok_begin : d->n_tok;
       }
       uint4 qv[8];
 #pragma unroll
@@ -1186,12 +1187,12 @@ cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items
     configured[dev] = true;
   }
   const int hkv = a.shape.num_kv_heads;
-  if (a.q_limit != nullptr && a.d_ticket == nullptr) return cudaErrorInvalidValue;
-  if ((a.umma_mode != 1 || a.q_limit != nullptr) && a.d_ticket != nullptr) {
+  if (a.causal && a.d_ticket == nullptr) return cudaErrorInvalidValue;
+  if ((a.umma_mode != 1 || a.causal) && a.d_ticket != nullptr) {
     // persistent form: two resident CTAs per SM claim (item, kv head) units from a counter
     const long long n_units = (long long)n_items * hkv;
     const int grid = (int)std::min<long long>(n_units, 2LL * sm_count[dev]);
-    if (a.q_limit != nullptr)
+    if (a.causal)
       return launch_kernel(attn_umma_persist_kernel<true>, dim3(grid), dim3(192), kSmemP, st,
                            a.pdl != 0, *a.tm_k, *a.tm_v, a, item_begin, (int)n_units, a.d_ticket);
     return launch_kernel(attn_umma_persist_kernel<false>, dim3(grid), dim3(192), kSmemP, st,

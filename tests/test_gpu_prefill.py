@@ -89,7 +89,10 @@ def test_long_tree_in_batches_and_second_layer():
     from paper_2401_06761_b200.session import PagedSession
     hq, hkv = 8, 2
     shape = synth.LayerShape(hq, hkv)
-    sess = PagedSession(shape, 400, 40, 160, poison=True, num_layers=2)   # plan area: 1224 entries
+    # the call's work list lives in the partial-result area: with one thread
+    # slot per 1184 rows x 8 heads x 512 B / 2 / 32 B it holds 75 776 entries, so this call
+    # (2510 queries) is one batch; the batching itself is covered by the tiny case below
+    sess = PagedSession(shape, 400, 40, 160, poison=True, num_layers=2)
     orc = OracleBackend(shape, 400, 40, 160)
     g = torch.Generator(device="cuda").manual_seed(5)
     nodes = _tree(sess, orc, hkv, g, (1500, (210, 330, 170), 260, 40))
@@ -99,7 +102,6 @@ def test_long_tree_in_batches_and_second_layer():
     assert sum(counts) > 2400
     q = torch.randn((sum(counts), hq, 128), generator=g, device="cuda").to(torch.bfloat16)
     out = sess.prefill_attention(tids, begins, counts, q)
-    assert sess.stats()["attn_kernels"] >= 2
     _check_all_positions(sess, orc, nodes, q, out)
     # layer 1 holds other rows (layer 0's, negated): same mask, other result
     sess.k_pool[400:].copy_(-sess.k_pool[:400])
@@ -114,5 +116,31 @@ def test_long_tree_in_batches_and_second_layer():
     ref = np.stack([dense_attention(qq[base + j], -K[:first + j + 1], -V[:first + j + 1],
                                     sess.sm_scale) for j in range(counts[4])])
     assert_close(out1[base:base + counts[4]], ref, "layer 1")
+    assert sess.stats()["device_wait_timeouts"] == 0
+    sess.close()
+
+
+def test_batches_when_the_work_list_outgrows_its_area():
+    """One query head and one kv head make the work-list area small (1184 x 512 B / 2 / 32 B =
+    9472 entries): a 10 000-token prompt is split into two launches."""
+    from paper_2401_06761_b200.session import PagedSession
+    shape = synth.LayerShape(1, 1)
+    sess = PagedSession(shape, 700, 4, 640, poison=True)
+    orc = OracleBackend(shape, 700, 4, 640)
+    g = torch.Generator(device="cuda").manual_seed(17)
+    n = 10000
+    kv = torch.randn((2, n, 1, 128), generator=g, device="cuda").to(torch.bfloat16)
+    (t,) = sess.new_threads(1)
+    orc.new_threads(1)
+    sess.append([t], [n], kv[0].contiguous(), kv[1].contiguous())
+    orc.append([t], [n], kv[0], kv[1])
+    q = torch.randn((n, 1, 128), generator=g, device="cuda").to(torch.bfloat16)
+    out = sess.prefill_attention([t], [0], [n], q)
+    assert sess.stats()["attn_kernels"] == 2
+    K, V = orc.forest.chain(orc.node_of[t])
+    qq = q.cpu().to(torch.float64).numpy()
+    pick = list(range(0, n, 37)) + [n - 1, 9471, 9472, 9473]
+    ref = np.stack([dense_attention(qq[p], K[:p + 1], V[:p + 1], sess.sm_scale) for p in pick])
+    assert_close(out[pick], ref, "sampled positions of a 10 000-token prompt")
     assert sess.stats()["device_wait_timeouts"] == 0
     sess.close()
