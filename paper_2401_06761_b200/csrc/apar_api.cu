@@ -1243,15 +1243,28 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
 
   // Work items: the queries of a segment in tiles of 64 rows (64 / group tokens); a tile reads
   // the chain from its start to the tile's last token once, for all of its rows, and every row
-  // stops at its own position (the mask is applied by the kernel).  Longest tiles first.
+  // stops at its own position (the mask is applied by the kernel).
   const int G = c->shape.group, per_tile = std::max(1, kMaxRowsPerItem / G);
   struct Tile { int32_t seg, first, count; };
   std::vector<Tile> tiles;
   for (int i = 0; i < n; ++i)
     for (int j = 0; j < q_count[i]; j += per_tile)
       tiles.push_back(Tile{i, j, std::min(per_tile, q_count[i] - j)});
+  // Order: segments by how far they reach (longest first), the tiles of a segment together,
+  // longest first.  The kernel walks this list once per kv head, so the CTAs that run at the
+  // same time work on a few segments of one head and find their K and V in the L2 cache.
+  std::vector<int32_t> seg_rank(n);
+  {
+    std::vector<int32_t> order(n);
+    for (int i = 0; i < n; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) {
+      return q_begin[x] + q_count[x] > q_begin[y] + q_count[y];
+    });
+    for (int i = 0; i < n; ++i) seg_rank[order[i]] = i;
+  }
   std::stable_sort(tiles.begin(), tiles.end(), [&](const Tile& x, const Tile& y) {
-    return q_begin[x.seg] + x.first + x.count > q_begin[y.seg] + y.first + y.count;
+    if (x.seg != y.seg) return seg_rank[x.seg] < seg_rank[y.seg];
+    return x.first > y.first;
   });
   std::vector<int64_t> seg_qbase(n);
   {

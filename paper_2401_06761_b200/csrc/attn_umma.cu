@@ -702,7 +702,11 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
         if (f_tick >= n_units) {
           f_phase = 3;                              // publish the end mark
         } else {
-          const int4* ip = (const int4*)(a.d_items + item_begin + f_tick / HKV);
+          // Decode: a unit's kv heads follow each other (they walk the same block ids).  Tree
+          // mask: the query tiles of one head follow each other - the tiles of a segment read
+          // the same K and V, so the units that run at the same time share them in L2.
+          const int item = kCausal ? f_tick % (n_units / HKV) : f_tick / HKV;
+          const int4* ip = (const int4*)(a.d_items + item_begin + item);
           if (lane < 2) f_item = __ldg(ip + lane);
           f_phase = 2;
         }
@@ -739,7 +743,7 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
             d->tok_begin = f_tok_begin;
             d->n_tok = tok_end - f_tok_begin;
             d->n_tiles = (tok_end - f_tok_begin + kTileTok - 1) / kTileTok;
-            d->kvh = f_tick % HKV;
+            d->kvh = kCausal ? f_tick / (n_units / HKV) : f_tick % HKV;
             d->n_users = f_n_users;
             d->slot_add = f_slot_add;
           }
