@@ -941,6 +941,7 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
     const int row = warp * 16 + (lane & 15);
     const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
     const float c = a.scale_log2e;
+    const float cc = c > 0.f ? c : 1.f;               // what is left to apply inside the exponent
     const int g8 = lane >> 2, qd = lane & 3;
     // rows 16w .. 16w+15 of unit description d into the A-operand layout (rows past the unit's
     // own as zeros)
@@ -998,20 +999,33 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
         // keys of this tile a row may see: all that exist, or (tree mask) those before its limit
         const int see_lo = kCausal ? min(tile_tok, lim_lo - t * kTileTok) : tile_tok;
         const int see_hi = kCausal ? min(tile_tok, lim_hi - t * kTileTok) : tile_tok;
+        // The raw scores stay in registers; the scale is applied to the row maximum and, fused
+        // with the subtraction of the reference, inside the exponent.  A key a row may not see
+        // becomes -inf (rows of K past the valid length hold unspecified bits); tiles that are
+        // visible in full to every row of the warp skip that pass.  (A scale that is not
+        // positive is applied up front, so that the maximum of the raw values is the maximum.)
+        if (!(c > 0.f)) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) sr[j] = __float_as_uint(__uint_as_float(sr[j]) * c);
+        }
+        if (!__all_sync(0xffffffffu, see_lo >= kTileTok && see_hi >= kTileTok)) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              if (8 * k + 2 * qd + e >= see_lo) sr[4 * k + e] = 0xff800000u;
+              if (8 * k + 2 * qd + e >= see_hi) sr[4 * k + 2 + e] = 0xff800000u;
+            }
+          }
+        }
         float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const bool in_lo = 8 * k + 2 * qd + e < see_lo, in_hi = 8 * k + 2 * qd + e < see_hi;
-            const float x_lo = in_lo ? __uint_as_float(sr[4 * k + e]) * c : -INFINITY;
-            const float x_hi = in_hi ? __uint_as_float(sr[4 * k + 2 + e]) * c : -INFINITY;
-            sr[4 * k + e] = __float_as_uint(x_lo);
-            sr[4 * k + 2 + e] = __float_as_uint(x_hi);
-            mx_lo = fmaxf(mx_lo, x_lo);
-            mx_hi = fmaxf(mx_hi, x_hi);
-          }
+          mx_lo = fmaxf(mx_lo, fmaxf(__uint_as_float(sr[4 * k]), __uint_as_float(sr[4 * k + 1])));
+          mx_hi = fmaxf(mx_hi, fmaxf(__uint_as_float(sr[4 * k + 2]), __uint_as_float(sr[4 * k + 3])));
         }
+        mx_lo *= cc;
+        mx_hi *= cc;
         mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
         mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
         mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
@@ -1050,10 +1064,10 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
         uint32_t pk_lo[8], pk_hi[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          const float a0 = ex2(__uint_as_float(sr[4 * k]) - ref_lo);
-          const float a1 = ex2(__uint_as_float(sr[4 * k + 1]) - ref_lo);
-          const float b0 = ex2(__uint_as_float(sr[4 * k + 2]) - ref_hi);
-          const float b1 = ex2(__uint_as_float(sr[4 * k + 3]) - ref_hi);
+          const float a0 = ex2(fmaf(__uint_as_float(sr[4 * k]), cc, -ref_lo));
+          const float a1 = ex2(fmaf(__uint_as_float(sr[4 * k + 1]), cc, -ref_lo));
+          const float b0 = ex2(fmaf(__uint_as_float(sr[4 * k + 2]), cc, -ref_hi));
+          const float b1 = ex2(fmaf(__uint_as_float(sr[4 * k + 3]), cc, -ref_hi));
           l_lo += a0 + a1;
           l_hi += b0 + b1;
           pk_lo[k] = pack2(a0, a1);
