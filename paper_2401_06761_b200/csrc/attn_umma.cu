@@ -598,6 +598,8 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 // fixed number of arrivals whatever the unit's width.
 constexpr int kDescSlots = 3;
 constexpr int kClaimTiles = 8;      // the next unit is claimed this many K tiles before the end
+constexpr uint32_t kPollSpin = kSpin * 16;   // bound of the roles that poll without suspending
+                                             // (a pass of theirs is some tens of cycles)
 struct UnitDesc {
   int32_t table_row, tok_begin, n_tok, n_tiles;     // n_tiles == 0: no more units
   int32_t kvh, n_users, slot_add, pad;
@@ -728,7 +730,7 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
       } else {
         const int slot = f_units % kDescSlots;
         int ok = f_units < kDescSlots ||
-                 bar_try(bar(DEMPTY0 + slot), ((f_units / kDescSlots) - 1) & 1);
+                 bar_test(bar(DEMPTY0 + slot), ((f_units / kDescSlots) - 1) & 1);
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) return;
         UnitDesc* d = descs + slot;
@@ -786,7 +788,7 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
     auto issue = [&](Cursor& c, int g, int stages, int empty0, int full0, uint32_t ring,
                      const CUtensorMap* map) -> bool {
       const int s = g % stages;
-      int ready = g < stages || bar_try(bar(empty0 + s), ((g / stages) - 1) & 1);
+      int ready = g < stages || bar_test(bar(empty0 + s), ((g / stages) - 1) & 1);
       ready = __shfl_sync(0xffffffffu, ready, 0);
       if (!ready) return false;
       const int t = c.t;
@@ -815,7 +817,9 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
     uint32_t idle = 0;
     // the first unit: its fetch is driven to the end at once
     for (int i = 0; i < 4 && f_units == 0; ++i) fetch_step(true);
-    while (!vc.done) {
+    // (both cursors have to reach the end mark: V tiles can be released and issued ahead of the
+    // K tiles of the same unit when a K copy comes in late)
+    while (!(kc.done && vc.done)) {
       bool did = false;
       if (!kc.active && !kc.done && kc.unit < f_units) open_unit(kc);
       bool did_k = false;
@@ -837,9 +841,9 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
         idle = 0;
       } else {
         ++idle;
-        int stop = idle > kSpin || ((idle & 255) == 0 && *cta_abort);
+        int stop = idle > kPollSpin || ((idle & 255) == 0 && *cta_abort);
         if (__shfl_sync(0xffffffffu, stop, 0)) {
-          if (lane == 0 && idle > kSpin) {
+          if (lane == 0 && idle > kPollSpin) {
             *cta_abort = 1;
             atomicCAS(a.d_error, 0, 6000 + (kg % 25) * 40 + vg % 40);
           }
@@ -868,15 +872,15 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
       uint32_t idle = 0;
       while (true) {
         bool did = false;
-        if (!q_done && q_tiles < 0 && bar_try(bar(DFULL0 + qu % kDescSlots), (qu / kDescSlots) & 1)) {
+        if (!q_done && q_tiles < 0 && bar_test(bar(DFULL0 + qu % kDescSlots), (qu / kDescSlots) & 1)) {
           q_tiles = descs[qu % kDescSlots].n_tiles;
           if (q_tiles == 0) q_done = true;
         }
         if (!q_done && q_tiles > 0) {
           const int g = qk_g, s = g % kKStages, b = g & 1;
-          if (bar_try(bar(KFULL0 + s), (g / kKStages) & 1) &&
-              (g < 2 || bar_try(bar(SFREE0 + b), ((g >> 1) - 1) & 1)) &&
-              (qt > 0 || bar_try(bar(QFULL), qu & 1))) {
+          if (bar_test(bar(KFULL0 + s), (g / kKStages) & 1) &&
+              (g < 2 || bar_test(bar(SFREE0 + b), ((g >> 1) - 1) & 1)) &&
+              (qt > 0 || bar_test(bar(QFULL), qu & 1))) {
             tc_fence_after();
             const uint32_t kb = base + s * kKV, qb = base + kQOff;
 #pragma unroll
@@ -902,8 +906,8 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
             p_tok = descs[pu % kDescSlots].n_tok;
           }
           const int g = pv_g, s = g % kVStages;
-          if (bar_try(bar(PFULL), g & 1) && bar_try(bar(VFULL0 + s), (g / kVStages) & 1) &&
-              (pt > 0 || pu == 0 || bar_try(bar(ODONE), (pu - 1) & 1))) {
+          if (bar_test(bar(PFULL), g & 1) && bar_test(bar(VFULL0 + s), (g / kVStages) & 1) &&
+              (pt > 0 || pu == 0 || bar_test(bar(ODONE), (pu - 1) & 1))) {
             tc_fence_after();
             const uint32_t vb = base + kVOff + s * kKV, pb = base + kPOff;
             const int nk = min(kTileBlocks, (p_tok - pt * kTileTok + kBlock - 1) / kBlock);
@@ -928,8 +932,8 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
         if (q_done && pv_g == qk_g) break;
         if (did) {
           idle = 0;
-        } else if (++idle > kSpin || ((idle & 255) == 0 && *cta_abort)) {
-          if (idle > kSpin) atomicCAS(a.d_error, 0, 7000 + (qk_g % 25) * 40 + pv_g % 40);
+        } else if (++idle > kPollSpin || ((idle & 255) == 0 && *cta_abort)) {
+          if (idle > kPollSpin) atomicCAS(a.d_error, 0, 7000 + (qk_g % 25) * 40 + pv_g % 40);
           *cta_abort = 1;
           break;
         }

@@ -32,6 +32,17 @@ __device__ __forceinline__ bool bar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// The same test without any suspension: for a role that polls several barriers in turn, where
+// try_wait (which may park the thread for a while on a barrier that is not ready) would delay
+// the look at the next one.
+__device__ __forceinline__ bool bar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      " selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
 // Bounded wait.  On giving up it records where (code = wait site * 1000 + detail) in the error
 // word and raises the CTA's abort flag; it also returns early when another role gave up.
 __device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile int* cta_abort,
