@@ -30,7 +30,7 @@ def test_hand_computed_two_keys():
 
 def test_single_thread_equals_causal_decode_library_routine():
     # A tree with one thread is ordinary causal decoding: the new token is the last row of
-    # causal attention over the sequence.  The library routine is the judge here.
+    # causal attention over the sequence.  The library routine decides here.
     rng = np.random.default_rng(1)
     L, Hq, Hkv = 37, 4, 4
     k, v = _rand(rng, L, Hkv, D), _rand(rng, L, Hkv, D)
