@@ -8,8 +8,8 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libapar.so")
-SOURCES = ["apar_api.cu", "planner.cpp", "kernels.cu", "attn_umma.cu", "attn_ws.cu", "attn_static.cu", "tensor_maps.cu"]
-HEADERS = ["apar_internal.h", "ptx.cuh", os.path.join("..", "..", "include", "apar.h")]
+SOURCES = ["apar_api.cu", "planner.cpp", "kernels.cu", "attn_umma.cu", "attn_prefill.cu", "attn_ws.cu", "attn_static.cu", "tensor_maps.cu"]
+HEADERS = ["apar_internal.h", "ptx.cuh", "tcgen05.cuh", os.path.join("..", "..", "include", "apar.h")]
 
 
 def _stale() -> bool:

@@ -122,6 +122,8 @@ struct apar_ctx {
   int umma_heads = 0;                   // > 0: kv heads per CTA of the tcgen05 kernel (testing)
   int umma_mode = 0;                    // 1: one CTA per (item, heads); 2: persistent CTAs
   int ws_mode = 0;                      // 1: one CTA per item; 2: persistent warps
+  int prefill_rows = 128;               // query rows per tensor-core tile of tree-masked attention
+  int64_t prefill_batch = INT64_MAX;    // work items per launch of it, at most (testing)
   int num_sms = 148;
   int use_pdl = 1;                      // warp-stream launches may start before the kernel before
                                         // them has finished (0: ordinary launches only)
@@ -621,6 +623,10 @@ apar_status create_impl(const apar_config* cfg, bool external, bool host_only, a
   c->umma_mode = (mode && !strcmp(mode, "grid")) ? 1 : (mode && !strcmp(mode, "persist")) ? 2 : 0;
   mode = getenv("APAR_WS_MODE");                         // "grid" | "persist"
   c->ws_mode = (mode && !strcmp(mode, "grid")) ? 1 : (mode && !strcmp(mode, "persist")) ? 2 : 0;
+  mode = getenv("APAR_PREFILL");                         // "m64" | "m128": rows per MMA tile
+  c->prefill_rows = (mode && !strcmp(mode, "m64")) ? 64 : 128;
+  mode = getenv("APAR_PREFILL_BATCH");                   // work items per launch, at most
+  if (mode && atoll(mode) > 0) c->prefill_batch = atoll(mode);
   c->auto_path = !path || !strcmp(path, "auto") || !*path;
   const char* planner = getenv("APAR_PLANNER");          // testing: "tables" = per-block walk
   c->plan_by_runs = !(planner && !strcmp(planner, "tables"));
@@ -1241,10 +1247,13 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
   if (rc) return rc;
   c->attn_book_seq = 0;                 // layer replays of a decode plan need a decode call
 
-  // Work items: the queries of a segment in tiles of 64 rows (64 / group tokens); a tile reads
-  // the chain from its start to the tile's last token once, for all of its rows, and every row
-  // stops at its own position (the mask is applied by the kernel).
-  const int G = c->shape.group, per_tile = std::max(1, kMaxRowsPerItem / G);
+  // Work items: the queries of a segment in tiles of 256 rows (2 * (128 / group) tokens; 64
+  // rows with the older kernel); a tile reads the chain from its start to the tile's last token
+  // once, for all of its rows, and every row stops at its own position (the mask is applied by
+  // the kernel).
+  const int G = c->shape.group;
+  const bool wide = c->prefill_rows == 128;
+  const int per_tile = wide ? 2 * (128 / G) : std::max(1, kMaxRowsPerItem / G);
   struct Tile { int32_t seg, first, count; };
   std::vector<Tile> tiles;
   for (int i = 0; i < n; ++i)
@@ -1282,7 +1291,8 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
   // that holds them in decode calls (by far the largest part of the workspace) takes this
   // call's work items and user entries instead, first half users, second half items.
   const size_t area = (size_t)c->lay.slot_capacity * c->shape.num_q_heads * kDim * sizeof(float);
-  const int64_t cap = (int64_t)(area / 2 / std::max(sizeof(UserRef), sizeof(WorkItem)));
+  const int64_t cap = std::min<int64_t>(
+      c->prefill_batch, (int64_t)(area / 2 / std::max(sizeof(UserRef), sizeof(WorkItem))));
   char* d_users = c->ws(c->lay.part_o);
   char* d_items = d_users + area / 2;
   a.d_items = (const WorkItem*)d_items;
@@ -1314,9 +1324,30 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
   };
   std::vector<WorkItem> items;
   std::vector<UserRef> users;
+  std::vector<PrefillItem> wide_items;
   int launches = 0;
   c->last.attn_work_items = 0;
   size_t t0 = 0;
+  CUtensorMap tm_q;
+  if (wide && make_query_tensor_map(q, total_q, c->shape.num_q_heads, G, &tm_q) != 0)
+    return APAR_ERR_INVALID_ARG;        // (a query array that is not 16-byte aligned)
+  while (wide && t0 < tiles.size()) {   // 128-row tiles: an item is four numbers, no user list
+    const size_t t1 = (size_t)std::min<int64_t>((int64_t)tiles.size(), (int64_t)t0 + cap);
+    wide_items.clear();
+    for (size_t i = t0; i < t1; ++i) {
+      const Tile& t = tiles[i];
+      wide_items.push_back(PrefillItem{seg_slot[t.seg], (int32_t)(seg_qbase[t.seg] + t.first),
+                                       q_begin[t.seg] + t.first, t.count});
+    }
+    rc = upload(wide_items.data(), wide_items.size() * sizeof(PrefillItem), d_items);
+    if (rc) return rc;
+    if (c->time_start && t0 == 0) APAR_CUDA(c, cudaEventRecord(c->time_start, st));
+    APAR_CUDA(c, launch_attention_prefill(a, &tm_q, (const PrefillItem*)d_items,
+                                          (int)wide_items.size(), st));
+    ++launches;
+    c->last.attn_work_items += (int64_t)wide_items.size();
+    t0 = t1;
+  }
   while (t0 < tiles.size()) {
     items.clear();
     users.clear();

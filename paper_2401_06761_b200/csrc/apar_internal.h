@@ -178,6 +178,19 @@ cudaError_t launch_attention_vec(const AttnArgs& a, int item_begin, int n_items,
                                  cudaStream_t st);
 // Blackwell tcgen05/TMEM path for items with up to 64 rows (any number of query tiles).
 cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items, cudaStream_t st);
+// Tree-masked attention of consecutive query tokens with 128-row tiles (tcgen05): item i is
+// n_tok (at most 2 * (128 / group)) tokens of the thread in table row table_row, the first at
+// chain position pos0; its queries are rows q_first .. q_first + n_tok - 1 of the query
+// array, which the kernel reads through tm_q (make_query_tensor_map).  Uses a.out, a.d_tables,
+// a.shape, a.scale_log2e, a.tm_k, a.tm_v, a.d_error, a.num_sms and words 0-1 of a.d_ticket.
+struct PrefillItem { int32_t table_row, q_first, pos0, n_tok; };
+cudaError_t launch_attention_prefill(const AttnArgs& a, const CUtensorMap* tm_q,
+                                     const PrefillItem* d_items, int n_items, cudaStream_t st);
+// TMA descriptor of a query array [n_rows][num_q_heads][128] bf16 (16-byte aligned): a box is
+// the 64-dim half of the rows of `group` consecutive heads of 128 / group consecutive tokens.
+// Returns 0 on success.
+int make_query_tensor_map(const void* q, int64_t n_rows, int num_q_heads, int group,
+                          CUtensorMap* tm_q);
 // Warp-stream path for items with at most 16 rows per kv head; one CTA per item, all kv heads.
 // ticket_index: which group of four words of a.d_ticket the persistent form uses (1 or 2; group
 // 0 belongs to the tcgen05 kernel).

@@ -51,10 +51,14 @@ def _check_all_positions(sess, orc, nodes, q, out):
     return assert_close(out, ref, "tree-masked attention at every position")
 
 
-@pytest.mark.parametrize("hq,hkv", [(8, 2), (4, 4), (64, 8), (6, 1)])
-def test_every_token_of_a_paragraph_tree(hq, hkv):
+@pytest.mark.parametrize("rows", ["m128", "m64"])
+@pytest.mark.parametrize("hq,hkv", [(8, 2), (4, 4), (64, 8), (6, 1), (2, 2)])
+def test_every_token_of_a_paragraph_tree(hq, hkv, rows, monkeypatch):
+    """Both tensor-core forms: 128-row tiles (two warpgroups share the K/V tiles; the default)
+    and 64-row tiles."""
     from paper_2401_06761_b200 import binding as B
     from paper_2401_06761_b200.session import PagedSession
+    monkeypatch.setenv("APAR_PREFILL", rows)
     shape = synth.LayerShape(hq, hkv)
     sess = PagedSession(shape, 200, 16, 40, poison=True)
     orc = OracleBackend(shape, 200, 16, 40)
@@ -120,10 +124,15 @@ def test_long_tree_in_batches_and_second_layer():
     sess.close()
 
 
-def test_batches_when_the_work_list_outgrows_its_area():
-    """One query head and one kv head make the work-list area small (1184 x 512 B / 2 / 32 B =
-    9472 entries): a 10 000-token prompt is split into two launches."""
+@pytest.mark.parametrize("rows,batch,launches", [("m64", None, 2), ("m128", "16", 3)])
+def test_batches_when_the_work_list_outgrows_its_area(rows, batch, launches, monkeypatch):
+    """A 10 000-token prompt with one query head.  64-row tiles: the work-list area is small
+    (1184 x 512 B / 2 / 32 B = 9472 entries), so the call is split into two launches.  128-row
+    tiles: 40 work items of 256 tokens, here limited to 16 per launch."""
     from paper_2401_06761_b200.session import PagedSession
+    monkeypatch.setenv("APAR_PREFILL", rows)
+    if batch:
+        monkeypatch.setenv("APAR_PREFILL_BATCH", batch)
     shape = synth.LayerShape(1, 1)
     sess = PagedSession(shape, 700, 4, 640, poison=True)
     orc = OracleBackend(shape, 700, 4, 640)
@@ -136,10 +145,10 @@ def test_batches_when_the_work_list_outgrows_its_area():
     orc.append([t], [n], kv[0], kv[1])
     q = torch.randn((n, 1, 128), generator=g, device="cuda").to(torch.bfloat16)
     out = sess.prefill_attention([t], [0], [n], q)
-    assert sess.stats()["attn_kernels"] == 2
+    assert sess.stats()["attn_kernels"] == launches
     K, V = orc.forest.chain(orc.node_of[t])
     qq = q.cpu().to(torch.float64).numpy()
-    pick = list(range(0, n, 37)) + [n - 1, 9471, 9472, 9473]
+    pick = list(range(0, n, 37)) + [n - 1, 9471, 9472, 9473, 4095, 4096, 127, 128, 255, 256]
     ref = np.stack([dense_attention(qq[p], K[:p + 1], V[:p + 1], sess.sm_scale) for p in pick])
     assert_close(out[pick], ref, "sampled positions of a 10 000-token prompt")
     assert sess.stats()["device_wait_timeouts"] == 0
