@@ -35,13 +35,13 @@ constexpr int kTile = 64;                          // tokens per K/V stage and p
 constexpr int kTileBlk = kTile / kBlock;           // 4 blocks
 constexpr int kBlkBytes = kBlock * kDim * 2;       // one block of one kv head: 4 KiB
 constexpr int kRowsWg = 128;                       // query rows of a warpgroup
-constexpr int kKS = 3, kVS = 3;                    // ring depths
+constexpr int kKVS = 3;                            // ring depth
 constexpr int kStage = kTile * kDim * 2;           // K (or V) of a stage: 16 KiB
+constexpr int kPair = 2 * kStage;                  // a stage: K tile, then V tile
 constexpr int kStageHalf = kStage / 2;             // one 64-dim half: [64 rows][128 B]
 constexpr int kQBytes = kRowsWg * kDim * 2;        // 32 KiB: [2 halves][128 rows][128 B]
 constexpr int kQHalf = kQBytes / 2;
-constexpr int kOffV = kKS * kStage;
-constexpr int kOffQ = kOffV + kVS * kStage;        // Q: [2 buffers][2 warpgroups]
+constexpr int kOffQ = kKVS * kPair;                // Q: [2 buffers][2 warpgroups]
 constexpr int kOffBar = kOffQ + 4 * kQBytes;
 constexpr int kOffDesc = kOffBar + 512;
 constexpr int kDescRing = 3;
@@ -58,8 +58,8 @@ struct PrefillUnit {                               // a claimed unit, as the rol
 constexpr int kSmemPrefill = kOffDesc + kDescRing * (int)sizeof(PrefillUnit) + 1024;
 static_assert(kSmemPrefill <= 227 * 1024, "shared memory");
 
-enum { B_KFULL = 0, B_KEMPTY = B_KFULL + kKS, B_VFULL = B_KEMPTY + kKS, B_VEMPTY = B_VFULL + kVS,
-       B_DFULL = B_VEMPTY + kVS, B_DEMPTY = B_DFULL + kDescRing,
+enum { B_KVFULL = 0, B_KVEMPTY = B_KVFULL + kKVS,
+       B_DFULL = B_KVEMPTY + kKVS, B_DEMPTY = B_DFULL + kDescRing,
        B_QFULL = B_DEMPTY + kDescRing, B_QEMPTY = B_QFULL + 2,
        B_WG = B_QEMPTY + 2,                        // per warpgroup from here, B_WG_N each
        W_SFULL = 0, W_PFULL = 2, W_PFREE = 4, W_ODONE = 6, B_WG_N = 7,
@@ -96,8 +96,10 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_v) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_q) : "memory");
-    for (int s = 0; s < kKS; ++s) { bar_init(bar(B_KFULL + s), 1); bar_init(bar(B_KEMPTY + s), 1); }
-    for (int s = 0; s < kVS; ++s) { bar_init(bar(B_VFULL + s), 1); bar_init(bar(B_VEMPTY + s), 1); }
+    for (int s = 0; s < kKVS; ++s) {
+      bar_init(bar(B_KVFULL + s), 1);
+      bar_init(bar(B_KVEMPTY + s), 1);
+    }
     for (int d = 0; d < kDescRing; ++d) {
       bar_init(bar(B_DFULL + d), 1);
       bar_init(bar(B_DEMPTY + d), 9);              // eight softmax warps and the MMA thread
@@ -202,13 +204,13 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
       }
     };
 
-    // K and V tiles are two independent sequences over the units; each has its own cursor.
+    // The K and V tiles of all units form one sequence; tile g goes to ring stage g mod depth.
     struct Cursor {
       int unit = 0, t = 0, n_tiles = 0, n_blk = 0, kvh = 0;   // unit ordinal, tile in the unit
       bool active = false, done = false;
       const int32_t* table = nullptr;
       int id_cur = 0, id_next = 0;
-    } kc, vc;
+    } kc;
     auto open_unit = [&](Cursor& c) {
       const PrefillUnit* d = descs + c.unit % kDescRing;
       const int n_tiles = d->n_tiles;
@@ -225,11 +227,11 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
       c.t = 0;
       c.active = true;
     };
-    // Issues tile c.t of the cursor's unit into ring slot (g mod stages) if that slot is free.
-    auto issue = [&](Cursor& c, int g, int stages, int empty0, int full0, uint32_t ring,
-                     const CUtensorMap* map) -> bool {
-      const int s = g % stages;
-      int ready = g < stages || bar_test(bar(empty0 + s), ((g / stages) - 1) & 1);
+    // Issues tile c.t of the cursor's unit (K: lanes 0-7, V: lanes 8-15; a lane copies one
+    // 64-dim half of one block) into ring stage g mod depth if that stage is free.
+    auto issue = [&](Cursor& c, int g) -> bool {
+      const int s = g % kKVS;
+      int ready = g < kKVS || bar_test(bar(B_KVEMPTY + s), ((g / kKVS) - 1) & 1);
       ready = __shfl_sync(0xffffffffu, ready, 0);
       if (!ready) return false;
       const int t = c.t;
@@ -238,14 +240,17 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         const int nxt = (t + 8) * kTileBlk + lane;
         c.id_next = nxt < c.n_blk ? c.table[nxt] : 0;
       }
-      const int blk = t * kTileBlk + (lane >> 1);
+      const int li = lane & 7, blk = t * kTileBlk + (li >> 1);
       const int bid = __shfl_sync(0xffffffffu, c.id_cur, blk & 31);
       if (lane == 0)
-        bar_expect_tx(bar(full0 + s), (uint32_t)min(kTileBlk, c.n_blk - t * kTileBlk) * kBlkBytes);
+        bar_expect_tx(bar(B_KVFULL + s),
+                      2u * (uint32_t)min(kTileBlk, c.n_blk - t * kTileBlk) * kBlkBytes);
       __syncwarp();
-      if (lane < 2 * kTileBlk && blk < c.n_blk)
-        tma_2d(ring + s * kStage + (lane & 1) * kStageHalf + (lane >> 1) * (kBlock * 128), map,
-               (lane & 1) * 64, (bid * HKV + c.kvh) * kBlock, bar(full0 + s));
+      if (lane < 4 * kTileBlk && blk < c.n_blk)
+        tma_2d(base + s * kPair + (lane >> 3) * kStage + (li & 1) * kStageHalf +
+                   (li >> 1) * (kBlock * 128),
+               lane < 8 ? &tm_k : &tm_v, (li & 1) * 64, (bid * HKV + c.kvh) * kBlock,
+               bar(B_KVFULL + s));
       if (++c.t == c.n_tiles) {
         c.active = false;
         ++c.unit;
@@ -277,23 +282,16 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
       ++qu;
       return true;
     };
-    int kg = 0, vg = 0;               // tiles issued so far, all units
+    int kg = 0;                       // tiles issued so far, all units
     uint32_t idle = 0;
     for (int i = 0; i < 4 && f_units == 0; ++i) fetch_step(true);   // the first unit at once
-    // (both cursors have to reach the end mark: V tiles can be released and issued ahead of the
-    // K tiles of the same unit when a K copy comes in late)
-    while (!(kc.done && vc.done && q_done)) {
+    while (!(kc.done && q_done)) {
       bool did = false, did_k = false;
       if (!q_done && qu < f_units && issue_q()) did = true;
       if (!kc.active && !kc.done && kc.unit < f_units) open_unit(kc);
-      if (kc.active && issue(kc, kg, kKS, B_KEMPTY, B_KFULL, base, &tm_k)) {
+      if (kc.active && issue(kc, kg)) {
         ++kg;
         did = did_k = true;
-      }
-      if (!vc.active && !vc.done && vc.unit < f_units) open_unit(vc);
-      if (vc.active && issue(vc, vg, kVS, B_VEMPTY, B_VFULL, base + kOffV, &tm_v)) {
-        ++vg;
-        did = true;
       }
       // claim the next unit towards the end of the K stream of the current one (or at once
       // when the K cursor has nothing to do); one phase per tile issued or per idle pass
@@ -308,7 +306,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         if (__shfl_sync(0xffffffffu, stop, 0)) {
           if (lane == 0 && idle > kPollLimit) {
             *cta_abort = 1;
-            atomicCAS(a.d_error, 0, 16000 + (kg % 25) * 40 + vg % 40);
+            atomicCAS(a.d_error, 0, 16000 + kg % 1000);
           }
           break;
         }
@@ -332,6 +330,10 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
     // softmax warps are at work on the last ones.  MMAs of one thread execute in issue order:
     // Q K^T of tile j + 2 overwrites the S buffer that held P of tile j after P V of tile j
     // has read it.
+    // A look at a barrier takes more than a hundred cycles even when its phase is complete, so
+    // the barriers of a step are looked at (without waiting) ahead of the MMAs issued before
+    // that step; the results arrive while those are issued, and a blocking wait follows only
+    // for a barrier that was not ready then.
     constexpr uint32_t kIdescQK = instr_desc(kTile, false, kRowsWg);
     constexpr uint32_t kIdescPV = instr_desc(kDim, true, kRowsWg);
     constexpr unsigned kAll = 0xffffffffu;
@@ -341,21 +343,41 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
     int pv_j = -1, pv_t = 0, pv_tok = 0, pv_unit = 0;   // the P V that is due
     bool pv_side0 = false, pv_last = false;
     bool ok = true;
-    auto do_pv = [&]() -> bool {
-      const int vs = pv_j % kVS;
-      bool w8 = bar_wait(bar(B_VFULL + vs), (pv_j / kVS) & 1, cta_abort, a.d_error, 17200);
-      const uint32_t vb = base + kOffV + vs * kStage;
-      const int nk = min(kTileBlk, (pv_tok - pv_t * kTile + kBlock - 1) / kBlock);
+    bool kv_seen = false;                       // tile j's K and V were there at the last look
+    // what the due P V waits for, looked at now: bit w = P of warpgroup w is there (or not needed)
+    auto look_pv = [&]() -> uint32_t {
+      uint32_t seen = 0;
 #pragma unroll
       for (int w = 0; w < 2; ++w) {
-        if (w == 0 && !pv_side0) continue;
-        w8 = w8 && bar_wait(wbar(w, W_PFULL + (pg[w] & 1)), (pg[w] >> 1) & 1, cta_abort, a.d_error,
-                            17300 + w);
-        if (pv_t == 0 && pv_unit > 0)           // the unit before has read its O out
-          w8 = w8 && bar_wait(wbar(w, W_ODONE), (pv_unit - 1) & 1, cta_abort, a.d_error, 17400 + w);
+        bool r = true;
+        if (w == 1 || pv_side0) {
+          r = bar_test(wbar(w, W_PFULL + (pg[w] & 1)), (pg[w] >> 1) & 1);
+          if (pv_t == 0 && pv_unit > 0) r = r && bar_test(wbar(w, W_ODONE), (pv_unit - 1) & 1);
+        }
+        seen |= (r ? 1u : 0u) << w;
       }
-      if (!__all_sync(kAll, w8)) return false;
+      return seen;
+    };
+    auto do_pv = [&](uint32_t seen) -> bool {
+      const int vs = pv_j % kKVS;               // (its K and V arrived together)
+      const uint32_t vb = base + vs * kPair + kStage;
+      const int nk = min(kTileBlk, (pv_tok - pv_t * kTile + kBlock - 1) / kBlock);
+      if (!__all_sync(kAll, seen == 3u)) {
+        bool w8 = true;
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+          if (w == 0 && !pv_side0) continue;
+          w8 = w8 && bar_wait(wbar(w, W_PFULL + (pg[w] & 1)), (pg[w] >> 1) & 1, cta_abort,
+                              a.d_error, 17300 + w);
+          if (pv_t == 0 && pv_unit > 0)         // the unit before has read its O out
+            w8 = w8 && bar_wait(wbar(w, W_ODONE), (pv_unit - 1) & 1, cta_abort, a.d_error,
+                                17400 + w);
+        }
+        if (!__all_sync(kAll, w8)) return false;
+      }
       tc_fence_after();
+      // (a look at the next tile's K and V, for the next step)
+      kv_seen = bar_test(bar(B_KVFULL + (pv_j + 2) % kKVS), ((pv_j + 2) / kKVS) & 1);
       if (lead) {
         // the two warpgroups' products alternate: consecutive MMAs do not wait for each other's
         // accumulator
@@ -372,13 +394,11 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         }
         if (pv_side0) umma_commit(wbar(0, W_PFREE + (pg[0] & 1)));
         umma_commit(wbar(1, W_PFREE + (pg[1] & 1)));
+        umma_commit(bar(B_KVEMPTY + vs));       // both of the tile's products have been issued
+        if (pv_last) bar_arrive(bar(B_DEMPTY + pv_unit % kDescRing));
       }
       if (pv_side0) ++pg[0];
       ++pg[1];
-      if (lead) {
-        umma_commit(bar(B_VEMPTY + vs));
-        if (pv_last) bar_arrive(bar(B_DEMPTY + pv_unit % kDescRing));
-      }
       return true;
     };
     for (int u = 0; ok; ++u) {
@@ -392,16 +412,20 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
       const int tiles0 = __shfl_sync(kAll, d->tiles_wg0, 0);
       const int chain_tok = __shfl_sync(kAll, d->chain_tok, 0);
       for (int t = 0; t < n_tiles; ++t, ++j) {
-        const int s = j % kKS;
-        bool w8 = bar_wait(bar(B_KFULL + s), (j / kKS) & 1, cta_abort, a.d_error, 17100);
-        if (t == 0)
-          w8 = w8 && bar_wait(bar(B_QFULL + (u & 1)), (u >> 1) & 1, cta_abort, a.d_error, 17500);
-        if (!__all_sync(kAll, w8)) {
-          ok = false;
-          break;
+        const int s = j % kKVS;
+        if (!__all_sync(kAll, kv_seen) || t == 0) {
+          bool w8 = bar_wait(bar(B_KVFULL + s), (j / kKVS) & 1, cta_abort, a.d_error, 17100);
+          if (t == 0)
+            w8 = w8 && bar_wait(bar(B_QFULL + (u & 1)), (u >> 1) & 1, cta_abort, a.d_error, 17500);
+          if (!__all_sync(kAll, w8)) {
+            ok = false;
+            break;
+          }
         }
+        kv_seen = false;
         tc_fence_after();
-        const uint32_t kb = base + s * kStage;
+        const uint32_t seen = pv_j >= 0 ? look_pv() : 0u;
+        const uint32_t kb = base + s * kPair;
         const bool side0 = t < tiles0;            // (else: beyond the first warpgroup's last row)
         if (lead) {
 #pragma unroll
@@ -418,12 +442,11 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
           }
           if (side0) umma_commit(wbar(0, W_SFULL + (qg[0] & 1)));
           umma_commit(wbar(1, W_SFULL + (qg[1] & 1)));
-          umma_commit(bar(B_KEMPTY + s));
           if (t == n_tiles - 1) umma_commit(bar(B_QEMPTY + (u & 1)));   // the unit's rows are done with
         }
         if (side0) ++qg[0];
         ++qg[1];
-        if (pv_j >= 0 && !do_pv()) {
+        if (pv_j >= 0 && !do_pv(seen)) {
           ok = false;
           break;
         }
@@ -435,7 +458,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         pv_last = t == n_tiles - 1;
       }
     }
-    if (ok && pv_j >= 0) do_pv();
+    if (ok && pv_j >= 0) do_pv(0u);
     __syncwarp();
   } else {
     // ---------------------------------------------------------------- softmax warpgroups
@@ -537,12 +560,12 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         // the unit's last tile: each before its own P is handed over.
         const int tile_tok = chain_tok - t * kTile;
         if (tile_tok < kTile && wq == 0) {
-          const int vt = all0 + t, vs = vt % kVS;
-          if (!bar_wait(bar(B_VFULL + vs), (vt / kVS) & 1, cta_abort, a.d_error, 14000 + t % 1000)) {
+          const int vt = all0 + t, vs = vt % kKVS;
+          if (!bar_wait(bar(B_KVFULL + vs), (vt / kKVS) & 1, cta_abort, a.d_error, 14000 + t % 1000)) {
             alive = false;
             break;
           }
-          uint8_t* vptr = bp + kOffV + vs * kStage;
+          uint8_t* vptr = bp + vs * kPair + kStage;
           const int last = ((tile_tok + kBlock - 1) / kBlock) * kBlock;
           for (int x = lane; x < (last - tile_tok) * 16; x += 32)
             *(uint4*)(vptr + kv_off(tile_tok + (x >> 4), x & 15)) = make_uint4(0u, 0u, 0u, 0u);
