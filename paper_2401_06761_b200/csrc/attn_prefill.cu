@@ -70,7 +70,7 @@ __device__ __forceinline__ uint32_t kv_off(int row, int c) {  // a 64-token stag
   return (uint32_t)((c >> 3) * kStageHalf + row * 128 + (((c & 7) ^ (row & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(320)
+__global__ void __launch_bounds__(352)
 attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v,
                     const __grid_constant__ CUtensorMap tm_q, const AttnArgs a,
@@ -98,15 +98,15 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_q) : "memory");
     for (int s = 0; s < kKVS; ++s) {
       bar_init(bar(B_KVFULL + s), 1);
-      bar_init(bar(B_KVEMPTY + s), 1);
+      bar_init(bar(B_KVEMPTY + s), 2);             // both MMA issuers
     }
     for (int d = 0; d < kDescRing; ++d) {
       bar_init(bar(B_DFULL + d), 1);
-      bar_init(bar(B_DEMPTY + d), 9);              // eight softmax warps and the MMA thread
+      bar_init(bar(B_DEMPTY + d), 10);             // eight softmax warps and the two MMA issuers
     }
     for (int b = 0; b < 2; ++b) {
       bar_init(bar(B_QFULL + b), 1);
-      bar_init(bar(B_QEMPTY + b), 1);
+      bar_init(bar(B_QEMPTY + b), 2);
     }
     for (int w = 0; w < 2; ++w) {
       for (int b = 0; b < 2; ++b) {
@@ -321,84 +321,68 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         ticket[1] = 0;
       }
     }
-  } else if (warp == 9) {
-    // ---------------------------------------------------------------- MMA issuer
-    // The whole warp walks a fixed schedule with warp-uniform control flow (every value that
-    // forms an operand is derived from loop counters, so that the descriptors can live in
-    // uniform registers); lane 0 issues.  Per K/V tile j: S = Q K^T for each warpgroup, then
-    // O += P V of tile j - 1, so that the tensor pipe computes the next scores while the
-    // softmax warps are at work on the last ones.  MMAs of one thread execute in issue order:
-    // Q K^T of tile j + 2 overwrites the S buffer that held P of tile j after P V of tile j
-    // has read it.
-    // A look at a barrier takes more than a hundred cycles even when its phase is complete, so
-    // the barriers of a step are looked at (without waiting) ahead of the MMAs issued before
-    // that step; the results arrive while those are issued, and a blocking wait follows only
-    // for a barrier that was not ready then.
+  } else if (warp >= 9) {
+    // ---------------------------------------------------------------- MMA issuers
+    // One warp per warpgroup of query rows (warp 9: the first, warp 10: the second), each with
+    // warp-uniform control flow and lane 0 issuing.  A tcgen05.mma occupies its issuing thread
+    // until the tensor pipe takes it, and a look at a barrier takes that thread more than a
+    // hundred cycles: with two issuers, one's products keep the pipe busy while the other
+    // synchronises.  Per K/V tile j an issuer issues S = Q K^T of tile j, then O += P V of
+    // tile j - 1, so that the pipe computes the next scores while the softmax warps are at
+    // work on the last ones.  MMAs of one thread execute in issue order: Q K^T of tile j + 2
+    // overwrites the S buffer that held P of tile j after P V of tile j has read it.
     constexpr uint32_t kIdescQK = instr_desc(kTile, false, kRowsWg);
     constexpr uint32_t kIdescPV = instr_desc(kDim, true, kRowsWg);
     constexpr unsigned kAll = 0xffffffffu;
+    const int w = warp - 9;
     const bool lead = lane == 0;
+    const uint32_t tm_w = tmem + 256u * w;
     int j = 0;                                  // K/V tiles so far, all units
-    int qg[2] = {0, 0}, pg[2] = {0, 0};         // S tiles / P V products issued, per warpgroup
+    int qg = 0, pg = 0;                         // S tiles / P V products issued by this warp
     int pv_j = -1, pv_t = 0, pv_tok = 0, pv_unit = 0;   // the P V that is due
-    bool pv_side0 = false, pv_last = false;
+    bool pv_last = false;
     bool ok = true;
     bool kv_seen = false;                       // tile j's K and V were there at the last look
-    // what the due P V waits for, looked at now: bit w = P of warpgroup w is there (or not needed)
-    auto look_pv = [&]() -> uint32_t {
-      uint32_t seen = 0;
-#pragma unroll
-      for (int w = 0; w < 2; ++w) {
-        bool r = true;
-        if (w == 1 || pv_side0) {
-          r = bar_test(wbar(w, W_PFULL + (pg[w] & 1)), (pg[w] >> 1) & 1);
-          if (pv_t == 0 && pv_unit > 0) r = r && bar_test(wbar(w, W_ODONE), (pv_unit - 1) & 1);
-        }
-        seen |= (r ? 1u : 0u) << w;
-      }
-      return seen;
+    auto look_pv = [&]() -> bool {              // what the due P V waits for, looked at now
+      bool r = bar_test(wbar(w, W_PFULL + (pg & 1)), (pg >> 1) & 1);
+      if (pv_t == 0 && pv_unit > 0) r = r && bar_test(wbar(w, W_ODONE), (pv_unit - 1) & 1);
+      return r;
     };
-    auto do_pv = [&](uint32_t seen) -> bool {
+    auto do_pv = [&](bool seen) -> bool {
       const int vs = pv_j % kKVS;               // (its K and V arrived together)
       const uint32_t vb = base + vs * kPair + kStage;
       const int nk = min(kTileBlk, (pv_tok - pv_t * kTile + kBlock - 1) / kBlock);
-      if (!__all_sync(kAll, seen == 3u)) {
-        bool w8 = true;
-#pragma unroll
-        for (int w = 0; w < 2; ++w) {
-          if (w == 0 && !pv_side0) continue;
-          w8 = w8 && bar_wait(wbar(w, W_PFULL + (pg[w] & 1)), (pg[w] >> 1) & 1, cta_abort,
-                              a.d_error, 17300 + w);
-          if (pv_t == 0 && pv_unit > 0)         // the unit before has read its O out
-            w8 = w8 && bar_wait(wbar(w, W_ODONE), (pv_unit - 1) & 1, cta_abort, a.d_error,
-                                17400 + w);
-        }
+      if (!__all_sync(kAll, seen)) {
+        bool w8 = bar_wait(wbar(w, W_PFULL + (pg & 1)), (pg >> 1) & 1, cta_abort, a.d_error,
+                           17300 + w);
+        if (pv_t == 0 && pv_unit > 0)           // the unit before has read its O out
+          w8 = w8 && bar_wait(wbar(w, W_ODONE), (pv_unit - 1) & 1, cta_abort, a.d_error, 17400 + w);
         if (!__all_sync(kAll, w8)) return false;
       }
       tc_fence_after();
-      // (a look at the next tile's K and V, for the next step)
-      kv_seen = bar_test(bar(B_KVFULL + (pv_j + 2) % kKVS), ((pv_j + 2) / kKVS) & 1);
       if (lead) {
-        // the two warpgroups' products alternate: consecutive MMAs do not wait for each other's
-        // accumulator
+        // operands are formed once per tile; inside the unrolled loop only constants are added
+        const uint64_t vd = smem_desc(vb, kStageHalf, 1024);
+        const uint32_t p = tm_w + 64u * (pg & 1);
+        const uint32_t acc0 = pv_t != 0;
+        if (nk == kTileBlk) {
 #pragma unroll
-        for (int kk = 0; kk < kTileBlk; ++kk) {
-          if (kk >= nk) break;
-#pragma unroll
-          for (int w = 0; w < 2; ++w) {
-            if (w == 0 && !pv_side0) continue;
-            umma_bf16_ts(tmem + 256u * w + 128u, tmem + 256u * w + 64u * (pg[w] & 1) + 8u * kk,
-                         smem_desc(vb + kk * (kBlock * 128), kStageHalf, 1024), kIdescPV,
-                         (pv_t | kk) != 0);
-          }
+          for (int kk = 0; kk < kTileBlk; ++kk)
+            umma_bf16_ts(tm_w + 128u, p + 8u * kk, vd + (uint64_t)(kk * (kBlock * 128) >> 4),
+                         kIdescPV, kk ? 1u : acc0);
+        } else {
+          for (int kk = 0; kk < nk; ++kk)
+            umma_bf16_ts(tm_w + 128u, p + 8u * kk, vd + (uint64_t)(kk * (kBlock * 128) >> 4),
+                         kIdescPV, kk ? 1u : acc0);
         }
-        if (pv_side0) umma_commit(wbar(0, W_PFREE + (pg[0] & 1)));
-        umma_commit(wbar(1, W_PFREE + (pg[1] & 1)));
-        umma_commit(bar(B_KVEMPTY + vs));       // both of the tile's products have been issued
+        umma_commit(wbar(w, W_PFREE + (pg & 1)));
+        umma_commit(bar(B_KVEMPTY + vs));       // this warpgroup is done with the tile
         if (pv_last) bar_arrive(bar(B_DEMPTY + pv_unit % kDescRing));
       }
-      if (pv_side0) ++pg[0];
-      ++pg[1];
+      ++pg;
+      // (a look at the next tile's K and V, for the next step: the products just issued run
+      // while the answer comes)
+      kv_seen = bar_test(bar(B_KVFULL + (pv_j + 2) % kKVS), ((pv_j + 2) / kKVS) & 1);
       return true;
     };
     for (int u = 0; ok; ++u) {
@@ -409,10 +393,29 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
       const PrefillUnit* d = descs + ds;
       const int n_tiles = __shfl_sync(kAll, d->n_tiles, 0);
       if (n_tiles == 0) break;
-      const int tiles0 = __shfl_sync(kAll, d->tiles_wg0, 0);
+      const int my_tiles = w == 0 ? __shfl_sync(kAll, d->tiles_wg0, 0) : n_tiles;
       const int chain_tok = __shfl_sync(kAll, d->chain_tok, 0);
+      const uint64_t qd = smem_desc(base + kOffQ + ((u & 1) * 2 + w) * kQBytes, 16, 1024);
       for (int t = 0; t < n_tiles; ++t, ++j) {
         const int s = j % kKVS;
+        if (t >= my_tiles) {
+          // beyond this warpgroup's last row: the P V that is still due, and the tile is let go
+          if (pv_j >= 0 && !do_pv(false)) {
+            ok = false;
+            break;
+          }
+          pv_j = -1;
+          kv_seen = false;
+          // (the tile's copies have been requested, so the stage's release before this one
+          // is complete: this arrival cannot be counted for it)
+          if (!__all_sync(kAll, bar_wait(bar(B_KVFULL + s), (j / kKVS) & 1, cta_abort, a.d_error,
+                                         17600))) {
+            ok = false;
+            break;
+          }
+          if (lead) bar_arrive(bar(B_KVEMPTY + s));
+          continue;
+        }
         if (!__all_sync(kAll, kv_seen) || t == 0) {
           bool w8 = bar_wait(bar(B_KVFULL + s), (j / kKVS) & 1, cta_abort, a.d_error, 17100);
           if (t == 0)
@@ -424,41 +427,33 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         }
         kv_seen = false;
         tc_fence_after();
-        const uint32_t seen = pv_j >= 0 ? look_pv() : 0u;
-        const uint32_t kb = base + s * kPair;
-        const bool side0 = t < tiles0;            // (else: beyond the first warpgroup's last row)
         if (lead) {
+          const uint64_t kd = smem_desc(base + s * kPair, 16, 1024);
+          const uint32_t sd = tm_w + 64u * (qg & 1);
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-#pragma unroll
-            for (int w = 0; w < 2; ++w) {
-              if (w == 0 && !side0) continue;
-              umma_bf16(tmem + 256u * w + 64u * (qg[w] & 1),
-                        smem_desc(base + kOffQ + ((u & 1) * 2 + w) * kQBytes + (ks >> 2) * kQHalf +
-                                      (ks & 3) * 32, 16, 1024),
-                        smem_desc(kb + (ks >> 2) * kStageHalf + (ks & 3) * 32, 16, 1024),
-                        kIdescQK, ks > 0);
-            }
-          }
-          if (side0) umma_commit(wbar(0, W_SFULL + (qg[0] & 1)));
-          umma_commit(wbar(1, W_SFULL + (qg[1] & 1)));
-          if (t == n_tiles - 1) umma_commit(bar(B_QEMPTY + (u & 1)));   // the unit's rows are done with
+          for (int ks = 0; ks < 8; ++ks)
+            umma_bf16(sd, qd + (uint64_t)(((ks >> 2) * kQHalf + (ks & 3) * 32) >> 4),
+                      kd + (uint64_t)(((ks >> 2) * kStageHalf + (ks & 3) * 32) >> 4), kIdescQK,
+                      ks > 0);
+          umma_commit(wbar(w, W_SFULL + (qg & 1)));
+          if (t == my_tiles - 1) umma_commit(bar(B_QEMPTY + (u & 1)));   // done with the unit's rows
         }
-        if (side0) ++qg[0];
-        ++qg[1];
-        if (pv_j >= 0 && !do_pv(seen)) {
-          ok = false;
-          break;
+        ++qg;
+        if (pv_j >= 0) {
+          const bool seen = look_pv();          // (answers while the products above run)
+          if (!do_pv(seen)) {
+            ok = false;
+            break;
+          }
         }
         pv_j = j;
         pv_t = t;
         pv_tok = chain_tok;
         pv_unit = u;
-        pv_side0 = t < tiles0;
-        pv_last = t == n_tiles - 1;
+        pv_last = t == my_tiles - 1;
       }
     }
-    if (ok && pv_j >= 0) do_pv(0u);
+    if (ok && pv_j >= 0) do_pv(false);
     __syncwarp();
   } else {
     // ---------------------------------------------------------------- softmax warpgroups
@@ -639,7 +634,7 @@ cudaError_t launch_attention_prefill(const AttnArgs& a, const CUtensorMap* tm_q,
   }
   const long long n_units = (long long)n_items * a.shape.num_kv_heads;
   const int grid = (int)std::min<long long>(n_units, a.num_sms);
-  return launch_kernel(attn_prefill_kernel, dim3(grid), dim3(320), kSmemPrefill, st, false, *a.tm_k,
+  return launch_kernel(attn_prefill_kernel, dim3(grid), dim3(352), kSmemPrefill, st, false, *a.tm_k,
                        *a.tm_v, *tm_q, a, d_items, n_items, a.d_ticket);
 }
 
