@@ -343,10 +343,14 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
     bool pv_last = false;
     bool ok = true;
     bool kv_seen = false;                       // tile j's K and V were there at the last look
-    auto look_pv = [&]() -> bool {              // what the due P V waits for, looked at now
-      bool r = bar_test(wbar(w, W_PFULL + (pg & 1)), (pg >> 1) & 1);
-      if (pv_t == 0 && pv_unit > 0) r = r && bar_test(wbar(w, W_ODONE), (pv_unit - 1) & 1);
-      return r;
+    // What the due P V waits for, and the next tile's K and V, looked at now (the looks go out
+    // together, so that their answers come together).
+    auto look_pv = [&]() -> bool {
+      const bool p = bar_test(wbar(w, W_PFULL + (pg & 1)), (pg >> 1) & 1);
+      const bool k = bar_test(bar(B_KVFULL + (pv_j + 2) % kKVS), ((pv_j + 2) / kKVS) & 1);
+      const bool o = !(pv_t == 0 && pv_unit > 0) || bar_test(wbar(w, W_ODONE), (pv_unit - 1) & 1);
+      kv_seen = k;
+      return p && o;
     };
     auto do_pv = [&](bool seen) -> bool {
       const int vs = pv_j % kKVS;               // (its K and V arrived together)
@@ -380,9 +384,6 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         if (pv_last) bar_arrive(bar(B_DEMPTY + pv_unit % kDescRing));
       }
       ++pg;
-      // (a look at the next tile's K and V, for the next step: the products just issued run
-      // while the answer comes)
-      kv_seen = bar_test(bar(B_KVFULL + (pv_j + 2) % kKVS), ((pv_j + 2) / kKVS) & 1);
       return true;
     };
     for (int u = 0; ok; ++u) {
@@ -400,12 +401,12 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         const int s = j % kKVS;
         if (t >= my_tiles) {
           // beyond this warpgroup's last row: the P V that is still due, and the tile is let go
+          kv_seen = false;
           if (pv_j >= 0 && !do_pv(false)) {
             ok = false;
             break;
           }
           pv_j = -1;
-          kv_seen = false;
           // (the tile's copies have been requested, so the stage's release before this one
           // is complete: this arrival cannot be counted for it)
           if (!__all_sync(kAll, bar_wait(bar(B_KVFULL + s), (j / kKVS) & 1, cta_abort, a.d_error,
@@ -425,7 +426,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
             break;
           }
         }
-        kv_seen = false;
+        kv_seen = false;                          // (set again by the look below)
         tc_fence_after();
         if (lead) {
           const uint64_t kd = smem_desc(base + s * kPair, 16, 1024);
