@@ -35,13 +35,13 @@ constexpr int kTile = 64;                          // tokens per K/V stage and p
 constexpr int kTileBlk = kTile / kBlock;           // 4 blocks
 constexpr int kBlkBytes = kBlock * kDim * 2;       // one block of one kv head: 4 KiB
 constexpr int kRowsWg = 128;                       // query rows of a warpgroup
-constexpr int kKVS = 3;                            // ring depth
+constexpr int kKS = 3, kVS = 3;                    // ring depths
 constexpr int kStage = kTile * kDim * 2;           // K (or V) of a stage: 16 KiB
-constexpr int kPair = 2 * kStage;                  // a stage: K tile, then V tile
 constexpr int kStageHalf = kStage / 2;             // one 64-dim half: [64 rows][128 B]
 constexpr int kQBytes = kRowsWg * kDim * 2;        // 32 KiB: [2 halves][128 rows][128 B]
 constexpr int kQHalf = kQBytes / 2;
-constexpr int kOffQ = kKVS * kPair;                // Q: [2 buffers][2 warpgroups]
+constexpr int kOffV = kKS * kStage;
+constexpr int kOffQ = kOffV + kVS * kStage;        // Q: [2 buffers][2 warpgroups]
 constexpr int kOffBar = kOffQ + 4 * kQBytes;
 constexpr int kOffDesc = kOffBar + 512;
 constexpr int kDescRing = 3;
@@ -58,8 +58,8 @@ struct PrefillUnit {                               // a claimed unit, as the rol
 constexpr int kSmemPrefill = kOffDesc + kDescRing * (int)sizeof(PrefillUnit) + 1024;
 static_assert(kSmemPrefill <= 227 * 1024, "shared memory");
 
-enum { B_KVFULL = 0, B_KVEMPTY = B_KVFULL + kKVS,
-       B_DFULL = B_KVEMPTY + kKVS, B_DEMPTY = B_DFULL + kDescRing,
+enum { B_KFULL = 0, B_KEMPTY = B_KFULL + kKS, B_VFULL = B_KEMPTY + kKS, B_VEMPTY = B_VFULL + kVS,
+       B_DFULL = B_VEMPTY + kVS, B_DEMPTY = B_DFULL + kDescRing,
        B_QFULL = B_DEMPTY + kDescRing, B_QEMPTY = B_QFULL + 2,
        B_WG = B_QEMPTY + 2,                        // per warpgroup from here, B_WG_N each
        W_SFULL = 0, W_PFULL = 2, W_PFREE = 4, W_ODONE = 6, B_WG_N = 7,
@@ -70,7 +70,7 @@ __device__ __forceinline__ uint32_t kv_off(int row, int c) {  // a 64-token stag
   return (uint32_t)((c >> 3) * kStageHalf + row * 128 + (((c & 7) ^ (row & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(352)
+__global__ void __launch_bounds__(384)
 attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v,
                     const __grid_constant__ CUtensorMap tm_q, const AttnArgs a,
@@ -96,13 +96,17 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_v) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tm_q) : "memory");
-    for (int s = 0; s < kKVS; ++s) {
-      bar_init(bar(B_KVFULL + s), 1);
-      bar_init(bar(B_KVEMPTY + s), 2);             // both MMA issuers
+    for (int s = 0; s < kKS; ++s) {
+      bar_init(bar(B_KFULL + s), 1);
+      bar_init(bar(B_KEMPTY + s), 2);              // both MMA issuers
+    }
+    for (int s = 0; s < kVS; ++s) {
+      bar_init(bar(B_VFULL + s), 1);
+      bar_init(bar(B_VEMPTY + s), 2);
     }
     for (int d = 0; d < kDescRing; ++d) {
       bar_init(bar(B_DFULL + d), 1);
-      bar_init(bar(B_DEMPTY + d), 10);             // eight softmax warps and the two MMA issuers
+      bar_init(bar(B_DEMPTY + d), 11);             // softmax warps, MMA issuers, V producer
     }
     for (int b = 0; b < 2; ++b) {
       bar_init(bar(B_QFULL + b), 1);
@@ -204,7 +208,11 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
       }
     };
 
-    // The K and V tiles of all units form one sequence; tile g goes to ring stage g mod depth.
+    // K and V tiles are two independent sequences over the units (a K tile is free again as
+    // soon as its Q K^T products are done, a V tile one softmax later), each with its own ring
+    // and its own warp: a warp's tensor copy instruction takes some seventy cycles per box, a
+    // tile is eight boxes of 2 KiB for K and eight for V, and one warp issuing both could not
+    // keep up with the tensor pipe.  This warp copies K; warp 11 copies V.
     struct Cursor {
       int unit = 0, t = 0, n_tiles = 0, n_blk = 0, kvh = 0;   // unit ordinal, tile in the unit
       bool active = false, done = false;
@@ -227,11 +235,11 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
       c.t = 0;
       c.active = true;
     };
-    // Issues tile c.t of the cursor's unit (K: lanes 0-7, V: lanes 8-15; a lane copies one
-    // 64-dim half of one block) into ring stage g mod depth if that stage is free.
-    auto issue = [&](Cursor& c, int g) -> bool {
-      const int s = g % kKVS;
-      int ready = g < kKVS || bar_test(bar(B_KVEMPTY + s), ((g / kKVS) - 1) & 1);
+    // Issues tile c.t of the cursor's unit into ring slot (g mod stages) if that slot is free.
+    auto issue = [&](Cursor& c, int g, int stages, int empty0, int full0, uint32_t ring,
+                     const CUtensorMap* map) -> bool {
+      const int s = g % stages;
+      int ready = g < stages || bar_test(bar(empty0 + s), ((g / stages) - 1) & 1);
       ready = __shfl_sync(0xffffffffu, ready, 0);
       if (!ready) return false;
       const int t = c.t;
@@ -240,17 +248,14 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         const int nxt = (t + 8) * kTileBlk + lane;
         c.id_next = nxt < c.n_blk ? c.table[nxt] : 0;
       }
-      const int li = lane & 7, blk = t * kTileBlk + (li >> 1);
+      const int blk = t * kTileBlk + (lane >> 1);
       const int bid = __shfl_sync(0xffffffffu, c.id_cur, blk & 31);
       if (lane == 0)
-        bar_expect_tx(bar(B_KVFULL + s),
-                      2u * (uint32_t)min(kTileBlk, c.n_blk - t * kTileBlk) * kBlkBytes);
+        bar_expect_tx(bar(full0 + s), (uint32_t)min(kTileBlk, c.n_blk - t * kTileBlk) * kBlkBytes);
       __syncwarp();
-      if (lane < 4 * kTileBlk && blk < c.n_blk)
-        tma_2d(base + s * kPair + (lane >> 3) * kStage + (li & 1) * kStageHalf +
-                   (li >> 1) * (kBlock * 128),
-               lane < 8 ? &tm_k : &tm_v, (li & 1) * 64, (bid * HKV + c.kvh) * kBlock,
-               bar(B_KVFULL + s));
+      if (lane < 2 * kTileBlk && blk < c.n_blk)
+        tma_2d(ring + s * kStage + (lane & 1) * kStageHalf + (lane >> 1) * (kBlock * 128), map,
+               (lane & 1) * 64, (bid * HKV + c.kvh) * kBlock, bar(full0 + s));
       if (++c.t == c.n_tiles) {
         c.active = false;
         ++c.unit;
@@ -282,14 +287,14 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
       ++qu;
       return true;
     };
-    int kg = 0;                       // tiles issued so far, all units
+    int kg = 0;                       // K tiles issued so far, all units
     uint32_t idle = 0;
     for (int i = 0; i < 4 && f_units == 0; ++i) fetch_step(true);   // the first unit at once
     while (!(kc.done && q_done)) {
       bool did = false, did_k = false;
       if (!q_done && qu < f_units && issue_q()) did = true;
       if (!kc.active && !kc.done && kc.unit < f_units) open_unit(kc);
-      if (kc.active && issue(kc, kg)) {
+      if (kc.active && issue(kc, kg, kKS, B_KEMPTY, B_KFULL, base, &tm_k)) {
         ++kg;
         did = did_k = true;
       }
@@ -321,6 +326,47 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         ticket[1] = 0;
       }
     }
+  } else if (warp == 11) {
+    // ---------------------------------------------------------------- V producer
+    int vg = 0;                       // V tiles issued so far, all units
+    bool ok = true;
+    for (int u = 0; ok; ++u) {
+      const int ds = u % kDescRing;
+      ok = __all_sync(0xffffffffu, bar_wait(bar(B_DFULL + ds), (u / kDescRing) & 1, cta_abort,
+                                            a.d_error, 18000));
+      if (!ok) break;
+      const PrefillUnit* d = descs + ds;
+      const int n_tiles = __shfl_sync(0xffffffffu, d->n_tiles, 0);
+      if (n_tiles == 0) break;
+      const int n_blk = (__shfl_sync(0xffffffffu, d->chain_tok, 0) + kBlock - 1) / kBlock;
+      const int kvh = __shfl_sync(0xffffffffu, d->kvh, 0);
+      const int32_t* table =
+          a.d_tables + (size_t)__shfl_sync(0xffffffffu, d->table_row, 0) * a.shape.table_stride;
+      int id_cur = d->ids[lane], id_next = d->ids[lane + 32];
+      __syncwarp();
+      if (lane == 0) bar_arrive(bar(B_DEMPTY + ds));   // what it needs of the description is copied
+      for (int t = 0; t < n_tiles; ++t, ++vg) {
+        const int s = vg % kVS;
+        if (vg >= kVS) {
+          ok = __all_sync(0xffffffffu, bar_wait(bar(B_VEMPTY + s), ((vg / kVS) - 1) & 1, cta_abort,
+                                                a.d_error, 18100));
+          if (!ok) break;
+        }
+        if (t > 0 && (t & 7) == 0) {                // 32 block ids last for 8 tiles
+          id_cur = id_next;
+          const int nxt = (t + 8) * kTileBlk + lane;
+          id_next = nxt < n_blk ? table[nxt] : 0;
+        }
+        const int blk = t * kTileBlk + (lane >> 1);
+        const int bid = __shfl_sync(0xffffffffu, id_cur, blk & 31);
+        if (lane == 0)
+          bar_expect_tx(bar(B_VFULL + s), (uint32_t)min(kTileBlk, n_blk - t * kTileBlk) * kBlkBytes);
+        __syncwarp();
+        if (lane < 2 * kTileBlk && blk < n_blk)
+          tma_2d(base + kOffV + s * kStage + (lane & 1) * kStageHalf + (lane >> 1) * (kBlock * 128),
+                 &tm_v, (lane & 1) * 64, (bid * HKV + kvh) * kBlock, bar(B_VFULL + s));
+      }
+    }
   } else if (warp >= 9) {
     // ---------------------------------------------------------------- MMA issuers
     // One warp per warpgroup of query rows (warp 9: the first, warp 10: the second), each with
@@ -342,23 +388,21 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
     int pv_j = -1, pv_t = 0, pv_tok = 0, pv_unit = 0;   // the P V that is due
     bool pv_last = false;
     bool ok = true;
-    bool kv_seen = false;                       // tile j's K and V were there at the last look
-    // What the due P V waits for, and the next tile's K and V, looked at now (the looks go out
-    // together, so that their answers come together).
-    auto look_pv = [&]() -> bool {
-      const bool p = bar_test(wbar(w, W_PFULL + (pg & 1)), (pg >> 1) & 1);
-      const bool k = bar_test(bar(B_KVFULL + (pv_j + 2) % kKVS), ((pv_j + 2) / kKVS) & 1);
-      const bool o = !(pv_t == 0 && pv_unit > 0) || bar_test(wbar(w, W_ODONE), (pv_unit - 1) & 1);
-      kv_seen = k;
-      return p && o;
+    bool k_seen = false;                        // tile j's K was there at the last look
+    auto look_pv = [&]() -> bool {              // what the due P V waits for, looked at now
+      bool r = bar_test(wbar(w, W_PFULL + (pg & 1)), (pg >> 1) & 1);
+      r = r && bar_test(bar(B_VFULL + pv_j % kVS), (pv_j / kVS) & 1);
+      if (pv_t == 0 && pv_unit > 0) r = r && bar_test(wbar(w, W_ODONE), (pv_unit - 1) & 1);
+      return r;
     };
     auto do_pv = [&](bool seen) -> bool {
-      const int vs = pv_j % kKVS;               // (its K and V arrived together)
-      const uint32_t vb = base + vs * kPair + kStage;
+      const int vs = pv_j % kVS;
+      const uint32_t vb = base + kOffV + vs * kStage;
       const int nk = min(kTileBlk, (pv_tok - pv_t * kTile + kBlock - 1) / kBlock);
       if (!__all_sync(kAll, seen)) {
         bool w8 = bar_wait(wbar(w, W_PFULL + (pg & 1)), (pg >> 1) & 1, cta_abort, a.d_error,
                            17300 + w);
+        w8 = w8 && bar_wait(bar(B_VFULL + vs), (pv_j / kVS) & 1, cta_abort, a.d_error, 17200 + w);
         if (pv_t == 0 && pv_unit > 0)           // the unit before has read its O out
           w8 = w8 && bar_wait(wbar(w, W_ODONE), (pv_unit - 1) & 1, cta_abort, a.d_error, 17400 + w);
         if (!__all_sync(kAll, w8)) return false;
@@ -380,10 +424,13 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
                          kIdescPV, kk ? 1u : acc0);
         }
         umma_commit(wbar(w, W_PFREE + (pg & 1)));
-        umma_commit(bar(B_KVEMPTY + vs));       // this warpgroup is done with the tile
+        umma_commit(bar(B_VEMPTY + vs));        // this warpgroup is done with the V tile
         if (pv_last) bar_arrive(bar(B_DEMPTY + pv_unit % kDescRing));
       }
       ++pg;
+      // (a look at the next tile's K, for the next step: the products just issued run while
+      // the answer comes)
+      k_seen = bar_test(bar(B_KFULL + (pv_j + 2) % kKS), ((pv_j + 2) / kKS) & 1);
       return true;
     };
     for (int u = 0; ok; ++u) {
@@ -398,27 +445,32 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
       const int chain_tok = __shfl_sync(kAll, d->chain_tok, 0);
       const uint64_t qd = smem_desc(base + kOffQ + ((u & 1) * 2 + w) * kQBytes, 16, 1024);
       for (int t = 0; t < n_tiles; ++t, ++j) {
-        const int s = j % kKVS;
+        const int s = j % kKS;
         if (t >= my_tiles) {
           // beyond this warpgroup's last row: the P V that is still due, and the tile is let go
-          kv_seen = false;
           if (pv_j >= 0 && !do_pv(false)) {
             ok = false;
             break;
           }
           pv_j = -1;
-          // (the tile's copies have been requested, so the stage's release before this one
-          // is complete: this arrival cannot be counted for it)
-          if (!__all_sync(kAll, bar_wait(bar(B_KVFULL + s), (j / kKVS) & 1, cta_abort, a.d_error,
-                                         17600))) {
+          k_seen = false;
+          // (the tile's copies have been requested, so the releases before these of the two
+          // stages are complete: these arrivals cannot be counted for them)
+          if (!__all_sync(kAll, bar_wait(bar(B_KFULL + s), (j / kKS) & 1, cta_abort, a.d_error,
+                                         17600) &&
+                                    bar_wait(bar(B_VFULL + j % kVS), (j / kVS) & 1, cta_abort,
+                                             a.d_error, 17601))) {
             ok = false;
             break;
           }
-          if (lead) bar_arrive(bar(B_KVEMPTY + s));
+          if (lead) {
+            bar_arrive(bar(B_KEMPTY + s));
+            bar_arrive(bar(B_VEMPTY + j % kVS));
+          }
           continue;
         }
-        if (!__all_sync(kAll, kv_seen) || t == 0) {
-          bool w8 = bar_wait(bar(B_KVFULL + s), (j / kKVS) & 1, cta_abort, a.d_error, 17100);
+        if (!__all_sync(kAll, k_seen) || t == 0) {
+          bool w8 = bar_wait(bar(B_KFULL + s), (j / kKS) & 1, cta_abort, a.d_error, 17100);
           if (t == 0)
             w8 = w8 && bar_wait(bar(B_QFULL + (u & 1)), (u >> 1) & 1, cta_abort, a.d_error, 17500);
           if (!__all_sync(kAll, w8)) {
@@ -426,10 +478,10 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
             break;
           }
         }
-        kv_seen = false;                          // (set again by the look below)
+        k_seen = false;
         tc_fence_after();
         if (lead) {
-          const uint64_t kd = smem_desc(base + s * kPair, 16, 1024);
+          const uint64_t kd = smem_desc(base + s * kStage, 16, 1024);
           const uint32_t sd = tm_w + 64u * (qg & 1);
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)
@@ -437,6 +489,7 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
                       kd + (uint64_t)(((ks >> 2) * kStageHalf + (ks & 3) * 32) >> 4), kIdescQK,
                       ks > 0);
           umma_commit(wbar(w, W_SFULL + (qg & 1)));
+          umma_commit(bar(B_KEMPTY + s));         // this warpgroup is done with the K tile
           if (t == my_tiles - 1) umma_commit(bar(B_QEMPTY + (u & 1)));   // done with the unit's rows
         }
         ++qg;
@@ -508,11 +561,16 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
           for (int j = 0; j < 64; ++j)
             if (j >= see) sr[j] = 0xff800000u;
         }
-        float mx = -INFINITY;
+        // (four independent chains: one chain of 64 would wait for itself)
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int j = 0; j < 64; j += 2)
-          mx = fmaxf(mx, fmaxf(__uint_as_float(sr[j]), __uint_as_float(sr[j + 1])));
-        mx *= cc;
+        for (int j = 0; j < 64; j += 8) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            mx4[e] = fmaxf(mx4[e], fmaxf(__uint_as_float(sr[j + 2 * e]),
+                                         __uint_as_float(sr[j + 2 * e + 1])));
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * cc;
         const bool move = mx > ref + kSlack || ref == -INFINITY;
         const float ref_new = move ? mx : ref;
         const bool rescale = t > 0 && __any_sync(0xffffffffu, move);
@@ -541,13 +599,15 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         }
         ref = ref_new;
         uint32_t pk[32];
+        float l4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           const float p0 = ex2(fmaf(__uint_as_float(sr[2 * j]), cc, -ref));
           const float p1 = ex2(fmaf(__uint_as_float(sr[2 * j + 1]), cc, -ref));
-          l += p0 + p1;
+          l4[j & 3] += p0 + p1;
           pk[j] = pack2(p0, p1);
         }
+        l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
         // P takes the place of the scores it was made from
         TMEM_ST_32((tm_s + 64u * b) | lane_sel, pk);
         tmem_wait_st();
@@ -556,12 +616,12 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         // the unit's last tile: each before its own P is handed over.
         const int tile_tok = chain_tok - t * kTile;
         if (tile_tok < kTile && wq == 0) {
-          const int vt = all0 + t, vs = vt % kKVS;
-          if (!bar_wait(bar(B_KVFULL + vs), (vt / kKVS) & 1, cta_abort, a.d_error, 14000 + t % 1000)) {
+          const int vt = all0 + t, vs = vt % kVS;
+          if (!bar_wait(bar(B_VFULL + vs), (vt / kVS) & 1, cta_abort, a.d_error, 14000 + t % 1000)) {
             alive = false;
             break;
           }
-          uint8_t* vptr = bp + vs * kPair + kStage;
+          uint8_t* vptr = bp + kOffV + vs * kStage;
           const int last = ((tile_tok + kBlock - 1) / kBlock) * kBlock;
           for (int x = lane; x < (last - tile_tok) * 16; x += 32)
             *(uint4*)(vptr + kv_off(tile_tok + (x >> 4), x & 15)) = make_uint4(0u, 0u, 0u, 0u);
@@ -635,7 +695,7 @@ cudaError_t launch_attention_prefill(const AttnArgs& a, const CUtensorMap* tm_q,
   }
   const long long n_units = (long long)n_items * a.shape.num_kv_heads;
   const int grid = (int)std::min<long long>(n_units, a.num_sms);
-  return launch_kernel(attn_prefill_kernel, dim3(grid), dim3(352), kSmemPrefill, st, false, *a.tm_k,
+  return launch_kernel(attn_prefill_kernel, dim3(grid), dim3(384), kSmemPrefill, st, false, *a.tm_k,
                        *a.tm_v, *tm_q, a, d_items, n_items, a.d_ticket);
 }
 
