@@ -663,7 +663,7 @@ def run_prefill(args):
                      "frac": achieved / peak_tf, "traffic": None,
                      "peak_kind": f"cuBLAS bf16 GEMM, {peak_kind}",
                      "flops_per_step": flops, "attention_ms": attn_ms,
-                     "kernel": "tcgen05 kernel, tree-mask form (64-row query tiles)"},
+                     "kernel": "attn_prefill_kernel: tcgen05, 2 x 128 query rows per CTA share the K/V tiles"},
         "tree_mask": {"workload": "every token of a config-3-shaped forest of 64 requests",
                       "queries": nq, "segments": len(segs), "ms": tree_ms,
                       "tflops": t_flops / (tree_ms * 1e-3) / 1e12,

@@ -232,12 +232,12 @@ apar_status apar_accept_candidates(apar_ctx* ctx, int32_t n, const int32_t* tid 
  * must already be in the pool: append first); the query at position p attends positions
  * 0 .. p of that thread's chain.  A prompt is one segment from position 0; every node of a
  * paragraph tree is one segment of its thread that starts where the node's own tokens start.
- * q, out [device] bf16 [sum q_count][num_q_heads][128], segments in order.  The queries of a
- * segment are processed 64 rows at a time (64 / group tokens x group heads) on the tensor
- * cores; a tile reads its chain once for all of its rows and masks every row at its own
- * position.  Any number of queries per call (they are launched in batches that fit the
- * workspace); `layer` selects the pool layer.  Invalidates the cached decode plan.
- * Errors: INVALID_ARG (also a range outside the thread), BAD_THREAD, CUDA. */
+ * q, out [device] bf16 [sum q_count][num_q_heads][128], segments in order, q 16-byte aligned
+ * (it is read by TMA).  The queries of a segment are processed 256 rows at a time
+ * (2 * (128 / group) tokens x group heads) on the tensor cores; a tile reads its chain once
+ * for all of its rows and masks every row at its own position.  Any number of queries per
+ * call; `layer` selects the pool layer.  Invalidates the cached decode plan.
+ * Errors: INVALID_ARG (also a range outside the thread, or a misaligned q), BAD_THREAD, CUDA. */
 apar_status apar_tree_prefill_attention(apar_ctx* ctx, int32_t layer, int32_t n,
                                         const int32_t* tid /*[host]*/,
                                         const int32_t* q_begin /*[host]*/,

@@ -122,8 +122,8 @@ struct apar_ctx {
   int umma_heads = 0;                   // > 0: kv heads per CTA of the tcgen05 kernel (testing)
   int umma_mode = 0;                    // 1: one CTA per (item, heads); 2: persistent CTAs
   int ws_mode = 0;                      // 1: one CTA per item; 2: persistent warps
-  int prefill_rows = 128;               // query rows per tensor-core tile of tree-masked attention
-  int64_t prefill_batch = INT64_MAX;    // work items per launch of it, at most (testing)
+  int64_t prefill_batch = INT64_MAX;    // tree-masked attention: work items per launch, at most
+                                        // (testing)
   int num_sms = 148;
   int use_pdl = 1;                      // warp-stream launches may start before the kernel before
                                         // them has finished (0: ordinary launches only)
@@ -623,9 +623,8 @@ apar_status create_impl(const apar_config* cfg, bool external, bool host_only, a
   c->umma_mode = (mode && !strcmp(mode, "grid")) ? 1 : (mode && !strcmp(mode, "persist")) ? 2 : 0;
   mode = getenv("APAR_WS_MODE");                         // "grid" | "persist"
   c->ws_mode = (mode && !strcmp(mode, "grid")) ? 1 : (mode && !strcmp(mode, "persist")) ? 2 : 0;
-  mode = getenv("APAR_PREFILL");                         // "m64" | "m128": rows per MMA tile
-  c->prefill_rows = (mode && !strcmp(mode, "m64")) ? 64 : 128;
-  mode = getenv("APAR_PREFILL_BATCH");                   // work items per launch, at most
+  mode = getenv("APAR_PREFILL_BATCH");                   // tree-masked attention: work items per
+                                                         // launch, at most
   if (mode && atoll(mode) > 0) c->prefill_batch = atoll(mode);
   c->auto_path = !path || !strcmp(path, "auto") || !*path;
   const char* planner = getenv("APAR_PLANNER");          // testing: "tables" = per-block walk
@@ -1247,13 +1246,11 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
   if (rc) return rc;
   c->attn_book_seq = 0;                 // layer replays of a decode plan need a decode call
 
-  // Work items: the queries of a segment in tiles of 256 rows (2 * (128 / group) tokens; 64
-  // rows with the older kernel); a tile reads the chain from its start to the tile's last token
-  // once, for all of its rows, and every row stops at its own position (the mask is applied by
-  // the kernel).
+  // Work items: the queries of a segment in tiles of 256 rows (2 * (128 / group) tokens); a
+  // tile reads the chain from its start to the tile's last token once, for all of its rows,
+  // and every row stops at its own position (the mask is applied by the kernel).
   const int G = c->shape.group;
-  const bool wide = c->prefill_rows == 128;
-  const int per_tile = wide ? 2 * (128 / G) : std::max(1, kMaxRowsPerItem / G);
+  const int per_tile = 2 * (128 / G);
   struct Tile { int32_t seg, first, count; };
   std::vector<Tile> tiles;
   for (int i = 0; i < n; ++i)
@@ -1289,14 +1286,10 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
   a.d_lens = (const int32_t*)c->ws(c->lay.lens);
   // Every tile covers its rows' whole chains, so no partial results are written: the area
   // that holds them in decode calls (by far the largest part of the workspace) takes this
-  // call's work items and user entries instead, first half users, second half items.
+  // call's work items instead.
   const size_t area = (size_t)c->lay.slot_capacity * c->shape.num_q_heads * kDim * sizeof(float);
-  const int64_t cap = std::min<int64_t>(
-      c->prefill_batch, (int64_t)(area / 2 / std::max(sizeof(UserRef), sizeof(WorkItem))));
-  char* d_users = c->ws(c->lay.part_o);
-  char* d_items = d_users + area / 2;
-  a.d_items = (const WorkItem*)d_items;
-  a.d_users = (const UserRef*)d_users;
+  const int64_t cap = std::min<int64_t>(c->prefill_batch, (int64_t)(area / sizeof(PrefillItem)));
+  char* d_items = c->ws(c->lay.part_o);
   a.part_o = nullptr;
   a.part_ml = nullptr;
   a.shape = c->shape;
@@ -1306,7 +1299,9 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
   a.d_error = (int*)c->ws(c->lay.err);
   a.num_sms = c->num_sms;
   a.d_ticket = (int*)c->ws(c->lay.ticket);
-  a.causal = true;                      // each user entry carries its query's visible length
+  CUtensorMap tm_q;
+  if (make_query_tensor_map(q, total_q, c->shape.num_q_heads, G, &tm_q) != 0)
+    return APAR_ERR_INVALID_ARG;        // (a query array that is not 16-byte aligned)
 
   auto upload = [&](const void* src, size_t bytes, char* dst) -> apar_status {
     size_t done = 0;
@@ -1322,59 +1317,23 @@ apar_status apar_tree_prefill_attention(apar_ctx* c, int32_t layer, int32_t n,
     }
     return APAR_OK;
   };
-  std::vector<WorkItem> items;
-  std::vector<UserRef> users;
-  std::vector<PrefillItem> wide_items;
+  std::vector<PrefillItem> items;
   int launches = 0;
   c->last.attn_work_items = 0;
   size_t t0 = 0;
-  CUtensorMap tm_q;
-  if (wide && make_query_tensor_map(q, total_q, c->shape.num_q_heads, G, &tm_q) != 0)
-    return APAR_ERR_INVALID_ARG;        // (a query array that is not 16-byte aligned)
-  while (wide && t0 < tiles.size()) {   // 128-row tiles: an item is four numbers, no user list
+  while (t0 < tiles.size()) {           // (one launch unless the list outgrows its area)
     const size_t t1 = (size_t)std::min<int64_t>((int64_t)tiles.size(), (int64_t)t0 + cap);
-    wide_items.clear();
+    items.clear();
     for (size_t i = t0; i < t1; ++i) {
       const Tile& t = tiles[i];
-      wide_items.push_back(PrefillItem{seg_slot[t.seg], (int32_t)(seg_qbase[t.seg] + t.first),
-                                       q_begin[t.seg] + t.first, t.count});
+      items.push_back(PrefillItem{seg_slot[t.seg], (int32_t)(seg_qbase[t.seg] + t.first),
+                                  q_begin[t.seg] + t.first, t.count});
     }
-    rc = upload(wide_items.data(), wide_items.size() * sizeof(PrefillItem), d_items);
+    rc = upload(items.data(), items.size() * sizeof(PrefillItem), d_items);
     if (rc) return rc;
     if (c->time_start && t0 == 0) APAR_CUDA(c, cudaEventRecord(c->time_start, st));
-    APAR_CUDA(c, launch_attention_prefill(a, &tm_q, (const PrefillItem*)d_items,
-                                          (int)wide_items.size(), st));
-    ++launches;
-    c->last.attn_work_items += (int64_t)wide_items.size();
-    t0 = t1;
-  }
-  while (t0 < tiles.size()) {
-    items.clear();
-    users.clear();
-    size_t t1 = t0;
-    while (t1 < tiles.size() && (int64_t)users.size() + tiles[t1].count <= cap &&
-           (int64_t)items.size() < cap) {
-      const Tile& t = tiles[t1];
-      WorkItem it;
-      it.table_row = seg_slot[t.seg];
-      it.tok_begin = 0;
-      it.tok_end = q_begin[t.seg] + t.first + t.count;
-      it.user_begin = (int32_t)users.size();
-      it.n_users = t.count;
-      it.slot_add = 0;
-      it.fin_n = it.fin_begin = 0;
-      items.push_back(it);
-      for (int k = 0; k < t.count; ++k)
-        users.push_back(UserRef{(int32_t)(seg_qbase[t.seg] + t.first + k),
-                                -1 - (q_begin[t.seg] + t.first + k + 1)});
-      ++t1;
-    }
-    rc = upload(items.data(), items.size() * sizeof(WorkItem), d_items);
-    if (rc) return rc;
-    rc = upload(users.data(), users.size() * sizeof(UserRef), d_users);
-    if (rc) return rc;
-    if (c->time_start && t0 == 0) APAR_CUDA(c, cudaEventRecord(c->time_start, st));
-    APAR_CUDA(c, launch_attention_umma(a, 0, (int)items.size(), st));
+    APAR_CUDA(c, launch_attention_prefill(a, &tm_q, (const PrefillItem*)d_items, (int)items.size(),
+                                          st));
     ++launches;
     c->last.attn_work_items += (int64_t)items.size();
     t0 = t1;

@@ -165,9 +165,6 @@ struct AttnArgs {
   int umma_heads = 0;                 // > 0: kv heads per CTA of the tcgen05 kernel (testing)
   int umma_mode = 0;                  // tcgen05 kernel: 0 default, 1 one CTA per (item, heads),
                                       // 2 persistent CTAs that claim units from *d_ticket
-  // tree-mask (prefill) form of the tcgen05 kernel: every user entry carries slot = -1 - L,
-  // L = how many tokens of the chain that query sees (its position + 1)
-  bool causal = false;
   int ws_mode = 0;                    // warp-stream kernel: 0 default, 1 one CTA per item, 2 persistent
   int* d_ticket = nullptr;            // [device] counters of the persistent forms, zero when no
                                       // launch is in flight: words 0-2 tcgen05 kernel, 4-6 and

@@ -5,17 +5,26 @@
 // thread times the group's query heads - and the chain they attend, from its first token to the
 // last query's own position.  One persistent CTA per SM claims units from a device counter.
 //   warps 0-3 and 4-7  two softmax warpgroups.  Warpgroup w owns the unit's tokens
-//              w * (128 / group) onward: its own Q operand, its own S (double-buffered) and O
-//              accumulators in TMEM, its own P operand.  Row r of a warpgroup is TMEM lane r, so
-//              one thread owns one whole row: the row maximum and sum need no shuffles.  Every
-//              row is masked at its own position.
-//   warp 8     producer: TMA copies of 64-token K and V tiles into two rings; claims the next
-//              unit in the background (one phase of that fetch per tile issued).
-//   warp 9     one thread issues, per 64-token tile and warpgroup, S = Q K^T (M 128, N 64,
-//              K 128) and O += P V (M 128, N 128, K 64) with tcgen05.mma.  K and V tiles are
-//              shared by the two warpgroups: a 32 KiB tile pair feeds 256 query rows.  The
-//              first warpgroup's rows end earlier in the chain than the second's; it skips the
-//              tiles beyond its last row.
+//              w * (128 / group) onward: its own Q operand in shared memory, its own S
+//              (double-buffered) and O accumulators in tensor memory.  Row r of a warpgroup is
+//              TMEM lane r, so one thread owns one whole row: the row maximum and sum need no
+//              shuffles.  Every row is masked at its own position.  P (bf16) is written over the
+//              first half of the S buffer it was made from and read from there by the MMA.
+//   warp 8     claims units (one phase of that fetch per tile issued, so that its memory
+//              round trips pass in the background) and copies, by TMA, the units' query rows
+//              (double-buffered) and their 64-token K tiles into a ring.
+//   warp 11    copies the V tiles into a second ring.
+//   warps 9, 10  one MMA issuer per warpgroup (lane 0 issues): per K/V tile S = Q K^T (M 128,
+//              N 64, K 128) and, one tile behind, O += P V (M 128, N 128, K 64, A operand in
+//              tensor memory).  K and V tiles are shared by the two warpgroups: a 32 KiB tile
+//              pair feeds 256 query rows.  The first warpgroup's rows end earlier in the chain
+//              than the second's; it skips the tiles beyond its last row.
+// Why the roles are cut this way (measured, cycles of the SM clock): a tcgen05.mma holds its
+// issuing thread until the tensor pipe takes it (M 128 x N 64 x K 16 every 48 cycles, N 128
+// every 64), a look at an mbarrier costs a thread 100-250 cycles on a busy SM, and a warp's
+// tensor copy instruction about 70 cycles per 2 KiB box.  So two threads issue MMAs (one keeps
+// the pipe busy while the other synchronises), each looks at its next step's barriers before
+// it needs the answer, and the sixteen boxes of a tile pair are issued by two warps.
 // All waits are bounded; a wait that gives up raises the error word and every role unwinds to
 // the common exit where TMEM is released.
 #include <algorithm>

@@ -538,11 +538,6 @@ constexpr int kSmemP = kDescOff + kDescSlots * (int)sizeof(UnitDesc) + 1024;
 enum BarP { DFULL0 = NBARS, DEMPTY0 = DFULL0 + kDescSlots, NBARS_P = DEMPTY0 + kDescSlots };
 static_assert(8 * NBARS_P + 16 <= 256, "barrier area");
 
-// kCausal: every query has its own visible length L in chain positions (its user entry carries
-// slot = -1 - L: negative, so the row is written out as a final result): a key at or beyond L
-// is masked out for that row.  This is the tree mask of prefill / training
-// attention, where the queries of a unit are consecutive tokens of one node.
-template <bool kCausal>
 __global__ void __launch_bounds__(192, 2)
 attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
                          const __grid_constant__ CUtensorMap tm_v, const AttnArgs a,
@@ -631,10 +626,8 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
         if (f_tick >= n_units) {
           f_phase = 3;                              // publish the end mark
         } else {
-          // Decode: a unit's kv heads follow each other (they walk the same block ids).  Tree
-          // mask: the query tiles of one head follow each other - the tiles of a segment read
-          // the same K and V, so the units that run at the same time share them in L2.
-          const int item = kCausal ? f_tick % (n_units / HKV) : f_tick / HKV;
+          // a unit's kv heads follow each other (they walk the same block ids)
+          const int item = f_tick / HKV;
           const int4* ip = (const int4*)(a.d_items + item_begin + item);
           if (lane < 2) f_item = __ldg(ip + lane);
           f_phase = 2;
@@ -672,7 +665,7 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
             d->tok_begin = f_tok_begin;
             d->n_tok = tok_end - f_tok_begin;
             d->n_tiles = (tok_end - f_tok_begin + kTileTok - 1) / kTileTok;
-            d->kvh = kCausal ? f_tick / (n_units / HKV) : f_tick % HKV;
+            d->kvh = f_tick % HKV;
             d->n_users = f_n_users;
             d->slot_add = f_slot_add;
           }
@@ -876,15 +869,8 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
     const int g8 = lane >> 2, qd = lane & 3;
     // rows 16w .. 16w+15 of unit description d into the A-operand layout (rows past the unit's
     // own as zeros)
-    int lim_lo_next = 0, lim_hi_next = 0;             // visible keys of rows g8 / g8 + 8,
-                                                      // relative to the unit's first token
     auto stage_q = [&](const UnitDesc* d) {
       const int R = d->n_users * G, kvh = d->kvh;
-      if (kCausal) {
-        const int r_lo = warp * 16 + g8, r_hi = r_lo + 8;
-        lim_lo_next = r_lo < R ? -d->users[r_lo / G].slot - 1 - d->tok_begin : d->n_tok;
-        lim_hi_next = r_hi < R ? -d->users[r_hi / G].slot - 1 - d->tok_begin : d->n_tok;
-      }
       uint4 qv[8];
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
@@ -911,7 +897,6 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
       const int n_tiles = d->n_tiles;
       if (n_tiles == 0) break;
       const int n_tok = d->n_tok, R = d->n_users * G, kvh = d->kvh, slot_add = d->slot_add;
-      const int lim_lo = lim_lo_next, lim_hi = lim_hi_next;    // (of this unit: staged with its Q)
       float ref_lo = -INFINITY, ref_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
       for (int t = 0; t < n_tiles; ++t) {
         const int g = g0 + t, b = g & 1;
@@ -927,25 +912,21 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
         __syncwarp();
         if (lane == 0) bar_arrive(bar(SFREE0 + b));
         const int tile_tok = min(kTileTok, n_tok - t * kTileTok);
-        // keys of this tile a row may see: all that exist, or (tree mask) those before its limit
-        const int see_lo = kCausal ? min(tile_tok, lim_lo - t * kTileTok) : tile_tok;
-        const int see_hi = kCausal ? min(tile_tok, lim_hi - t * kTileTok) : tile_tok;
         // The raw scores stay in registers; the scale is applied to the row maximum and, fused
-        // with the subtraction of the reference, inside the exponent.  A key a row may not see
-        // becomes -inf (rows of K past the valid length hold unspecified bits); tiles that are
-        // visible in full to every row of the warp skip that pass.  (A scale that is not
-        // positive is applied up front, so that the maximum of the raw values is the maximum.)
+        // with the subtraction of the reference, inside the exponent.  A key past the unit's
+        // last token becomes -inf (rows of K past the valid length hold unspecified bits); full
+        // tiles skip that pass.  (A scale that is not positive is applied up front, so that the
+        // maximum of the raw values is the maximum.)
         if (!(c > 0.f)) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) sr[j] = __float_as_uint(__uint_as_float(sr[j]) * c);
         }
-        if (!__all_sync(0xffffffffu, see_lo >= kTileTok && see_hi >= kTileTok)) {
+        if (tile_tok < kTileTok) {
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-              if (8 * k + 2 * qd + e >= see_lo) sr[4 * k + e] = 0xff800000u;
-              if (8 * k + 2 * qd + e >= see_hi) sr[4 * k + 2 + e] = 0xff800000u;
+              if (8 * k + 2 * qd + e >= tile_tok) sr[4 * k + e] = sr[4 * k + 2 + e] = 0xff800000u;
             }
           }
         }
@@ -1125,10 +1106,7 @@ cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items
     cudaError_t e = cudaFuncSetAttribute(attn_umma_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_umma_persist_kernel<false>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemP);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(attn_umma_persist_kernel<true>,
+    e = cudaFuncSetAttribute(attn_umma_persist_kernel,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemP);
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
@@ -1136,16 +1114,12 @@ cudaError_t launch_attention_umma(const AttnArgs& a, int item_begin, int n_items
     configured[dev] = true;
   }
   const int hkv = a.shape.num_kv_heads;
-  if (a.causal && a.d_ticket == nullptr) return cudaErrorInvalidValue;
-  if ((a.umma_mode != 1 || a.causal) && a.d_ticket != nullptr) {
+  if (a.umma_mode != 1 && a.d_ticket != nullptr) {
     // persistent form: two resident CTAs per SM claim (item, kv head) units from a counter
     const long long n_units = (long long)n_items * hkv;
     const int grid = (int)std::min<long long>(n_units, 2LL * sm_count[dev]);
-    if (a.causal)
-      return launch_kernel(attn_umma_persist_kernel<true>, dim3(grid), dim3(192), kSmemP, st,
-                           a.pdl != 0, *a.tm_k, *a.tm_v, a, item_begin, (int)n_units, a.d_ticket);
-    return launch_kernel(attn_umma_persist_kernel<false>, dim3(grid), dim3(192), kSmemP, st,
-                         a.pdl != 0, *a.tm_k, *a.tm_v, a, item_begin, (int)n_units, a.d_ticket);
+    return launch_kernel(attn_umma_persist_kernel, dim3(grid), dim3(192), kSmemP, st, a.pdl != 0,
+                         *a.tm_k, *a.tm_v, a, item_begin, (int)n_units, a.d_ticket);
   }
   // Heads per CTA: up to kHeadsMax, if that leaves at least kWavesMin CTAs for each of the
   // machine's CTA slots (two per SM), so that the hardware scheduler can still even out the

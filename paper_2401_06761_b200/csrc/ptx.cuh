@@ -55,15 +55,6 @@ __device__ __forceinline__ bool bar_wait(uint32_t bar, uint32_t parity, volatile
   atomicCAS(err_word, 0, code);
   return false;
 }
-// The same for a whole (converged) warp: lane 0 waits, the others take the outcome from it.
-// 32 lanes polling one barrier cost some hundreds of cycles even when the phase is complete.
-__device__ __forceinline__ bool bar_wait_warp(uint32_t bar, uint32_t parity,
-                                              volatile int* cta_abort, int* err_word, int code) {
-  int ok = 1;
-  if ((threadIdx.x & 31) == 0) ok = bar_wait(bar, parity, cta_abort, err_word, code);
-  __syncwarp();
-  return __shfl_sync(0xffffffffu, ok, 0) != 0;
-}
 // One box of a 2-D tensor map into shared memory; completion is counted on `bar`.
 __device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
                                        uint32_t bar) {
