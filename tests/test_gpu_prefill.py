@@ -80,6 +80,11 @@ def test_every_token_of_a_paragraph_tree(hq, hkv):
         with pytest.raises(B.AparError) as e:
             sess.prefill_attention(*bad, qd[:1].contiguous())
         assert e.value.code == "INVALID_ARG"
+    # the queries are read by TMA: an array that does not start on a 16-byte boundary is refused
+    flat = torch.zeros(hq * 128 + 8, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.AparError) as e:
+        sess.prefill_attention([tids[0]], [0], [1], flat[1:1 + hq * 128].view(1, hq, 128))
+    assert e.value.code == "INVALID_ARG"
     sess.close()
 
 
