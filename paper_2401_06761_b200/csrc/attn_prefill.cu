@@ -326,6 +326,15 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
         }
       }
     }
+    // After a wait that gave up, the copies this warp still has in flight are waited for (with
+    // a limit of their own) before the CTA's shared memory goes away.  (Otherwise every copy
+    // has been consumed: its consumer waited for it.)
+    if (*cta_abort && lane == 0) {
+      for (int g = max(0, kg - kKS); g < kg; ++g)
+        for (uint32_t i = 0; i < kSpin && !bar_try(bar(B_KFULL + g % kKS), (g / kKS) & 1); ++i) {}
+      for (int x = max(0, qu - 2); x < qu; ++x)
+        for (uint32_t i = 0; i < kSpin && !bar_try(bar(B_QFULL + (x & 1)), (x >> 1) & 1); ++i) {}
+    }
     // ticket[0] unit counter, ticket[1] producers that have stopped claiming: the last one puts
     // both back to zero, so that nothing has to be cleared between launches
     if (lane == 0) {
@@ -376,6 +385,9 @@ attn_prefill_kernel(const __grid_constant__ CUtensorMap tm_k,
                  &tm_v, (lane & 1) * 64, (bid * HKV + kvh) * kBlock, bar(B_VFULL + s));
       }
     }
+    if (*cta_abort && lane == 0)      // (as in the K producer: copies in flight after a give-up)
+      for (int g = max(0, vg - kVS); g < vg; ++g)
+        for (uint32_t i = 0; i < kSpin && !bar_try(bar(B_VFULL + g % kVS), (g / kVS) & 1); ++i) {}
   } else if (warp >= 9) {
     // ---------------------------------------------------------------- MMA issuers
     // One warp per warpgroup of query rows (warp 9: the first, warp 10: the second), each with

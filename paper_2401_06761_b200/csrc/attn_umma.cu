@@ -225,6 +225,14 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
       }
     }
+    // After a wait that gave up, the copies still in flight are waited for (with a limit of
+    // their own) before the CTA's shared memory goes away.
+    if (*cta_abort && lane == 0) {
+      for (int g = max(0, k_next - kKStages); g < k_next; ++g)
+        for (uint32_t i = 0; i < kSpin && !bar_try(bar(KFULL0 + g % kKStages), (g / kKStages) & 1); ++i) {}
+      for (int g = max(0, v_next - kVStages); g < v_next; ++g)
+        for (uint32_t i = 0; i < kSpin && !bar_try(bar(VFULL0 + g % kVStages), (g / kVStages) & 1); ++i) {}
+    }
   } else if (warp == 5) {
     // ---------------------------------------------------------------- MMA issuer
     constexpr uint32_t kIdescQK = instr_desc(kTileTok, false);
@@ -770,6 +778,15 @@ attn_umma_persist_kernel(const __grid_constant__ CUtensorMap tm_k,
           break;
         }
       }
+    }
+    // After a wait that gave up, the copies this warp still has in flight are waited for (with
+    // a limit of their own) before the CTA's shared memory goes away.  (Otherwise every copy
+    // has been consumed: its consumer waited for it.)
+    if (*cta_abort && lane == 0) {
+      for (int g = max(0, kg - kKStages); g < kg; ++g)
+        for (uint32_t i = 0; i < kSpin && !bar_try(bar(KFULL0 + g % kKStages), (g / kKStages) & 1); ++i) {}
+      for (int g = max(0, vg - kVStages); g < vg; ++g)
+        for (uint32_t i = 0; i < kSpin && !bar_try(bar(VFULL0 + g % kVStages), (g / kVStages) & 1); ++i) {}
     }
     // ticket[0] unit counter, ticket[1] producers that have stopped claiming: the last one puts
     // both back to zero, so that nothing has to be cleared between launches
